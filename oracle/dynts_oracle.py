@@ -1,0 +1,270 @@
+"""Float64 CPU oracle for budget-limited decode attention, importance accumulation and eviction.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain statement of what the hot path
+computes.  It shares no code with the CUDA library and must never be imported by the product
+package; only the tests, the smoke check and the benchmark's CPU-baseline leg use it.
+
+What each function follows in the paper:
+
+* ``attention_weights`` / ``decode_step`` -- token-level attention of the decode query over the
+  retained cache, Eq. 4 (softmax of q.k/sqrt(d_k) over every cached position, the new one
+  included) and Eq. 5 (weighted sum of values).
+* ``decode_step`` (delta/score part) -- Eq. 6: a token's importance is the attention it receives
+  summed over query rows.  Here the rows are the decode queries seen so far, summed over the
+  query heads that share the KV head (Appendix B.1 aggregates heads; sum is this build's reading).
+* ``select_keep`` / ``evict`` -- Section 4.2: the question window (the first M rows) and the local
+  window (the last W rows) are always retained, the top-k of the selection window by score are
+  retained, the rest are evicted.  Ties go to the lower index; retained rows keep their order.
+* ``eviction_count`` / ``effective_length`` -- Section 5, the closed form for the cache length.
+* ``attn_flops`` / ``predictor_flops`` / ``break_even_volume`` -- Appendix A and Eq. 9-10.
+
+Pinned by tests/test_oracle_*.py against a library attention routine, closed forms, brute-force
+ranking and the values the paper prints.  Parity unpinned: the synthetic "planted critical key"
+input recipe (it is an input distribution, not part of the method).
+"""
+from __future__ import annotations
+
+import math
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+
+# ----------------------------------------------------------------------------------------------
+# Eq. 4-5: attention of one query head over n cached rows
+# ----------------------------------------------------------------------------------------------
+
+def attention_weights(q: np.ndarray, K: np.ndarray) -> np.ndarray:
+    """alpha_j = exp(e_j) / sum_i exp(e_i), e_j = q.k_j / sqrt(d_k)   (Eq. 4).
+
+    q: [G, d] query heads of one group, K: [n, d].  Returns alpha [G, n] in float64.
+    The row maximum is subtracted before exponentiation; this leaves Eq. 4 unchanged.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    d_k = K.shape[1]
+    e = (q @ K.T) / math.sqrt(d_k)
+    e = e - e.max(axis=1, keepdims=True)
+    p = np.exp(e)
+    return p / p.sum(axis=1, keepdims=True)
+
+
+def attention_output(alpha: np.ndarray, V: np.ndarray) -> np.ndarray:
+    """o = sum_j alpha_j v_j   (Eq. 5).  alpha [G, n], V [n, d] -> [G, d]."""
+    return alpha @ np.asarray(V, dtype=np.float64)
+
+
+# ----------------------------------------------------------------------------------------------
+# Cache state
+# ----------------------------------------------------------------------------------------------
+
+class Slab:
+    """Retained rows of one (layer, sequence, KV head): K, V, original positions and scores."""
+
+    __slots__ = ("K", "V", "pos", "score", "n")
+
+    def __init__(self, capacity: int, d: int):
+        self.K = np.zeros((capacity, d), dtype=np.float64)
+        self.V = np.zeros((capacity, d), dtype=np.float64)
+        self.pos = np.zeros(capacity, dtype=np.int64)
+        self.score = np.zeros(capacity, dtype=np.float64)
+        self.n = 0
+
+
+class OracleCache:
+    def __init__(self, layers: int, batch: int, q_heads: int, kv_heads: int, head_dim: int,
+                 window: int, capacity: int):
+        assert q_heads % kv_heads == 0
+        self.layers, self.batch = layers, batch
+        self.q_heads, self.kv_heads, self.head_dim = q_heads, kv_heads, head_dim
+        self.group = q_heads // kv_heads
+        self.window = window
+        self.capacity = capacity
+        self.slabs = [[[Slab(capacity, head_dim) for _ in range(kv_heads)]
+                       for _ in range(batch)] for _ in range(layers)]
+        self.n_pinned = [0] * batch      # M: question rows, immune to eviction
+        self.next_pos = [0] * batch      # position id given to the next appended token
+
+    def slab(self, layer: int, seq: int, head: int) -> Slab:
+        return self.slabs[layer][seq][head]
+
+    def length(self, seq: int) -> int:
+        return self.slabs[0][seq][0].n
+
+    def units(self):
+        for l in range(self.layers):
+            for b in range(self.batch):
+                for h in range(self.kv_heads):
+                    yield l, b, h, self.slabs[l][b][h]
+
+
+def prefill(cache: OracleCache, k: np.ndarray, v: np.ndarray, n_pinned: Optional[int] = None,
+            seq: Optional[int] = None) -> None:
+    """Load prompt rows.  k, v: [L, Nb, Hkv, T, d] (or [L, Hkv, T, d] with ``seq`` given).
+
+    The first ``n_pinned`` rows (default: all T) are the question window; they get score +inf
+    (Section 4.2) and are never evicted.  The remaining rows start with score 0.
+    """
+    seqs = range(cache.batch) if seq is None else [seq]
+    for b in seqs:
+        T = k.shape[-2]
+        m = T if n_pinned is None else n_pinned
+        assert 0 <= m <= T <= cache.capacity
+        for l in range(cache.layers):
+            for h in range(cache.kv_heads):
+                s = cache.slabs[l][b][h]
+                src_k = k[l, b, h] if seq is None else k[l, h]
+                src_v = v[l, b, h] if seq is None else v[l, h]
+                s.K[:T] = src_k
+                s.V[:T] = src_v
+                s.pos[:T] = np.arange(T)
+                s.score[:T] = 0.0
+                s.score[:m] = np.inf
+                s.n = T
+        cache.n_pinned[b] = m
+        cache.next_pos[b] = T
+
+
+def decode_step(cache: OracleCache, q: np.ndarray, k_new: np.ndarray, v_new: np.ndarray,
+                active: Optional[Sequence[bool]] = None):
+    """One decode step for every (layer, sequence, KV head).
+
+    q [L, Nb, Hq, d]; k_new, v_new [L, Nb, Hkv, d].  For each slab: append the new row (its
+    score starts at 0), attend over all n rows including the new one (Eq. 4-5), add each row's
+    attention mass summed over the group's query heads to its score (Eq. 6).
+
+    Returns (out [L, Nb, Hq, d] float64, delta) where delta[l][b][h] is this step's mass per
+    row, an array of length n.
+    """
+    L, Nb, Hkv, G, d = cache.layers, cache.batch, cache.kv_heads, cache.group, cache.head_dim
+    out = np.zeros((L, Nb, cache.q_heads, d), dtype=np.float64)
+    delta = [[[None] * Hkv for _ in range(Nb)] for _ in range(L)]
+    for l, b, h, s in cache.units():
+        if active is not None and not active[b]:
+            continue
+        assert s.n < cache.capacity, "append past capacity: an eviction was skipped"
+        s.K[s.n] = k_new[l, b, h]
+        s.V[s.n] = v_new[l, b, h]
+        s.pos[s.n] = cache.next_pos[b]
+        s.score[s.n] = 0.0
+        s.n += 1
+        n = s.n
+        qg = q[l, b, h * G:(h + 1) * G]
+        alpha = attention_weights(qg, s.K[:n])                 # Eq. 4
+        out[l, b, h * G:(h + 1) * G] = attention_output(alpha, s.V[:n])   # Eq. 5
+        dl = alpha.sum(axis=0)                                 # Eq. 6, one more query row per head
+        s.score[:n] += dl
+        delta[l][b][h] = dl
+    for b in range(Nb):
+        if active is None or active[b]:
+            cache.next_pos[b] += 1
+    return out, delta
+
+
+# ----------------------------------------------------------------------------------------------
+# Section 4.2: budgeted selection
+# ----------------------------------------------------------------------------------------------
+
+def select_keep(score32: np.ndarray, n: int, n_pinned: int, window: int, target: int) -> np.ndarray:
+    """Indices (ascending) of the rows that survive an eviction down to ``target`` rows.
+
+    Rows [0, n_pinned) (question window) and [n - window, n) (local window) always survive.
+    Of the selection window [n_pinned, n - window) the k = target - n_pinned - window rows with
+    the highest score survive; equal scores are ranked by lower index first.  Scores are
+    compared as float32 values (the precision the scores are stored in on the device).
+    If n <= target nothing is evicted.
+    """
+    if n <= target:
+        return np.arange(n, dtype=np.int64)
+    k = target - n_pinned - window
+    if k < 0:
+        raise ValueError("question window + local window exceed the target length")
+    lo, hi = n_pinned, n - window
+    sc = np.asarray(score32[:n], dtype=np.float32)
+    ranked = sorted(range(lo, hi), key=lambda j: (-float(sc[j]), j))
+    kept = list(range(0, lo)) + sorted(ranked[:k]) + list(range(hi, n))
+    return np.asarray(kept, dtype=np.int64)
+
+
+def evict(cache: OracleCache, target, scores32=None):
+    """Evict every slab down to ``target`` rows (an int, or one int per sequence).
+
+    ``scores32(l, b, h)`` may supply the float32 score array the decision is taken from (used to
+    replay the device's decisions from the device's own scores); by default the slab's own
+    score, rounded to float32, decides.  Survivors are gathered in ascending index order into
+    rows [0, target); K, V, pos and score move together.
+
+    Returns kept[l][b][h] = the surviving row indices (before compaction).
+    """
+    L, Nb, Hkv = cache.layers, cache.batch, cache.kv_heads
+    kept_all = [[[None] * Hkv for _ in range(Nb)] for _ in range(L)]
+    for l, b, h, s in cache.units():
+        tgt = int(target if np.isscalar(target) else target[b])
+        sc = s.score[:s.n].astype(np.float32) if scores32 is None else scores32(l, b, h)
+        kept = select_keep(sc, s.n, cache.n_pinned[b], cache.window, tgt)
+        m = len(kept)
+        s.K[:m] = s.K[kept]
+        s.V[:m] = s.V[kept]
+        s.pos[:m] = s.pos[kept]
+        s.score[:m] = s.score[kept]
+        s.n = m
+        kept_all[l][b][h] = kept
+    return kept_all
+
+
+# ----------------------------------------------------------------------------------------------
+# Section 5 / Appendix A: closed forms
+# ----------------------------------------------------------------------------------------------
+
+def eviction_count(M: int, i: int, B: int, K: int) -> int:
+    """n_i = max(0, floor(((M + i) - B) / K) + 1): eviction events up to decode step i."""
+    return max(0, (M + i - B) // K + 1)
+
+
+def effective_length(M: int, i: int, B: int, K: int) -> int:
+    """S_i = M + i - n_i * K: cache length at decode step i when K rows leave at each event."""
+    return M + i - eviction_count(M, i, B, K) * K
+
+
+def attn_flops(L: int, d: int, S: int) -> int:
+    """Attention cost of one decode step over a cache of S rows: 4 * L * d * S (Appendix A)."""
+    return 4 * L * d * S
+
+
+def predictor_flops(d: int) -> int:
+    """MLP d -> 2d -> d/2 -> 1: 2*(d*2d + 2d*d/2 + d/2*1) = 6 d^2 + d (Appendix A)."""
+    return 2 * (d * (2 * d) + (2 * d) * (d // 2) + (d // 2) * 1)
+
+
+def computational_gain(L: int, d: int, K: int, n_i: int) -> int:
+    """Delta C(i) = n_i * 4 L d K - (6 d^2 + d)   (Eq. 9)."""
+    return n_i * 4 * L * d * K - predictor_flops(d)
+
+
+def break_even_volume(d: int, L: int, n_i: int = 1) -> float:
+    """Smallest eviction volume with a net gain: (6 d^2 + d) / (n_i * 4 L d)   (Eq. 10)."""
+    return predictor_flops(d) / (n_i * 4 * L * d)
+
+
+# ----------------------------------------------------------------------------------------------
+# Schedule driver (prefill, then decode with an eviction every E steps)
+# ----------------------------------------------------------------------------------------------
+
+def run_schedule(cache: OracleCache, prompt_k, prompt_v, stream, steps: int, budget: int,
+                 evict_interval: int, on_step=None, on_evict=None) -> List[int]:
+    """Prefill (all prompt rows pinned), then ``steps`` decode steps; after every
+    ``evict_interval``-th step evict down to ``budget``.  Returns the cache length after each
+    step (after that step's eviction, if any)."""
+    prefill(cache, prompt_k, prompt_v)
+    lengths = []
+    for s in range(1, steps + 1):
+        q, k_new, v_new = stream.step(s)
+        out, delta = decode_step(cache, q, k_new, v_new)
+        if on_step is not None:
+            on_step(s, out, delta)
+        if s % evict_interval == 0:
+            kept = evict(cache, budget)
+            if on_evict is not None:
+                on_evict(s, kept)
+        lengths.append(cache.length(0))
+    return lengths
