@@ -1,0 +1,187 @@
+/*
+ * dynts.h -- C ABI of the B200 (sm_100a) decode hot path of Dynamic Thinking-Token Selection:
+ * GQA decode attention over a budget-limited KV cache, fused with accumulation of each retained
+ * token's attention mass (its importance score), and the periodic eviction that keeps the
+ * question window, the local window and the top-scoring tokens of the selection window.
+ *
+ * Conventions
+ * -----------
+ *  - "device" pointers are CUDA device memory on the current device; "host" pointers are ordinary
+ *    host memory.  The library never frees caller memory.
+ *  - Every call that launches work is asynchronous on the cache's stream (see
+ *    dynts_cache_set_stream) unless stated otherwise.  Caller buffers must stay valid until the
+ *    stream reaches the work.
+ *  - Errors detectable on the host are returned before anything is launched and leave the cache
+ *    unchanged; dynts_last_error() then holds a message.  Errors detected on the device (a bound
+ *    that the host mirror should have made impossible) are reported by dynts_poll_error().
+ *  - A handle is not thread-safe; use one thread per handle.
+ *  - Shapes: L layers, Nb sequences, Hq query heads, Hkv KV heads, G = Hq / Hkv, d head_dim,
+ *    cap rows per slab.  A slab is one (layer, sequence, KV head): K[cap][d], V[cap][d] in the
+ *    cache dtype, pos[cap] int32, score[cap] fp32.  All tensors are contiguous, row-major, in the
+ *    index order written, and 16-byte aligned.
+ */
+#ifndef DYNTS_H
+#define DYNTS_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dynts_cache dynts_cache_t; /* opaque, owned by the library */
+
+typedef enum dynts_status {
+  DYNTS_OK = 0,
+  DYNTS_ERR_INVALID_ARG = 1, /* NULL/misaligned pointer, bad index, unsupported shape */
+  DYNTS_ERR_OOM = 2,         /* device or host allocation failed / storage too small */
+  DYNTS_ERR_CAPACITY = 3,    /* append past the slab capacity: an eviction was skipped */
+  DYNTS_ERR_BUDGET = 4,      /* question window + local window exceed the eviction target */
+  DYNTS_ERR_STATE = 5,       /* call not allowed in the cache's current state */
+  DYNTS_ERR_CUDA = 6,        /* a CUDA runtime call failed */
+  DYNTS_ERR_DEVICE = 7       /* a kernel found an inconsistent length or bound and skipped work */
+} dynts_status_t;
+
+typedef enum dynts_dtype { DYNTS_BF16 = 0, DYNTS_FP32 = 1 } dynts_dtype_t;
+
+typedef struct dynts_config {
+  int layers, batch, q_heads, kv_heads, head_dim;
+  int budget;         /* B: default eviction target (rows kept per slab) */
+  int window;         /* W_l: most recent rows, always kept */
+  int evict_interval; /* E: decode steps between evictions; slab capacity = max budget + E */
+  int capacity;       /* rows per slab; 0 => max budget + evict_interval */
+  int dtype;          /* dynts_dtype_t of q, k, v, out and the slabs */
+  const int* seq_budgets; /* host [batch] per-sequence targets, or NULL => budget for all */
+  void* storage;          /* device memory for the whole cache, 256-byte aligned, or NULL:
+                             the library then allocates with cudaMalloc and frees in destroy */
+  size_t storage_bytes;   /* size of storage; must be >= dynts_cache_bytes(cfg) */
+  void* stream;           /* cudaStream_t, NULL => the default stream */
+} dynts_config_t;
+
+/* ---- lifetime ------------------------------------------------------------------------------ */
+
+/* Create a cache for the paper's problem statement (Section 4.2: a KV budget B with a local
+ * window W_l, per layer and KV head).  Defaults: batch 1, q_heads = kv_heads, bf16,
+ * evict_interval = max(window, 64); storage is allocated at the first prefill/decode so that
+ * dynts_cache_set_shape can still change them.  Returns NULL on failure. */
+dynts_cache_t* dynts_cache_create(int layers, int kv_heads, int head_dim, int budget, int window);
+
+/* Change batch / q_heads / dtype / evict_interval of a cache made by dynts_cache_create; only
+ * before its first prefill or decode (else DYNTS_ERR_STATE). */
+dynts_status_t dynts_cache_set_shape(dynts_cache_t* c, int batch, int q_heads, int dtype, int evict_interval);
+
+/* Bytes of device storage a cache with this configuration needs (0 if the config is invalid). */
+size_t dynts_cache_bytes(const dynts_config_t* cfg);
+
+/* Create from a full configuration; storage may come from the caller (e.g. a PyTorch tensor).
+ * The storage is zeroed on the stream.  *out receives the handle. */
+dynts_status_t dynts_cache_create_ex(const dynts_config_t* cfg, dynts_cache_t** out);
+
+/* Release the handle and whatever the library allocated itself.  Synchronises the stream. */
+void dynts_cache_destroy(dynts_cache_t* c);
+
+/* All later work of this cache is issued on `stream` (a cudaStream_t). */
+dynts_status_t dynts_cache_set_stream(dynts_cache_t* c, void* stream);
+
+/* ---- the hot path -------------------------------------------------------------------------- */
+
+/* Load prompt rows into every slab (Section 4.2: the question window W_q holds the prefill
+ * tokens).  k, v: device [L, Nb, Hkv, n_tokens, d].  The first n_pinned rows get score +inf and
+ * are never evicted (the paper pins all of them: n_pinned = n_tokens); the rest start at 0.
+ * Positions are 0..n_tokens-1.  Replaces the sequences' previous content. */
+dynts_status_t dynts_prefill(dynts_cache_t* c, const void* k, const void* v, int n_tokens, int n_pinned);
+
+/* The same for one sequence of a ragged batch; k, v: device [L, Hkv, n_tokens, d].  Marks the
+ * sequence active. */
+dynts_status_t dynts_prefill_seq(dynts_cache_t* c, int seq, const void* k, const void* v, int n_tokens, int n_pinned);
+
+/* One decode step for all layers (Eq. 4-6).  For every slab of every active sequence:
+ * append k_new/v_new as row n (position = tokens seen so far, score 0), attend with the group's
+ * G query heads over rows [0, n] (the new row included) with weights softmax(q.k / sqrt(d)),
+ * write out = sum_j alpha_j v_j, and add to each row's score its attention mass summed over
+ * the G heads.
+ *   q, out:        device [L, Nb, Hq, d]  (cache dtype; out is rounded to nearest even)
+ *   k_new, v_new:  device [L, Nb, Hkv, d]
+ *   scores:        NULL, or device [L, Nb, Hkv, cap] fp32 that additionally receives this step's
+ *                  mass per row (rows [0, n] of each slab are overwritten, the rest untouched).
+ * The cache length of each active sequence grows by one.  DYNTS_ERR_CAPACITY if any active
+ * sequence is already at capacity.  Rows of inactive sequences in `out` are left untouched. */
+dynts_status_t dynts_decode_attn(dynts_cache_t* c, const void* q, const void* k_new, const void* v_new,
+                                 void* out, float* scores);
+
+/* The same for one layer (a model whose layer l+1 query depends on layer l's output).
+ *   q, out: device [Nb, Hq, d];  k_new, v_new: device [Nb, Hkv, d];  scores: as above (full
+ *   [L, Nb, Hkv, cap] buffer; only this layer's part is written).
+ * Layers must be called in order 0..L-1 within a step; lengths grow after layer L-1. */
+dynts_status_t dynts_decode_attn_layer(dynts_cache_t* c, int layer, const void* q, const void* k_new,
+                                       const void* v_new, void* out, float* scores);
+
+/* dynts_decode_attn with HOST buffers: copies q, k_new, v_new to the device, runs the step,
+ * copies out back and synchronises the stream.  Pinned host memory makes the copies asynchronous
+ * up to that synchronisation.  (Staging buffers are allocated at the first call.) */
+dynts_status_t dynts_decode_attn_host(dynts_cache_t* c, const void* q, const void* k_new, const void* v_new,
+                                      void* out);
+
+/* Eviction (Section 4.2).  Every slab longer than the target keeps: rows [0, M) (question
+ * window), its last `window` rows (local window), and of the rows between them the
+ * k = target - M - window with the highest score, equal scores going to the lower index.
+ * Survivors are compacted in place, in their original order, into rows [0, target): K, V, pos and
+ * score move together.  budget <= 0 => each sequence's configured budget.  Sequences no longer
+ * than the target are untouched.  DYNTS_ERR_BUDGET if M + window > target for a sequence that
+ * must shrink. */
+dynts_status_t dynts_evict(dynts_cache_t* c, int budget);
+
+/* Eviction with one target per sequence; seq_targets: host [Nb]. */
+dynts_status_t dynts_evict_ex(dynts_cache_t* c, const int* seq_targets);
+
+/* ---- sequence management and inspection ---------------------------------------------------- */
+
+/* Ragged batches: mark a sequence finished (length 0, inactive) until its next prefill_seq. */
+dynts_status_t dynts_seq_reset(dynts_cache_t* c, int seq);
+
+/* Host mirror of a sequence's cache length (no synchronisation); -1 on a bad argument. */
+int dynts_cache_len(const dynts_cache_t* c, int seq);
+
+/* Rows per slab. */
+int dynts_cache_capacity(const dynts_cache_t* c);
+
+/* Device [L, Nb, Hkv, cap] fp32 score accumulator.  The caller may overwrite it on the cache's
+ * stream to drive the eviction with external scores (e.g. a predictor's).  NULL before storage
+ * exists. */
+float* dynts_cache_scores(dynts_cache_t* c);
+
+/* Copy one slab to host buffers (any may be NULL): K, V [n][d] in the cache dtype, pos [n] int32,
+ * score [n] fp32, *n rows.  Synchronises the stream. */
+dynts_status_t dynts_cache_export(dynts_cache_t* c, int layer, int seq, int head, void* K, void* V,
+                                  int* pos, float* score, int* n);
+
+/* Overwrite one slab from host buffers holding n rows (all four required).  The sequence's length
+ * becomes n once every slab of it has been imported with the same n (the caller's duty).
+ * Synchronises the stream. */
+dynts_status_t dynts_cache_import(dynts_cache_t* c, int layer, int seq, int head, const void* K,
+                                  const void* V, const int* pos, const float* score, int n, int n_pinned);
+
+/* Reads the device status word (pinned host memory written by kernels): DYNTS_OK or
+ * DYNTS_ERR_DEVICE.  Does not synchronise; call after dynts_synchronize for a definite answer. */
+dynts_status_t dynts_poll_error(dynts_cache_t* c);
+
+/* Wait for the cache's stream. */
+dynts_status_t dynts_synchronize(dynts_cache_t* c);
+
+/* Launch configuration of the decode kernel, for tuning: cluster size (1, 2, 4, 8 or 16; 0 =>
+ * automatic) and kernel variant (0 => automatic, 1 => generic FMA kernel, 2 => tensor-core kernel;
+ * the tensor-core kernel needs bf16, d = 128, G <= 8). */
+dynts_status_t dynts_cache_set_launch(dynts_cache_t* c, int cluster, int variant);
+
+/* Number of kernels this library has launched on behalf of the cache so far. */
+long long dynts_cache_launch_count(const dynts_cache_t* c);
+
+/* Message of the calling thread's last failed call. */
+const char* dynts_last_error(void);
+
+const char* dynts_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DYNTS_H */

@@ -1,0 +1,93 @@
+// Shared declarations of the sm_100a kernels: parameter blocks, small device helpers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace dynts {
+
+constexpr int kMaxGroup = 8;        // query heads per KV head handled by the kernels
+constexpr int kErrTileOverflow = 1; // device status bits
+constexpr int kErrLenOverflow = 2;
+constexpr int kErrEvictSmem = 4;
+
+// One decode launch covers `n_layers` layers starting at `layer0`.
+struct DecodeParams {
+  const void* q;      // [n_layers, Nb, Hq, d] of this launch
+  const void* k_new;  // [n_layers, Nb, Hkv, d]
+  const void* v_new;
+  void* out;          // [n_layers, Nb, Hq, d]
+  float* delta_out;   // NULL or full [L, Nb, Hkv, cap]
+  void* K;            // full [L, Nb, Hkv, cap, d]
+  void* V;
+  int* pos;           // full [L, Nb, Hkv, cap]
+  float* score;       // full [L, Nb, Hkv, cap]
+  int* len;           // [Nb] rows per slab of each sequence
+  int* tot;           // [Nb] tokens seen so far (next position id)
+  const int* active;  // [Nb]
+  unsigned int* ticket;
+  int* err;           // pinned host status word
+  int layer0, n_layers, Nb, Hkv, G, d, cap;
+  int advance;        // 1: the last CTA to finish increments len/tot of active sequences
+  int tile_tokens;    // rows of logits a CTA can hold in shared memory
+  float scale_log2;   // log2(e) / sqrt(d)
+};
+
+struct EvictParams {
+  void* K;
+  void* V;
+  int* pos;
+  float* score;
+  int* src;           // [slabs, cap] gather list: src[dst] = surviving row index
+  int* hdr;           // [slabs, 4]: {first moved dst, rows kept, old length, unused}
+  int* len;           // [Nb]
+  const int* pinned;  // [Nb]
+  const int* target;  // [Nb]
+  int* err;
+  int L, Nb, Hkv, d, cap, window, elt_bytes;
+};
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ void from_float(float* p, float x) { *p = x; }
+__device__ __forceinline__ void from_float(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+
+// Streaming 16-byte load that bypasses L1 allocation (each K/V byte is read once per step).
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p));
+  return r;
+}
+
+// The last CTA of the grid to finish advances the per-sequence lengths: every other CTA has
+// read them before taking its ticket, so the update cannot race with a read of this launch.
+__device__ __forceinline__ void finish_ticket(const DecodeParams& p) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    unsigned int t = atomicAdd(p.ticket, 1u);
+    if (t == gridDim.x - 1) {
+      *p.ticket = 0u;
+      if (p.advance) {
+        for (int b = 0; b < p.Nb; ++b) {
+          if (p.active[b]) {
+            p.len[b] += 1;
+            p.tot[b] += 1;
+          }
+        }
+      }
+      __threadfence();
+    }
+  }
+}
+
+}  // namespace dynts

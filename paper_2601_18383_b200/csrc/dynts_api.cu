@@ -1,0 +1,676 @@
+// Host side of the C ABI declared in include/dynts.h: argument checks, the host mirror of the
+// per-sequence lengths, storage layout and kernel launches.  Every step of the path runs in the
+// kernels of decode_attn.cuh and evict.cuh; nothing here computes on the CPU.
+#include "../../include/dynts.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "decode_attn.cuh"
+#include "evict.cuh"
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+dynts_status_t fail(dynts_status_t st, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return st;
+}
+
+#define CUDA_TRY(expr)                                                                        \
+  do {                                                                                        \
+    cudaError_t e_ = (expr);                                                                  \
+    if (e_ != cudaSuccess) return fail(DYNTS_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); \
+  } while (0)
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {
+  size_t K, V, pos, score, src, hdr, len, tot, pinned, target, active, ticket, total;
+};
+
+int elt_bytes_of(int dtype) { return dtype == DYNTS_FP32 ? 4 : 2; }
+
+bool config_ok(const dynts_config_t* c, int* cap_out) {
+  if (!c) return false;
+  if (c->layers < 1 || c->batch < 1 || c->q_heads < 1 || c->kv_heads < 1 || c->head_dim < 8) return false;
+  if (c->q_heads % c->kv_heads) return false;
+  if (c->q_heads / c->kv_heads > dynts::kMaxGroup) return false;
+  if (c->head_dim % 8 || c->head_dim > 256) return false;
+  if (c->dtype != DYNTS_BF16 && c->dtype != DYNTS_FP32) return false;
+  if (c->budget < 1 || c->window < 0 || c->window > c->budget || c->evict_interval < 1) return false;
+  int maxb = c->budget;
+  if (c->seq_budgets)
+    for (int b = 0; b < c->batch; ++b) {
+      if (c->seq_budgets[b] < 1 || c->window > c->seq_budgets[b]) return false;
+      maxb = std::max(maxb, c->seq_budgets[b]);
+    }
+  int cap = c->capacity > 0 ? c->capacity : maxb + c->evict_interval;
+  if (cap < maxb) return false;
+  if (cap_out) *cap_out = cap;
+  return true;
+}
+
+Layout make_layout(const dynts_config_t* c, int cap) {
+  Layout L;
+  const size_t slabs = (size_t)c->layers * c->batch * c->kv_heads;
+  const size_t kv = slabs * cap * c->head_dim * elt_bytes_of(c->dtype);
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  };
+  L.K = take(kv);
+  L.V = take(kv);
+  L.pos = take(slabs * cap * 4);
+  L.score = take(slabs * cap * 4);
+  L.src = take(slabs * cap * 4);
+  L.hdr = take(slabs * 16);
+  L.len = take((size_t)c->batch * 4);
+  L.tot = take((size_t)c->batch * 4);
+  L.pinned = take((size_t)c->batch * 4);
+  L.target = take((size_t)c->batch * 4);
+  L.active = take((size_t)c->batch * 4);
+  L.ticket = take(256);
+  L.total = off;
+  return L;
+}
+
+}  // namespace
+
+struct dynts_cache {
+  dynts_config_t cfg;
+  int cap = 0;
+  int G = 1;
+  int elt = 2;
+  bool ready = false;        // storage exists
+  bool owns_storage = false;
+  char* base = nullptr;
+  Layout lay{};
+  cudaStream_t stream = nullptr;
+  int* err_host = nullptr;   // pinned, mapped
+  int* err_dev = nullptr;
+  std::vector<int> seq_budget, len_h, pinned_h, target_h, active_h;
+  int layer_cursor = 0;      // next layer expected by dynts_decode_attn_layer
+  int cluster = 0, variant = 0;
+  long long launches = 0;
+  // staging for the host-buffer entry point
+  char* stage_dev = nullptr;
+  size_t stage_bytes = 0;
+  bool attr_generic_f32 = false, attr_generic_bf16 = false, attr_mma = false, attr_select = false;
+
+  void* K() const { return base + lay.K; }
+  void* V() const { return base + lay.V; }
+  int* pos() const { return reinterpret_cast<int*>(base + lay.pos); }
+  float* score() const { return reinterpret_cast<float*>(base + lay.score); }
+  int* src() const { return reinterpret_cast<int*>(base + lay.src); }
+  int* hdr() const { return reinterpret_cast<int*>(base + lay.hdr); }
+  int* len() const { return reinterpret_cast<int*>(base + lay.len); }
+  int* tot() const { return reinterpret_cast<int*>(base + lay.tot); }
+  int* pinned() const { return reinterpret_cast<int*>(base + lay.pinned); }
+  int* target() const { return reinterpret_cast<int*>(base + lay.target); }
+  int* active() const { return reinterpret_cast<int*>(base + lay.active); }
+  unsigned int* ticket() const { return reinterpret_cast<unsigned int*>(base + lay.ticket); }
+  size_t slabs() const { return (size_t)cfg.layers * cfg.batch * cfg.kv_heads; }
+};
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+dynts_status_t materialise(dynts_cache* c) {
+  if (c->ready) return DYNTS_OK;
+  int cap = 0;
+  if (!config_ok(&c->cfg, &cap)) return fail(DYNTS_ERR_INVALID_ARG, "invalid cache configuration");
+  c->cap = cap;
+  c->G = c->cfg.q_heads / c->cfg.kv_heads;
+  c->elt = elt_bytes_of(c->cfg.dtype);
+  c->lay = make_layout(&c->cfg, cap);
+  if (c->cfg.storage) {
+    if ((reinterpret_cast<uintptr_t>(c->cfg.storage) & 255u) != 0)
+      return fail(DYNTS_ERR_INVALID_ARG, "storage must be 256-byte aligned");
+    if (c->cfg.storage_bytes < c->lay.total)
+      return fail(DYNTS_ERR_OOM, "storage too small: %zu < %zu bytes", c->cfg.storage_bytes, c->lay.total);
+    c->base = static_cast<char*>(c->cfg.storage);
+    c->owns_storage = false;
+  } else {
+    void* p = nullptr;
+    cudaError_t e = cudaMalloc(&p, c->lay.total);
+    if (e != cudaSuccess) return fail(DYNTS_ERR_OOM, "cudaMalloc(%zu): %s", c->lay.total, cudaGetErrorString(e));
+    c->base = static_cast<char*>(p);
+    c->owns_storage = true;
+  }
+  if (!c->err_host) {
+    cudaError_t e = cudaHostAlloc(reinterpret_cast<void**>(&c->err_host), 64, cudaHostAllocMapped);
+    if (e != cudaSuccess) return fail(DYNTS_ERR_OOM, "cudaHostAlloc: %s", cudaGetErrorString(e));
+    *c->err_host = 0;
+    CUDA_TRY(cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->err_dev), c->err_host, 0));
+  }
+  CUDA_TRY(cudaMemsetAsync(c->base, 0, c->lay.total, c->stream));
+  const int Nb = c->cfg.batch;
+  c->seq_budget.assign(Nb, c->cfg.budget);
+  if (c->cfg.seq_budgets)
+    for (int b = 0; b < Nb; ++b) c->seq_budget[b] = c->cfg.seq_budgets[b];
+  c->cfg.seq_budgets = nullptr;  // the caller's array is not kept
+  c->len_h.assign(Nb, 0);
+  c->pinned_h.assign(Nb, 0);
+  c->active_h.assign(Nb, 1);
+  c->target_h = c->seq_budget;
+  CUDA_TRY(cudaMemcpyAsync(c->target(), c->target_h.data(), Nb * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(cudaMemcpyAsync(c->active(), c->active_h.data(), Nb * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(cudaStreamSynchronize(c->stream));  // the host vectors above may be reused right away
+  c->ready = true;
+  return DYNTS_OK;
+}
+
+template <typename Kern>
+dynts_status_t ensure_smem_attr(Kern kern, size_t bytes, bool* done, bool nonportable) {
+  if (!*done) {
+    CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    if (nonportable) CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    *done = true;
+  }
+  if (bytes > 200 * 1024) return fail(DYNTS_ERR_INVALID_ARG, "shared-memory need %zu exceeds 200 KiB", bytes);
+  return DYNTS_OK;
+}
+
+int pick_cluster(const dynts_cache* c, int units, int n_max) {
+  if (c->cluster > 0) return c->cluster;
+  // Enough CTAs to fill 148 SMs several times over, but at least ~64 rows per CTA.
+  int s = 1;
+  while (s < 8 && (long long)units * s < 148 * 12 && n_max / (2 * s) >= 64) s *= 2;
+  return s;
+}
+
+dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const void* q, const void* k_new,
+                             const void* v_new, void* out, float* scores, bool advance) {
+  const dynts_config_t& f = c->cfg;
+  const int Nb = f.batch;
+  int n_max = 0;
+  bool any = false;
+  for (int b = 0; b < Nb; ++b) {
+    if (!c->active_h[b]) continue;
+    any = true;
+    if (c->len_h[b] + 1 > c->cap)
+      return fail(DYNTS_ERR_CAPACITY, "sequence %d is at capacity %d: evict before the next decode step", b, c->cap);
+    n_max = std::max(n_max, c->len_h[b] + 1);
+  }
+  if (!any) return DYNTS_OK;
+
+  const int units = n_layers * Nb * f.kv_heads;
+  const int S = pick_cluster(c, units, n_max);
+  const int units16 = (n_max + 15) / 16;
+  const int tile_tokens = (units16 + S - 1) / S * 16;
+
+  dynts::DecodeParams p;
+  p.q = q;
+  p.k_new = k_new;
+  p.v_new = v_new;
+  p.out = out;
+  p.delta_out = scores;
+  p.K = c->K();
+  p.V = c->V();
+  p.pos = c->pos();
+  p.score = c->score();
+  p.len = c->len();
+  p.tot = c->tot();
+  p.active = c->active();
+  p.ticket = c->ticket();
+  p.err = c->err_dev;
+  p.layer0 = layer0;
+  p.n_layers = n_layers;
+  p.Nb = Nb;
+  p.Hkv = f.kv_heads;
+  p.G = c->G;
+  p.d = f.head_dim;
+  p.cap = c->cap;
+  p.advance = advance ? 1 : 0;
+  p.tile_tokens = tile_tokens;
+  p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)f.head_dim));
+
+  const bool mma_ok = f.dtype == DYNTS_BF16 && f.head_dim == 128 && c->G <= 8;
+  int variant = c->variant;
+  if (variant == 0) variant = mma_ok ? 2 : 1;
+  if (variant == 2 && !mma_ok) return fail(DYNTS_ERR_INVALID_ARG, "tensor-core variant needs bf16, head_dim 128, G <= 8");
+
+  cudaLaunchConfig_t lc;
+  memset(&lc, 0, sizeof(lc));
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = S;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  lc.stream = c->stream;
+  lc.gridDim = dim3((unsigned)(units * S), 1, 1);
+
+  cudaError_t e;
+  if (variant == 2) {
+    const size_t smem = dynts::mma_smem_bytes(c->G, tile_tokens);
+    dynts_status_t st = ensure_smem_attr(dynts::decode_attn_mma_kernel, smem, &c->attr_mma, true);
+    if (st != DYNTS_OK) return st;
+    lc.blockDim = dim3(dynts::kMmaThreads, 1, 1);
+    lc.dynamicSmemBytes = smem;
+    e = cudaLaunchKernelEx(&lc, dynts::decode_attn_mma_kernel, p);
+  } else if (f.dtype == DYNTS_FP32) {
+    const size_t smem = dynts::generic_smem_bytes(c->G, f.head_dim, tile_tokens);
+    dynts_status_t st = ensure_smem_attr(dynts::decode_attn_generic_kernel<float>, smem, &c->attr_generic_f32, true);
+    if (st != DYNTS_OK) return st;
+    lc.blockDim = dim3(dynts::kGenericThreads, 1, 1);
+    lc.dynamicSmemBytes = smem;
+    e = cudaLaunchKernelEx(&lc, dynts::decode_attn_generic_kernel<float>, p);
+  } else {
+    const size_t smem = dynts::generic_smem_bytes(c->G, f.head_dim, tile_tokens);
+    dynts_status_t st =
+        ensure_smem_attr(dynts::decode_attn_generic_kernel<__nv_bfloat16>, smem, &c->attr_generic_bf16, true);
+    if (st != DYNTS_OK) return st;
+    lc.blockDim = dim3(dynts::kGenericThreads, 1, 1);
+    lc.dynamicSmemBytes = smem;
+    e = cudaLaunchKernelEx(&lc, dynts::decode_attn_generic_kernel<__nv_bfloat16>, p);
+  }
+  if (e != cudaSuccess) return fail(DYNTS_ERR_CUDA, "decode launch (cluster %d): %s", S, cudaGetErrorString(e));
+  c->launches += 1;
+  if (advance)
+    for (int b = 0; b < Nb; ++b)
+      if (c->active_h[b]) c->len_h[b] += 1;
+  return DYNTS_OK;
+}
+
+dynts_status_t check_decode_args(const dynts_cache* c, const void* q, const void* k_new, const void* v_new,
+                                 const void* out) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (!q || !k_new || !v_new || !out) return fail(DYNTS_ERR_INVALID_ARG, "NULL tensor pointer");
+  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out))
+    return fail(DYNTS_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+  return DYNTS_OK;
+}
+
+dynts_status_t do_prefill(dynts_cache* c, int seq, const void* k, const void* v, int T, int n_pinned) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  dynts_status_t st = materialise(c);
+  if (st != DYNTS_OK) return st;
+  if (!k || !v || !aligned16(k) || !aligned16(v))
+    return fail(DYNTS_ERR_INVALID_ARG, "prefill tensors must be non-NULL and 16-byte aligned");
+  if (T < 0 || T > c->cap) return fail(DYNTS_ERR_CAPACITY, "prefill of %d rows exceeds capacity %d", T, c->cap);
+  if (n_pinned < 0 || n_pinned > T) return fail(DYNTS_ERR_INVALID_ARG, "n_pinned %d outside [0, %d]", n_pinned, T);
+  if (seq >= c->cfg.batch) return fail(DYNTS_ERR_INVALID_ARG, "sequence %d out of range", seq);
+  if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "prefill in the middle of a layer-by-layer step");
+  dynts::PrefillParams p;
+  p.k = k;
+  p.v = v;
+  p.K = c->K();
+  p.V = c->V();
+  p.pos = c->pos();
+  p.score = c->score();
+  p.len = c->len();
+  p.tot = c->tot();
+  p.pinned = c->pinned();
+  p.active = c->active();
+  p.L = c->cfg.layers;
+  p.Nb = c->cfg.batch;
+  p.Hkv = c->cfg.kv_heads;
+  p.d = c->cfg.head_dim;
+  p.cap = c->cap;
+  p.elt_bytes = c->elt;
+  p.T = T;
+  p.n_pinned = n_pinned;
+  p.seq = seq;
+  const unsigned ny = (unsigned)(seq < 0 ? c->slabs() : (size_t)c->cfg.layers * c->cfg.kv_heads);
+  const size_t pieces = (size_t)T * c->cfg.head_dim * c->elt / 16;
+  const unsigned nx = (unsigned)std::max<size_t>(1, std::min<size_t>(64, (pieces + 255) / 256));
+  dynts::prefill_kernel<<<dim3(nx, ny, 1), 256, 0, c->stream>>>(p);
+  CUDA_TRY(cudaGetLastError());
+  c->launches += 1;
+  for (int b = 0; b < c->cfg.batch; ++b) {
+    if (seq >= 0 && b != seq) continue;
+    c->len_h[b] = T;
+    c->pinned_h[b] = n_pinned;
+    c->active_h[b] = 1;
+  }
+  return DYNTS_OK;
+}
+
+dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validated */) {
+  const int Nb = c->cfg.batch;
+  bool any = false;
+  for (int b = 0; b < Nb; ++b) {
+    if (!c->active_h[b] || c->len_h[b] <= targets[b]) continue;
+    if (c->pinned_h[b] + c->cfg.window > targets[b])
+      return fail(DYNTS_ERR_BUDGET, "sequence %d: question window %d + local window %d exceed target %d", b,
+                  c->pinned_h[b], c->cfg.window, targets[b]);
+    any = true;
+  }
+  if (!any) return DYNTS_OK;
+  bool same = true;
+  for (int b = 0; b < Nb; ++b) same = same && c->target_h[b] == targets[b];
+  if (!same) {
+    c->target_h.assign(targets, targets + Nb);
+    // pageable source: the runtime stages it before returning, so target_h may change afterwards
+    CUDA_TRY(cudaMemcpyAsync(c->target(), c->target_h.data(), Nb * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  }
+  dynts::EvictParams p;
+  p.K = c->K();
+  p.V = c->V();
+  p.pos = c->pos();
+  p.score = c->score();
+  p.src = c->src();
+  p.hdr = c->hdr();
+  p.len = c->len();
+  p.pinned = c->pinned();
+  p.target = c->target();
+  p.err = c->err_dev;
+  p.L = c->cfg.layers;
+  p.Nb = Nb;
+  p.Hkv = c->cfg.kv_heads;
+  p.d = c->cfg.head_dim;
+  p.cap = c->cap;
+  p.window = c->cfg.window;
+  p.elt_bytes = c->elt;
+  const size_t smem = (size_t)c->cap * 8;
+  dynts_status_t st = ensure_smem_attr(dynts::evict_select_kernel, smem, &c->attr_select, false);
+  if (st != DYNTS_OK) return st;
+  dynts::evict_select_kernel<<<(unsigned)c->slabs(), dynts::kSelectThreads, smem, c->stream>>>(p);
+  CUDA_TRY(cudaGetLastError());
+  const int pieces = c->cfg.head_dim * c->elt / 16;
+  const unsigned groups = (unsigned)((pieces + 3) / 4);
+  dynts::evict_compact_kernel<<<dim3(2 * groups, (unsigned)c->slabs(), 1), dynts::kCompactThreads, 0, c->stream>>>(p);
+  CUDA_TRY(cudaGetLastError());
+  c->launches += 2;
+  for (int b = 0; b < Nb; ++b)
+    if (c->active_h[b]) c->len_h[b] = std::min(c->len_h[b], targets[b]);
+  return DYNTS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* dynts_last_error(void) { return g_err; }
+const char* dynts_version(void) { return "dynts-b200 0.1 (sm_100a)"; }
+
+dynts_cache_t* dynts_cache_create(int layers, int kv_heads, int head_dim, int budget, int window) {
+  dynts_cache* c = new (std::nothrow) dynts_cache();
+  if (!c) {
+    fail(DYNTS_ERR_OOM, "out of host memory");
+    return nullptr;
+  }
+  memset(&c->cfg, 0, sizeof(c->cfg));
+  c->cfg.layers = layers;
+  c->cfg.batch = 1;
+  c->cfg.q_heads = kv_heads;
+  c->cfg.kv_heads = kv_heads;
+  c->cfg.head_dim = head_dim;
+  c->cfg.budget = budget;
+  c->cfg.window = window;
+  c->cfg.evict_interval = std::max(window, 64);
+  c->cfg.dtype = DYNTS_BF16;
+  if (!config_ok(&c->cfg, nullptr)) {
+    fail(DYNTS_ERR_INVALID_ARG, "invalid arguments: layers %d kv_heads %d head_dim %d budget %d window %d", layers,
+         kv_heads, head_dim, budget, window);
+    delete c;
+    return nullptr;
+  }
+  return c;
+}
+
+dynts_status_t dynts_cache_set_shape(dynts_cache_t* c, int batch, int q_heads, int dtype, int evict_interval) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (c->ready) return fail(DYNTS_ERR_STATE, "shape is fixed after the first prefill or decode");
+  dynts_config_t t = c->cfg;
+  t.batch = batch;
+  t.q_heads = q_heads;
+  t.dtype = dtype;
+  t.evict_interval = evict_interval;
+  if (!config_ok(&t, nullptr)) return fail(DYNTS_ERR_INVALID_ARG, "invalid shape");
+  c->cfg = t;
+  return DYNTS_OK;
+}
+
+size_t dynts_cache_bytes(const dynts_config_t* cfg) {
+  int cap = 0;
+  if (!config_ok(cfg, &cap)) return 0;
+  return make_layout(cfg, cap).total;
+}
+
+dynts_status_t dynts_cache_create_ex(const dynts_config_t* cfg, dynts_cache_t** out) {
+  if (!out) return fail(DYNTS_ERR_INVALID_ARG, "NULL out");
+  *out = nullptr;
+  if (!config_ok(cfg, nullptr)) return fail(DYNTS_ERR_INVALID_ARG, "invalid cache configuration");
+  dynts_cache* c = new (std::nothrow) dynts_cache();
+  if (!c) return fail(DYNTS_ERR_OOM, "out of host memory");
+  c->cfg = *cfg;
+  c->stream = static_cast<cudaStream_t>(cfg->stream);
+  dynts_status_t st = materialise(c);
+  if (st != DYNTS_OK) {
+    if (c->owns_storage && c->base) cudaFree(c->base);
+    if (c->err_host) cudaFreeHost(c->err_host);
+    delete c;
+    return st;
+  }
+  *out = c;
+  return DYNTS_OK;
+}
+
+void dynts_cache_destroy(dynts_cache_t* c) {
+  if (!c) return;
+  if (c->ready) cudaStreamSynchronize(c->stream);
+  if (c->owns_storage && c->base) cudaFree(c->base);
+  if (c->stage_dev) cudaFree(c->stage_dev);
+  if (c->err_host) cudaFreeHost(c->err_host);
+  delete c;
+}
+
+dynts_status_t dynts_cache_set_stream(dynts_cache_t* c, void* stream) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  c->stream = static_cast<cudaStream_t>(stream);
+  return DYNTS_OK;
+}
+
+dynts_status_t dynts_prefill(dynts_cache_t* c, const void* k, const void* v, int n_tokens, int n_pinned) {
+  return do_prefill(c, -1, k, v, n_tokens, n_pinned);
+}
+
+dynts_status_t dynts_prefill_seq(dynts_cache_t* c, int seq, const void* k, const void* v, int n_tokens, int n_pinned) {
+  if (seq < 0) return fail(DYNTS_ERR_INVALID_ARG, "sequence %d out of range", seq);
+  return do_prefill(c, seq, k, v, n_tokens, n_pinned);
+}
+
+dynts_status_t dynts_decode_attn(dynts_cache_t* c, const void* q, const void* k_new, const void* v_new, void* out,
+                                 float* scores) {
+  dynts_status_t st = check_decode_args(c, q, k_new, v_new, out);
+  if (st != DYNTS_OK) return st;
+  st = materialise(c);
+  if (st != DYNTS_OK) return st;
+  if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "a layer-by-layer step is in progress");
+  return launch_decode(c, 0, c->cfg.layers, q, k_new, v_new, out, scores, true);
+}
+
+dynts_status_t dynts_decode_attn_layer(dynts_cache_t* c, int layer, const void* q, const void* k_new,
+                                       const void* v_new, void* out, float* scores) {
+  dynts_status_t st = check_decode_args(c, q, k_new, v_new, out);
+  if (st != DYNTS_OK) return st;
+  st = materialise(c);
+  if (st != DYNTS_OK) return st;
+  if (layer != c->layer_cursor)
+    return fail(DYNTS_ERR_STATE, "layer %d called, layer %d expected", layer, c->layer_cursor);
+  const bool last = layer == c->cfg.layers - 1;
+  st = launch_decode(c, layer, 1, q, k_new, v_new, out, scores, last);
+  if (st == DYNTS_OK) c->layer_cursor = last ? 0 : layer + 1;
+  return st;
+}
+
+dynts_status_t dynts_decode_attn_host(dynts_cache_t* c, const void* q, const void* k_new, const void* v_new,
+                                      void* out) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (!q || !k_new || !v_new || !out) return fail(DYNTS_ERR_INVALID_ARG, "NULL tensor pointer");
+  dynts_status_t st = materialise(c);
+  if (st != DYNTS_OK) return st;
+  if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "a layer-by-layer step is in progress");
+  for (int b = 0; b < c->cfg.batch; ++b)
+    if (c->active_h[b] && c->len_h[b] + 1 > c->cap)
+      return fail(DYNTS_ERR_CAPACITY, "sequence %d is at capacity %d: evict before the next decode step", b, c->cap);
+  const dynts_config_t& f = c->cfg;
+  const size_t qb = align_up((size_t)f.layers * f.batch * f.q_heads * f.head_dim * c->elt, 256);
+  const size_t kb = align_up((size_t)f.layers * f.batch * f.kv_heads * f.head_dim * c->elt, 256);
+  const size_t need = 2 * qb + 2 * kb;
+  if (c->stage_bytes < need) {
+    if (c->stage_dev) cudaFree(c->stage_dev);
+    c->stage_dev = nullptr;
+    c->stage_bytes = 0;
+    void* ptr = nullptr;
+    cudaError_t e = cudaMalloc(&ptr, need);
+    if (e != cudaSuccess) return fail(DYNTS_ERR_OOM, "cudaMalloc(%zu): %s", need, cudaGetErrorString(e));
+    c->stage_dev = static_cast<char*>(ptr);
+    c->stage_bytes = need;
+  }
+  char* dq = c->stage_dev;
+  char* dk = dq + qb;
+  char* dv = dk + kb;
+  char* dout = dv + kb;
+  const size_t qn = (size_t)f.layers * f.batch * f.q_heads * f.head_dim * c->elt;
+  const size_t kn = (size_t)f.layers * f.batch * f.kv_heads * f.head_dim * c->elt;
+  CUDA_TRY(cudaMemcpyAsync(dq, q, qn, cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(cudaMemcpyAsync(dk, k_new, kn, cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(cudaMemcpyAsync(dv, v_new, kn, cudaMemcpyHostToDevice, c->stream));
+  st = launch_decode(c, 0, f.layers, dq, dk, dv, dout, nullptr, true);
+  if (st != DYNTS_OK) return st;
+  CUDA_TRY(cudaMemcpyAsync(out, dout, qn, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(cudaStreamSynchronize(c->stream));
+  return DYNTS_OK;
+}
+
+dynts_status_t dynts_evict(dynts_cache_t* c, int budget) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (!c->ready) return fail(DYNTS_ERR_STATE, "cache holds nothing yet");
+  if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "evict in the middle of a layer-by-layer step");
+  std::vector<int> t(c->cfg.batch);
+  for (int b = 0; b < c->cfg.batch; ++b) t[b] = budget > 0 ? budget : c->seq_budget[b];
+  return do_evict(c, t.data());
+}
+
+dynts_status_t dynts_evict_ex(dynts_cache_t* c, const int* seq_targets) {
+  if (!c || !seq_targets) return fail(DYNTS_ERR_INVALID_ARG, "NULL argument");
+  if (!c->ready) return fail(DYNTS_ERR_STATE, "cache holds nothing yet");
+  if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "evict in the middle of a layer-by-layer step");
+  for (int b = 0; b < c->cfg.batch; ++b)
+    if (seq_targets[b] < 1) return fail(DYNTS_ERR_INVALID_ARG, "target of sequence %d must be positive", b);
+  return do_evict(c, seq_targets);
+}
+
+dynts_status_t dynts_seq_reset(dynts_cache_t* c, int seq) {
+  if (!c || seq < 0 || seq >= c->cfg.batch) return fail(DYNTS_ERR_INVALID_ARG, "bad cache or sequence");
+  if (!c->ready) return fail(DYNTS_ERR_STATE, "cache holds nothing yet");
+  if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "reset in the middle of a layer-by-layer step");
+  CUDA_TRY(cudaMemsetAsync(c->len() + seq, 0, sizeof(int), c->stream));
+  CUDA_TRY(cudaMemsetAsync(c->tot() + seq, 0, sizeof(int), c->stream));
+  CUDA_TRY(cudaMemsetAsync(c->pinned() + seq, 0, sizeof(int), c->stream));
+  CUDA_TRY(cudaMemsetAsync(c->active() + seq, 0, sizeof(int), c->stream));
+  c->len_h[seq] = 0;
+  c->pinned_h[seq] = 0;
+  c->active_h[seq] = 0;
+  return DYNTS_OK;
+}
+
+int dynts_cache_len(const dynts_cache_t* c, int seq) {
+  if (!c || seq < 0 || seq >= c->cfg.batch) return -1;
+  if (!c->ready) return 0;
+  return c->len_h[seq];
+}
+
+int dynts_cache_capacity(const dynts_cache_t* c) {
+  if (!c) return -1;
+  if (c->ready) return c->cap;
+  int cap = 0;
+  return config_ok(&c->cfg, &cap) ? cap : -1;
+}
+
+float* dynts_cache_scores(dynts_cache_t* c) { return (c && c->ready) ? c->score() : nullptr; }
+
+dynts_status_t dynts_cache_export(dynts_cache_t* c, int layer, int seq, int head, void* K, void* V, int* pos,
+                                  float* score, int* n) {
+  if (!c || !c->ready) return fail(DYNTS_ERR_STATE, "cache holds nothing yet");
+  if (layer < 0 || layer >= c->cfg.layers || seq < 0 || seq >= c->cfg.batch || head < 0 || head >= c->cfg.kv_heads)
+    return fail(DYNTS_ERR_INVALID_ARG, "slab index out of range");
+  CUDA_TRY(cudaStreamSynchronize(c->stream));
+  const size_t slab = ((size_t)layer * c->cfg.batch + seq) * c->cfg.kv_heads + head;
+  const int rows = c->len_h[seq];
+  const size_t row_bytes = (size_t)c->cfg.head_dim * c->elt;
+  if (K) CUDA_TRY(cudaMemcpy(K, static_cast<char*>(c->K()) + slab * c->cap * row_bytes, rows * row_bytes, cudaMemcpyDeviceToHost));
+  if (V) CUDA_TRY(cudaMemcpy(V, static_cast<char*>(c->V()) + slab * c->cap * row_bytes, rows * row_bytes, cudaMemcpyDeviceToHost));
+  if (pos) CUDA_TRY(cudaMemcpy(pos, c->pos() + slab * c->cap, rows * sizeof(int), cudaMemcpyDeviceToHost));
+  if (score) CUDA_TRY(cudaMemcpy(score, c->score() + slab * c->cap, rows * sizeof(float), cudaMemcpyDeviceToHost));
+  if (n) *n = rows;
+  return DYNTS_OK;
+}
+
+dynts_status_t dynts_cache_import(dynts_cache_t* c, int layer, int seq, int head, const void* K, const void* V,
+                                  const int* pos, const float* score, int n, int n_pinned) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  dynts_status_t st = materialise(c);
+  if (st != DYNTS_OK) return st;
+  if (layer < 0 || layer >= c->cfg.layers || seq < 0 || seq >= c->cfg.batch || head < 0 || head >= c->cfg.kv_heads)
+    return fail(DYNTS_ERR_INVALID_ARG, "slab index out of range");
+  if (!K || !V || !pos || !score) return fail(DYNTS_ERR_INVALID_ARG, "NULL buffer");
+  if (n < 0 || n > c->cap) return fail(DYNTS_ERR_CAPACITY, "%d rows exceed capacity %d", n, c->cap);
+  if (n_pinned < 0 || n_pinned > n) return fail(DYNTS_ERR_INVALID_ARG, "n_pinned out of range");
+  if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "import in the middle of a layer-by-layer step");
+  CUDA_TRY(cudaStreamSynchronize(c->stream));
+  const size_t slab = ((size_t)layer * c->cfg.batch + seq) * c->cfg.kv_heads + head;
+  const size_t row_bytes = (size_t)c->cfg.head_dim * c->elt;
+  CUDA_TRY(cudaMemcpy(static_cast<char*>(c->K()) + slab * c->cap * row_bytes, K, n * row_bytes, cudaMemcpyHostToDevice));
+  CUDA_TRY(cudaMemcpy(static_cast<char*>(c->V()) + slab * c->cap * row_bytes, V, n * row_bytes, cudaMemcpyHostToDevice));
+  CUDA_TRY(cudaMemcpy(c->pos() + slab * c->cap, pos, n * sizeof(int), cudaMemcpyHostToDevice));
+  CUDA_TRY(cudaMemcpy(c->score() + slab * c->cap, score, n * sizeof(float), cudaMemcpyHostToDevice));
+  int next = n > 0 ? pos[n - 1] + 1 : 0;
+  int one = 1;
+  CUDA_TRY(cudaMemcpy(c->len() + seq, &n, sizeof(int), cudaMemcpyHostToDevice));
+  CUDA_TRY(cudaMemcpy(c->tot() + seq, &next, sizeof(int), cudaMemcpyHostToDevice));
+  CUDA_TRY(cudaMemcpy(c->pinned() + seq, &n_pinned, sizeof(int), cudaMemcpyHostToDevice));
+  CUDA_TRY(cudaMemcpy(c->active() + seq, &one, sizeof(int), cudaMemcpyHostToDevice));
+  c->len_h[seq] = n;
+  c->pinned_h[seq] = n_pinned;
+  c->active_h[seq] = 1;
+  return DYNTS_OK;
+}
+
+dynts_status_t dynts_poll_error(dynts_cache_t* c) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (c->err_host && *reinterpret_cast<volatile int*>(c->err_host) != 0)
+    return fail(DYNTS_ERR_DEVICE, "device status word 0x%x", *reinterpret_cast<volatile int*>(c->err_host));
+  return DYNTS_OK;
+}
+
+dynts_status_t dynts_synchronize(dynts_cache_t* c) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  CUDA_TRY(cudaStreamSynchronize(c->stream));
+  return DYNTS_OK;
+}
+
+dynts_status_t dynts_cache_set_launch(dynts_cache_t* c, int cluster, int variant) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (!(cluster == 0 || cluster == 1 || cluster == 2 || cluster == 4 || cluster == 8 || cluster == 16))
+    return fail(DYNTS_ERR_INVALID_ARG, "cluster size must be 0, 1, 2, 4, 8 or 16");
+  if (variant < 0 || variant > 2) return fail(DYNTS_ERR_INVALID_ARG, "variant must be 0, 1 or 2");
+  c->cluster = cluster;
+  c->variant = variant;
+  return DYNTS_OK;
+}
+
+long long dynts_cache_launch_count(const dynts_cache_t* c) { return c ? c->launches : -1; }
+
+}  // extern "C"

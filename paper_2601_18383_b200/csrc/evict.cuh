@@ -1,0 +1,264 @@
+// Budgeted eviction (Section 4.2) for sm_100a: selection, then in-place stable compaction.
+//
+//   evict_select_kernel   one CTA per slab.  Scores are compared through an order-preserving
+//                         map of their fp32 bit patterns to uint32, so every decision is integer
+//                         arithmetic.  A 4-pass, 8-bit radix select finds the k-th largest key T
+//                         of the selection window; rows with key > T survive, and of the rows
+//                         with key == T the lowest-indexed survive until k is reached (a prefix
+//                         count gives each its rank).  A second prefix count over the survivor
+//                         flags gives every survivor its destination row; the kernel writes the
+//                         gather list src[dst] and compacts score and pos itself.
+//   evict_compact_kernel  moves the K and V rows.  The gather is stable and only moves rows
+//                         towards lower indices (src[dst] >= dst, both increasing), so a CTA that
+//                         walks the destination rows in ascending chunks and, per chunk, loads
+//                         every source row before storing any destination row never overwrites
+//                         data it still needs.  CTAs split the row bytes into 64-byte column
+//                         groups (and K from V), which makes them fully independent: no
+//                         inter-CTA ordering, no second buffer.
+#pragma once
+
+#include "common.cuh"
+
+namespace dynts {
+
+constexpr int kSelectThreads = 1024;
+constexpr int kCompactThreads = 256;
+constexpr int kCompactUnroll = 8;                                         // 16-byte loads in flight per thread
+constexpr int kCompactRowsPerPass = kCompactThreads / 4;                  // 4 threads cover one 64-byte group
+constexpr int kCompactChunkRows = kCompactRowsPerPass * kCompactUnroll;   // rows per load/store phase
+
+// fp32 -> uint32 with the same order as the float comparison; -0 and +0 get the same key.
+__device__ __forceinline__ uint32_t order_key(uint32_t raw_bits) {
+  const float s = __fadd_rn(__uint_as_float(raw_bits), 0.0f);
+  const uint32_t b = __float_as_uint(s);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// Exclusive prefix count of a per-thread flag over the CTA, plus the CTA total.
+__device__ __forceinline__ int block_prefix_count(bool flag, int* warp_tot /* [32] shared */, int& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned bal = __ballot_sync(0xffffffffu, flag);
+  const int in_warp = __popc(bal & ((1u << lane) - 1u));
+  if (lane == 0) warp_tot[warp] = __popc(bal);
+  __syncthreads();
+  const int nwarps = blockDim.x >> 5;
+  int before = 0, tot = 0;
+  for (int w = 0; w < nwarps; ++w) {
+    const int t = warp_tot[w];
+    if (w < warp) before += t;
+    tot += t;
+  }
+  __syncthreads();  // warp_tot may be reused right after
+  total = tot;
+  return before + in_warp;
+}
+
+__global__ void __launch_bounds__(kSelectThreads) evict_select_kernel(const EvictParams p) {
+  const int slab = blockIdx.x;
+  const int b = (slab / p.Hkv) % p.Nb;
+  const int tid = threadIdx.x;
+  const int n = p.len[b];
+  const int tgt = p.target[b];
+  int* hdr = p.hdr + (size_t)slab * 4;
+  if (n <= tgt) {  // nothing to evict for this sequence
+    if (tid == 0) {
+      hdr[0] = n;
+      hdr[1] = n;
+      hdr[2] = n;
+    }
+    return;
+  }
+  const int M = p.pinned[b];
+  const int lo = M, hi = n - p.window;  // selection window [lo, hi)
+  const int k = tgt - M - p.window;     // survivors wanted from it (host guarantees 0 <= k < hi - lo)
+
+  extern __shared__ __align__(16) uint32_t esm[];
+  uint32_t* raw = esm;                                   // [cap] score bit patterns
+  int* posbuf = reinterpret_cast<int*>(esm + p.cap);     // [cap]
+  __shared__ unsigned int hist[256];
+  __shared__ int warp_tot[32];
+  __shared__ uint32_t s_prefix;
+  __shared__ int s_krem, s_first;
+
+  float* score = p.score + (size_t)slab * p.cap;
+  int* pos = p.pos + (size_t)slab * p.cap;
+  int* src = p.src + (size_t)slab * p.cap;
+  for (int j = tid; j < n; j += kSelectThreads) {
+    raw[j] = __float_as_uint(score[j]);
+    posbuf[j] = pos[j];
+  }
+  if (tid == 0) {
+    s_prefix = 0u;
+    s_krem = k;
+    s_first = n;
+  }
+  __syncthreads();
+
+  // Radix select: after the pass for `shift`, s_prefix holds the top bits of the k-th largest
+  // key and s_krem how many rows with exactly those top bits must still be taken.
+  uint32_t mask = 0u;
+  if (k > 0) {
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      if (tid < 256) hist[tid] = 0u;
+      __syncthreads();
+      const uint32_t prefix = s_prefix;
+      const int krem = s_krem;  // read by everyone before warp 0 updates it below
+      for (int j = lo + tid; j < hi; j += kSelectThreads) {
+        const uint32_t key = order_key(raw[j]);
+        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (tid < 32) {
+        // lane l owns bins 255-8l .. 248-8l (descending); find where the count from the top
+        // reaches krem.
+        unsigned int mine = 0;
+        for (int i = 0; i < 8; ++i) mine += hist[255 - 8 * tid - i];
+        unsigned int incl = mine;
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned int v = __shfl_up_sync(0xffffffffu, incl, o);
+          if (tid >= o) incl += v;
+        }
+        const unsigned int excl = incl - mine;
+        if ((int)excl < krem && krem <= (int)incl) {
+          unsigned int above = excl;
+          for (int i = 0; i < 8; ++i) {
+            const int bin = 255 - 8 * tid - i;
+            const unsigned int c = hist[bin];
+            if ((int)(above + c) >= krem) {
+              s_prefix = prefix | ((uint32_t)bin << shift);
+              s_krem = krem - (int)above;
+              break;
+            }
+            above += c;
+          }
+        }
+      }
+      mask |= 0xFFu << shift;
+      __syncthreads();
+    }
+  }
+  const uint32_t T = s_prefix;   // key of the k-th largest candidate
+  const int take_eq = s_krem;    // rows with key == T that survive (lowest indices first)
+
+  int carry_eq = 0, carry_keep = 0;
+  for (int base = 0; base < n; base += kSelectThreads) {
+    const int j = base + tid;
+    const bool in = j < n;
+    const bool cand = in && j >= lo && j < hi;
+    uint32_t key = 0u;
+    if (cand) key = order_key(raw[j]);
+    const bool gt = cand && k > 0 && key > T;
+    const bool eq = cand && k > 0 && key == T;
+    int tot_eq, tot_keep;
+    const int eq_rank = carry_eq + block_prefix_count(eq, warp_tot, tot_eq);
+    const bool keep = in && (!cand || gt || (eq && eq_rank < take_eq));
+    const int dst = carry_keep + block_prefix_count(keep, warp_tot, tot_keep);
+    if (keep) {
+      src[dst] = j;
+      score[dst] = __uint_as_float(raw[j]);
+      pos[dst] = posbuf[j];
+    } else if (in) {
+      atomicMin(&s_first, j);
+    }
+    carry_eq += tot_eq;
+    carry_keep += tot_keep;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    hdr[0] = s_first;      // rows below the first evicted one do not move
+    hdr[1] = carry_keep;   // == tgt
+    hdr[2] = n;
+  }
+}
+
+// grid.x = 2 * column groups (even: K, odd: V), grid.y = slabs.
+__global__ void __launch_bounds__(kCompactThreads) evict_compact_kernel(const EvictParams p) {
+  const int slab = blockIdx.y;
+  const int which = blockIdx.x & 1;
+  const int cgp = blockIdx.x >> 1;
+  const int tid = threadIdx.x;
+  const int* hdr = p.hdr + (size_t)slab * 4;
+  const int lo = hdr[0], hi = hdr[1];
+  // One designated CTA per sequence publishes the new length (no CTA of this launch reads len).
+  if (blockIdx.x == 0 && tid == 0 && slab < p.Nb * p.Hkv && slab % p.Hkv == 0) p.len[slab / p.Hkv] = hi;
+  if (lo >= hi) return;
+
+  const size_t row_bytes = (size_t)p.d * p.elt_bytes;
+  const int pieces = (int)(row_bytes >> 4);
+  const int piece = cgp * 4 + (tid & 3);
+  const bool col_ok = piece < pieces;
+  char* base = reinterpret_cast<char*>(which ? p.V : p.K) + (size_t)slab * p.cap * row_bytes + (size_t)piece * 16;
+  const int* src = p.src + (size_t)slab * p.cap;
+
+  for (int c0 = lo; c0 < hi; c0 += kCompactChunkRows) {
+    uint4 buf[kCompactUnroll];
+#pragma unroll
+    for (int uu = 0; uu < kCompactUnroll; ++uu) {
+      const int dst = c0 + uu * kCompactRowsPerPass + (tid >> 2);
+      if (col_ok && dst < hi) buf[uu] = *reinterpret_cast<const uint4*>(base + (size_t)src[dst] * row_bytes);
+    }
+    __syncthreads();  // every source row of the chunk is in registers before any row is overwritten
+#pragma unroll
+    for (int uu = 0; uu < kCompactUnroll; ++uu) {
+      const int dst = c0 + uu * kCompactRowsPerPass + (tid >> 2);
+      if (col_ok && dst < hi) *reinterpret_cast<uint4*>(base + (size_t)dst * row_bytes) = buf[uu];
+    }
+    // The next chunk reads rows src[dst'] >= dst' >= c0 + chunk, disjoint from the rows just
+    // written, so no second barrier is needed.
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Prompt load (question window, Section 4.2).  grid.x = row blocks, grid.y = slabs touched.
+// ---------------------------------------------------------------------------------------------
+struct PrefillParams {
+  const void* k;   // [L, Nb, Hkv, T, d] (seq < 0) or [L, Hkv, T, d] (one sequence)
+  const void* v;
+  void* K;
+  void* V;
+  int* pos;
+  float* score;
+  int* len;
+  int* tot;
+  int* pinned;
+  int* active;
+  int L, Nb, Hkv, d, cap, elt_bytes, T, n_pinned, seq;
+};
+
+__global__ void __launch_bounds__(256) prefill_kernel(const PrefillParams p) {
+  const int sl = blockIdx.y;  // index over the slabs of the source tensor
+  int l, b, h;
+  if (p.seq < 0) {
+    h = sl % p.Hkv;
+    b = (sl / p.Hkv) % p.Nb;
+    l = sl / (p.Hkv * p.Nb);
+  } else {
+    h = sl % p.Hkv;
+    l = sl / p.Hkv;
+    b = p.seq;
+  }
+  const size_t slab = ((size_t)l * p.Nb + b) * p.Hkv + h;
+  const size_t row_bytes = (size_t)p.d * p.elt_bytes;
+  const int pieces = (int)(row_bytes >> 4);
+  const char* ks = reinterpret_cast<const char*>(p.k) + (size_t)sl * p.T * row_bytes;
+  const char* vs = reinterpret_cast<const char*>(p.v) + (size_t)sl * p.T * row_bytes;
+  char* Kd = reinterpret_cast<char*>(p.K) + slab * p.cap * row_bytes;
+  char* Vd = reinterpret_cast<char*>(p.V) + slab * p.cap * row_bytes;
+  const size_t total = (size_t)p.T * pieces;
+  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+    reinterpret_cast<uint4*>(Kd)[e] = reinterpret_cast<const uint4*>(ks)[e];
+    reinterpret_cast<uint4*>(Vd)[e] = reinterpret_cast<const uint4*>(vs)[e];
+  }
+  for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < p.T; t += gridDim.x * blockDim.x) {
+    p.pos[slab * p.cap + t] = t;
+    p.score[slab * p.cap + t] = t < p.n_pinned ? __int_as_float(0x7f800000) : 0.f;
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0 && l == 0 && h == 0) {
+    p.len[b] = p.T;
+    p.tot[b] = p.T;
+    p.pinned[b] = p.n_pinned;
+    p.active[b] = 1;
+  }
+}
+
+}  // namespace dynts

@@ -1,0 +1,106 @@
+"""Full-size checks in the launch configuration the benchmark times (automatic cluster size and
+kernel variant): steady-state caches of the stated shapes are filled on the device from a seeded
+generator; sampled slabs are exported and the oracle recomputes them one by one."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from workloads import gen
+from oracle import dynts_oracle as O
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _steady_state(cfg, seed, rows):
+    gpu = H.make_gpu(cfg)
+    k, v = gen.torch_keys_values(cfg, seed, rows, "cuda:0")
+    gpu.prefill(k, v, n_pinned=cfg.prompt)
+    del k, v
+    return gpu
+
+
+def _check_sampled(gpu, cfg, seed, slabs, steps=3):
+    ring = gen.torch_step_ring(cfg, seed, steps, "cuda:0")
+    out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=H.tdtype(cfg), device="cuda:0")
+    delta = torch.zeros((cfg.layers, cfg.batch, cfg.kv_heads, gpu.capacity), dtype=torch.float32, device="cuda:0")
+    worst = dict(out=0.0, delta=0.0)
+    for s in range(steps):
+        orc = H.oracle_from_gpu(gpu, cfg, slabs=slabs)
+        q, k, v = ring[0][s], ring[1][s], ring[2][s]
+        gpu.decode_attn(q, k, v, out, delta)
+        gpu.synchronize()
+        gpu.poll_error()
+        qh, kh, vh = q.double().cpu().numpy(), k.double().cpu().numpy(), v.double().cpu().numpy()
+        og, dh = out.float().cpu().numpy(), delta.cpu().numpy()
+        G = cfg.group
+        for (l, b, h) in slabs:
+            sl = orc.slab(l, b, h)
+            sl.K[sl.n], sl.V[sl.n] = kh[l, b, h], vh[l, b, h]
+            n = sl.n + 1
+            alpha = O.attention_weights(qh[l, b, h * G:(h + 1) * G], sl.K[:n])
+            o_ref = O.attention_output(alpha, sl.V[:n])
+            worst["out"] = max(worst["out"], H.rel_err_vectors(og[l, b, h * G:(h + 1) * G], o_ref))
+            worst["delta"] = max(worst["delta"], float(np.abs(dh[l, b, h, :n] - alpha.sum(axis=0)).max()))
+    return worst
+
+
+def _sample_slabs(cfg, k, seed):
+    r = np.random.default_rng(seed)
+    all_ = [(l, b, h) for l in range(cfg.layers) for b in range(cfg.batch) for h in range(cfg.kv_heads)]
+    idx = r.choice(len(all_), size=min(k, len(all_)), replace=False)
+    return [all_[i] for i in idx] + [all_[0], all_[-1]]
+
+
+def test_config2_full_size():
+    cfg = W.get_config("c2_llama8b")
+    gpu = _steady_state(cfg, 2100, cfg.budget + 5)
+    slabs = _sample_slabs(cfg, 10, 1)
+    worst = _check_sampled(gpu, cfg, 2100, slabs, steps=cfg.evict_interval - 5 - 2)
+    assert worst["out"] <= H.TOL_OUT["bf16"] and worst["delta"] <= H.TOL_DELTA, worst
+    # run up to the eviction point with the accumulated (non-trivial) scores, then evict
+    ring = gen.torch_step_ring(cfg, 2101, 2, "cuda:0")
+    out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda:0")
+    for s in range(2):
+        gpu.decode_attn(ring[0][s], ring[1][s], ring[2][s], out)
+    assert gpu.len(0) == cfg.capacity
+    H.check_evict_bit_exact(gpu, cfg, 0, slabs=slabs)
+    assert gpu.len(0) == cfg.budget
+    worst = _check_sampled(gpu, cfg, 2102, slabs, steps=2)
+    assert worst["out"] <= H.TOL_OUT["bf16"] and worst["delta"] <= H.TOL_DELTA, worst
+    gpu.close()
+
+
+def test_config3_full_size():
+    cfg = W.get_config("c3_qwen7b")
+    gpu = _steady_state(cfg, 3100, cfg.capacity - 3)
+    slabs = _sample_slabs(cfg, 8, 2)
+    worst = _check_sampled(gpu, cfg, 3100, slabs, steps=3)
+    assert worst["out"] <= H.TOL_OUT["bf16"] and worst["delta"] <= H.TOL_DELTA, worst
+    assert gpu.len(0) == cfg.capacity
+    H.check_evict_bit_exact(gpu, cfg, 0, slabs=slabs)
+    assert gpu.len(15) == cfg.budget
+    gpu.close()
+    torch.cuda.empty_cache()
+
+
+def test_config4_full_size_ragged():
+    cfg = W.get_config("c4_ragged")
+    gpu = H.make_gpu(cfg)
+    one = cfg.scaled(batch=1)
+    r = np.random.default_rng(4100)
+    rows = []
+    for b in range(cfg.batch):
+        n = int(cfg.seq_budgets[b] + r.integers(1, cfg.evict_interval - 2))
+        k, v = gen.torch_keys_values(one, 4100 + b, n, "cuda:0")
+        gpu.prefill_seq(b, k[:, 0], v[:, 0], n_pinned=cfg.prompt)
+        rows.append(n)
+    assert [gpu.len(b) for b in range(cfg.batch)] == rows
+    slabs = _sample_slabs(cfg, 10, 3)
+    worst = _check_sampled(gpu, cfg, 4100, slabs, steps=2)
+    assert worst["out"] <= H.TOL_OUT["bf16"] and worst["delta"] <= H.TOL_DELTA, worst
+    H.check_evict_bit_exact(gpu, cfg, 0, slabs=slabs)
+    assert [gpu.len(b) for b in range(cfg.batch)] == list(cfg.seq_budgets)
+    gpu.close()
+    torch.cuda.empty_cache()
