@@ -1,0 +1,440 @@
+#!/usr/bin/env python
+"""Benchmark of the decode hot path: fused decode attention + importance accumulation every
+step, eviction + compaction every E steps, on a steady-state budget-limited KV cache.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2_llama8b] [--impl ours|reference]
+
+A step is one decode step of the whole stack (all layers) for the whole batch; every
+evict_interval-th step is followed by an eviction down to the budget.  Rank 0 prints one JSON
+line.  With N > 1 (torchrun) every rank runs an independent replica of the workload: the path
+has no exchange step, so there is no collective on the data path ("replicas only").
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as W  # noqa: E402
+from workloads import gen  # noqa: E402
+
+METRIC = "decode tokens/s at budget B"
+UNIT = "tokens/s"
+BYTES_PER_SLOT = 520          # K row 256 + V row 256 + fp32 score read-modify-write 8 (bf16 d=128, fp32 d=64)
+# DRAM bytes moved per algorithmic byte by the decode kernel, from the ncu capture summarised in
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of one launch / its algorithmic bytes).
+NCU_TRAFFIC_RATIO = None
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        return {
+            "sm_mhz": statistics.median(self.samples) if self.samples else None,
+            "sm_max_mhz": self.max_mhz,
+            "reasons": sorted(self.reasons),
+            "samples": len(self.samples),
+        }
+
+
+def physical_gpu_index(local_index: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+def setup_cache(cfg, seed, device):
+    """A cache in steady state: every sequence holds `budget` rows (the prompt rows pinned)."""
+    import torch
+    import paper_2601_18383_b200 as D
+    cache = D.Cache(cfg.layers, cfg.batch, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.budget, cfg.window,
+                    cfg.evict_interval, dtype=cfg.dtype, seq_budgets=cfg.seq_budgets, device=device)
+    if cfg.seq_budgets:
+        one = cfg.scaled(batch=1)
+        for b in range(cfg.batch):
+            k, v = gen.torch_keys_values(one, seed + b, cfg.seq_budgets[b], device)
+            cache.prefill_seq(b, k[:, 0], v[:, 0], n_pinned=cfg.prompt)
+    else:
+        k, v = gen.torch_keys_values(cfg, seed, cfg.budget, device)
+        cache.prefill(k, v, n_pinned=cfg.prompt)
+    del k, v
+    torch.cuda.empty_cache()
+    return cache
+
+
+def slots_in_step(cfg, lens):
+    return cfg.layers * cfg.kv_heads * sum(lens)
+
+
+def run_ours(args, cfg, rank, world, device):
+    import torch
+    import torch.distributed as dist
+
+    E = cfg.evict_interval
+    ring_n = 64
+    cache = setup_cache(cfg, 1000 * int(cfg.name[1]) + rank, device)
+    q_ring, k_ring, v_ring = gen.torch_step_ring(cfg, 77 + rank, ring_n, device)
+    out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=q_ring.dtype, device=device)
+    stream = torch.cuda.current_stream(device)
+
+    def step(i):
+        j = i % ring_n
+        cache.decode_attn(q_ring[j], k_ring[j], v_ring[j], out)
+        if (i + 1) % E == 0:
+            cache.evict(0)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(device)
+
+    # warm-up: at least one full eviction cycle so that scores and selection are non-trivial
+    warm = max(args.warmup, 3)
+    warm = (warm + E - 1) // E * E
+    for i in range(warm):
+        step(i)
+    barrier()
+    cache.poll_error()
+
+    # ---- timed region: exactly K steps, device-resident inputs --------------------------------
+    K = args.steps
+    sampler = ClockSampler(physical_gpu_index(torch.cuda.current_device()))
+    sampler.start()
+    launches0 = cache.launch_count()
+    lens = [cache.len(b) for b in range(cfg.batch)]
+    slot_steps = 0
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record(stream)
+    for i in range(K):
+        slot_steps += slots_in_step(cfg, [cache.len(b) + 1 for b in range(cfg.batch)])
+        step(i)
+    ev1.record(stream)
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop()
+    launches = cache.launch_count() - launches0
+    cache.poll_error()
+    if world > 1:
+        t = torch.tensor([ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    tokens = cfg.batch * K * world
+    value = tokens / (ms * 1e-3)
+
+    # ---- per-kernel durations (separate pass: event pairs around every launch) -----------------
+    Kp = min(K, 8 * E)
+    dec_events, ev_events, dec_bytes, ev_moved_bytes = [], [], [], []
+    for i in range(Kp):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        dec_bytes.append(BYTES_PER_SLOT * slots_in_step(cfg, [cache.len(bb) + 1 for bb in range(cfg.batch)]))
+        a.record(stream)
+        cache.decode_attn(q_ring[i % ring_n], k_ring[i % ring_n], v_ring[i % ring_n], out)
+        b.record(stream)
+        dec_events.append((a, b))
+        if (i + 1) % E == 0:
+            need = any(cache.len(bb) > (cfg.seq_budgets[bb] if cfg.seq_budgets else cfg.budget) for bb in range(cfg.batch))
+            if need:
+                # moved rows are known only on the device: read the first-moved index per slab
+                pos_before = None
+            a2, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            lens_before = [cache.len(bb) for bb in range(cfg.batch)]
+            a2.record(stream)
+            cache.evict(0)
+            b2.record(stream)
+            ev_events.append((a2, b2, lens_before))
+    torch.cuda.synchronize(device)
+    dec_ms = [a.elapsed_time(b) for a, b in dec_events]
+    dec_avg_ms = sum(dec_ms) / len(dec_ms)
+    dec_gbs = (sum(dec_bytes) / len(dec_bytes)) / (dec_avg_ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peaks()
+    algo_bytes = sum(dec_bytes) / len(dec_bytes)
+    roofline = {
+        "kernel": "decode_attn (fused append + attention + importance accumulation)",
+        "bound": "hbm", "achieved": round(dec_gbs, 1), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+        "frac": round(dec_gbs / peak, 4),
+        "traffic": None if NCU_TRAFFIC_RATIO is None else int(NCU_TRAFFIC_RATIO * algo_bytes),
+        "algorithmic_bytes_per_launch": int(algo_bytes), "avg_launch_us": round(dec_avg_ms * 1e3, 2),
+        "launches_timed": len(dec_ms),
+    }
+    evict = None
+    if ev_events:
+        ev_ms = [a.elapsed_time(b) for a, b, _ in ev_events]
+        evict = {"kernels": "evict_select + evict_compact", "avg_event_us": round(1e3 * sum(ev_ms) / len(ev_ms), 2),
+                 "events_timed": len(ev_ms)}
+
+    # ---- end to end through the host-buffer entry point ----------------------------------------
+    e2e = None
+    if rank == 0 or world > 1:
+        Ke = min(K, 4 * E)
+        hq = [q_ring[j].cpu().pin_memory() for j in range(ring_n)]
+        hk = [k_ring[j].cpu().pin_memory() for j in range(ring_n)]
+        hv = [v_ring[j].cpu().pin_memory() for j in range(ring_n)]
+        hout = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+        for i in range(3):
+            cache.decode_attn_host(hq[i], hk[i], hv[i], hout)
+        # re-align to the eviction cycle
+        while cache.len(0) % 1 == 0 and any(cache.len(bb) >= cache.capacity for bb in range(cfg.batch)):
+            cache.evict(0)
+        barrier()
+        t0 = time.perf_counter()
+        steps_done = 0
+        for i in range(Ke):
+            if any(cache.len(bb) + 1 > cache.capacity for bb in range(cfg.batch)):
+                cache.evict(0)
+            cache.decode_attn_host(hq[i % ring_n], hk[i % ring_n], hv[i % ring_n], hout)
+            steps_done += 1
+        torch.cuda.synchronize(device)
+        dt = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([dt], device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        e2e = {"value": round(cfg.batch * steps_done * world / dt, 1), "unit": UNIT,
+               "h2d_bytes_per_step": int(hq[0].numel() * hq[0].element_size() + 2 * hk[0].numel() * hk[0].element_size()),
+               "d2h_bytes_per_step": int(hout.numel() * hout.element_size()), "steps": steps_done,
+               "api": "dynts_decode_attn_host + dynts_evict"}
+
+    # ---- CPU baseline: the oracle, as it stands, on this machine's host cores (rank 0, N = 1) ------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = oracle_baseline(cfg, cache, q_ring, k_ring, v_ring, budget_s=args.cpu_seconds)
+
+    result = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": warm,
+        "ms_per_step": round(ms / K, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 inputs, fp32 accumulate" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "layers": cfg.layers, "batch": cfg.batch, "q_heads": cfg.q_heads,
+                   "kv_heads": cfg.kv_heads, "head_dim": cfg.head_dim, "budget": cfg.budget, "window": cfg.window,
+                   "evict_interval": E, "prompt_pinned": cfg.prompt, "dist": cfg.dist,
+                   "cache_bytes": cache.nbytes, "l2_policy": "inputs larger than L2 (KV cache %.0f MB vs 126 MB L2)" % (cache.nbytes / 1e6),
+                   "replicas": world},
+        "hbm_gbs_decode": round(dec_gbs, 1), "roofline": roofline, "evict": evict, "e2e": e2e,
+        "cpu_baseline": cpu, "clocks": clocks, "gpu_launches": int(launches),
+    }
+    cache.close()
+    return result
+
+
+def oracle_baseline(cfg, cache, q_ring, k_ring, v_ring, budget_s=20.0, slabs=None):
+    """Times oracle decode steps (and one eviction) on a bounded sample of the same workload: the
+    state of a subset of layers is exported from the device cache; throughput is scaled by the
+    fraction of slabs processed."""
+    import torch
+    from oracle import dynts_oracle as O
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    # sample: the first `nl` layers, all sequences and heads
+    total_slabs = cfg.layers * cfg.batch * cfg.kv_heads
+    nl = 1
+    sub = cfg.scaled(layers=nl)
+    orc = O.OracleCache(nl, cfg.batch, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.window, cache.capacity)
+    for b in range(cfg.batch):
+        for h in range(cfg.kv_heads):
+            K, V, pos, score = cache.export_slab(0, b, h)
+            s = orc.slab(0, b, h)
+            n = K.shape[0]
+            if n >= cache.capacity:
+                n = cache.capacity - 1
+            s.K[:n], s.V[:n] = K[:n].double().numpy(), V[:n].double().numpy()
+            s.pos[:n], s.score[:n], s.n = pos[:n].numpy(), score[:n].double().numpy(), n
+        orc.n_pinned[b] = cfg.prompt
+    q = q_ring[:, :nl].double().cpu().numpy()
+    k = k_ring[:, :nl].double().cpu().numpy()
+    v = v_ring[:, :nl].double().cpu().numpy()
+    t0 = time.perf_counter()
+    steps = 0
+    while time.perf_counter() - t0 < budget_s and steps < 4 * cfg.evict_interval:
+        if any(orc.slab(0, b, 0).n + 1 > cache.capacity for b in range(cfg.batch)):
+            O.evict(orc, list(cfg.seq_budgets) if cfg.seq_budgets else cfg.budget)
+        j = steps % q.shape[0]
+        O.decode_step(orc, q[j], k[j], v[j])
+        steps += 1
+    dt = time.perf_counter() - t0
+    frac = (nl * cfg.batch * cfg.kv_heads) / total_slabs
+    value = cfg.batch * steps / dt * frac
+    return {"value": round(value, 3), "unit": UNIT, "cores": int(threads), "kind": "oracle",
+            "sample": f"{steps} decode steps (+ evictions as they fall due) of layer 0 of {cfg.layers} "
+                      f"({nl * cfg.batch * cfg.kv_heads} of {total_slabs} slabs) in {dt:.1f} s; scaled by the slab fraction"}
+
+
+def run_reference(args, cfg, rank, world):
+    """The reference arm is the float64 oracle on the host cores (rank 0 only)."""
+    if rank != 0:
+        return None
+    from oracle import dynts_oracle as O
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    total_slabs = cfg.layers * cfg.batch * cfg.kv_heads
+    # calibrate one slab-step, then size the per-step sample so the whole run stays within ~2 min
+    one = cfg.scaled(layers=1, batch=1, kv_heads=1, q_heads=cfg.group, seq_budgets=None)
+    pk, pv = W.prompt_kv(one, 5, n_tokens=cfg.budget)
+    orc = O.OracleCache(1, 1, cfg.group, 1, cfg.head_dim, cfg.window, cfg.capacity)
+    O.prefill(orc, pk.astype(np.float64), pv.astype(np.float64), n_pinned=cfg.prompt)
+    st = W.DecodeStream(one, 5)
+    t0 = time.perf_counter()
+    for s in range(1, 4):
+        q, k, v = st.step(s)
+        O.decode_step(orc, q.astype(np.float64), k.astype(np.float64), v.astype(np.float64))
+    per_slab = (time.perf_counter() - t0) / 3
+    steps_total = args.steps + args.warmup
+    n_slabs = int(max(1, min(total_slabs, 100.0 / max(per_slab * steps_total, 1e-9))))
+    heads = min(cfg.kv_heads, n_slabs)
+    seqs = max(1, min(cfg.batch, n_slabs // heads))
+    layers = max(1, min(cfg.layers, n_slabs // (heads * seqs)))
+    sub = cfg.scaled(layers=layers, batch=seqs, kv_heads=heads, q_heads=heads * cfg.group,
+                     seq_budgets=cfg.seq_budgets[:seqs] if cfg.seq_budgets else None)
+    used = layers * seqs * heads
+    pk, pv = W.prompt_kv(sub, 6, n_tokens=min(sub.seq_budgets) if sub.seq_budgets else sub.budget)
+    orc = O.OracleCache(layers, seqs, sub.q_heads, heads, cfg.head_dim, cfg.window, cfg.capacity)
+    O.prefill(orc, pk.astype(np.float64), pv.astype(np.float64), n_pinned=cfg.prompt)
+    st = W.DecodeStream(sub, 6)
+    ring = [tuple(x.astype(np.float64) for x in st.step(s)) for s in range(1, 9)]
+    tgt = list(sub.seq_budgets) if sub.seq_budgets else sub.budget
+
+    def step(i):
+        O.decode_step(orc, *ring[i % len(ring)])
+        if (i + 1) % cfg.evict_interval == 0:
+            O.evict(orc, tgt)
+
+    for i in range(args.warmup):
+        step(i)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    dt = time.perf_counter() - t0
+    value = cfg.batch * args.steps / dt * (used / total_slabs)
+    sample = (f"each step = one oracle decode step (eviction every {cfg.evict_interval}) over {used} of {total_slabs} "
+              f"slabs ({layers} layers x {seqs} sequences x {heads} KV heads); throughput scaled by that fraction")
+    return {
+        "impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt / args.steps * 1e3 * (total_slabs / used), 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "layers": cfg.layers, "batch": cfg.batch, "q_heads": cfg.q_heads,
+                   "kv_heads": cfg.kv_heads, "head_dim": cfg.head_dim, "budget": cfg.budget, "window": cfg.window,
+                   "evict_interval": cfg.evict_interval},
+        "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": int(threads), "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=8192)
+    ap.add_argument("--warmup", type=int, default=128)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_llama8b", choices=sorted(W.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--cluster", type=int, default=0)
+    ap.add_argument("--variant", type=int, default=0)
+    args = ap.parse_args()
+    cfg = W.get_config(args.workload)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        res = run_reference(args, cfg, rank, world)
+        if res is not None:
+            print(json.dumps(res), flush=True)
+        return
+
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    if args.cluster or args.variant:
+        import paper_2601_18383_b200 as D
+        _orig = D.Cache.__init__
+
+        def _init(self, *a, **kw):
+            _orig(self, *a, **kw)
+            self.set_launch(args.cluster, args.variant)
+        D.Cache.__init__ = _init
+    res = run_ours(args, cfg, rank, world, device)
+    if rank == 0:
+        print(json.dumps(res), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -167,13 +167,13 @@ def test_host_buffer_entry_point_and_determinism():
 
 def test_capacity_error_and_inactive_sequences():
     import paper_2601_18383_b200 as D
-    cfg = W.get_config("c2_llama8b").scaled(layers=1, batch=2, prompt=30, budget=32, window=4, evict_interval=2)
+    cfg = W.get_config("c2_llama8b").scaled(layers=1, batch=2, prompt=28, budget=32, window=4, evict_interval=2)
     gpu = H.make_gpu(cfg)
     pk, pv = W.prompt_kv(cfg, 9)
     gpu.prefill(H.dev(pk, cfg), H.dev(pv, cfg))
     stream = W.DecodeStream(cfg, 9)
     out = torch.zeros((1, 2, cfg.q_heads, 128), dtype=torch.bfloat16, device="cuda:0")
-    for s in range(1, 5):
+    for s in range(1, 7):
         q, k, v = [H.dev(x, cfg) for x in stream.step(s)]
         gpu.decode_attn(q, k, v, out)
     assert gpu.len(0) == 34 == gpu.capacity
