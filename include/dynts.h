@@ -134,6 +134,34 @@ dynts_status_t dynts_evict(dynts_cache_t* c, int budget);
 /* Eviction with one target per sequence; seq_targets: host [Nb]. */
 dynts_status_t dynts_evict_ex(dynts_cache_t* c, const int* seq_targets);
 
+/* No counterpart in the paper: the eviction of Section 4.2 for callers that must not allocate.
+ *
+ * Some callers cannot call cudaMalloc where they need an eviction: code that runs inside a
+ * framework's memory-pool critical section, a real-time serving loop that forbids allocator
+ * calls after start-up, or a process whose whole device memory was handed to another allocator.
+ * This entry point evicts caller-owned slabs in place and allocates nothing, on the host or the
+ * device, and calls no routine that allocates (none of cudaMalloc, cudaFree, torch).  The
+ * gather list that connects the selection kernel to the compaction kernel, which a cache
+ * object keeps in its own storage, lives here in a fixed 4 MiB array built into the library's
+ * device image (every GPU that loads the library holds it until the process exits).
+ *
+ *   K, V:   device [n_slabs][capacity][head_dim] in `dtype`, compacted in place
+ *   pos:    device [n_slabs][capacity] int32;  score: device [n_slabs][capacity] fp32
+ *   n_rows: rows currently valid in every slab; n_pinned: leading rows never evicted
+ * Same selection rule, tie-break and stable compaction as dynts_evict; afterwards every slab
+ * holds min(n_rows, target) rows (the caller tracks the length).  Asynchronous on `stream`.
+ *
+ * Limits and caveats:
+ *  - n_slabs * capacity (+ a small header) must fit the built-in scratch: about one million
+ *    rows in total.  Larger requests return DYNTS_ERR_CAPACITY and launch nothing.
+ *  - All calls on one GPU share the array, which keeps the previous call's contents; the entry
+ *    point rewrites every word it later reads, so nothing needs clearing.  Two calls whose
+ *    kernels may overlap on the GPU (different streams) race on it: serialise them.
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current); make that first call before any stream capture begins. */
+dynts_status_t dynts_evict_noalloc(void* K, void* V, int* pos, float* score, int n_slabs, int head_dim, int dtype,
+                                   int capacity, int n_rows, int n_pinned, int window, int target, void* stream);
+
 /* ---- sequence management and inspection ---------------------------------------------------- */
 
 /* Ragged batches: mark a sequence finished (length 0, inactive) until its next prefill_seq. */

@@ -69,6 +69,7 @@ _sigs = {
     "dynts_decode_attn_host": (C.c_int, [_P, _P, _P, _P, _P]),
     "dynts_evict": (C.c_int, [_P, C.c_int]),
     "dynts_evict_ex": (C.c_int, [_P, C.POINTER(C.c_int)]),
+    "dynts_evict_noalloc": (C.c_int, [_P, _P, _P, _P] + [C.c_int] * 8 + [_P]),
     "dynts_seq_reset": (C.c_int, [_P, C.c_int]),
     "dynts_cache_len": (C.c_int, [_P, C.c_int]),
     "dynts_cache_capacity": (C.c_int, [_P]),
@@ -185,6 +186,13 @@ def dynts_evict(c, budget=0):
 def dynts_evict_ex(c, seq_targets: Sequence[int]):
     arr = (C.c_int * len(seq_targets))(*[int(x) for x in seq_targets])
     return _check(lib.dynts_evict_ex(c, arr))
+
+
+def dynts_evict_noalloc(K, V, pos, score, n_slabs, head_dim, dtype, capacity, n_rows, n_pinned, window, target,
+                        stream=None):
+    """In-place eviction of caller-owned slabs without any allocation (see include/dynts.h)."""
+    return _check(lib.dynts_evict_noalloc(_ptr(K), _ptr(V), _ptr(pos), _ptr(score), n_slabs, head_dim, dtype,
+                                          capacity, n_rows, n_pinned, window, target, stream))
 
 
 def dynts_seq_reset(c, seq):

@@ -11,6 +11,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -673,4 +674,99 @@ dynts_status_t dynts_cache_set_launch(dynts_cache_t* c, int cluster, int variant
 
 long long dynts_cache_launch_count(const dynts_cache_t* c) { return c ? c->launches : -1; }
 
+/* ---- eviction for callers that cannot allocate -------------------------------------------- */
+
+}  // extern "C" (the scratch array and its helpers have internal linkage)
+
+namespace {
+
+// Scratch of dynts_evict_noalloc: a small header (length, pinned, target, status), then the
+// per-slab headers, then the gather lists.  Every GPU that loads this library holds these
+// 4 MiB until the process exits.
+constexpr size_t kNoAllocInts = (size_t)1 << 20;
+constexpr size_t kNoAllocHeaderInts = 64;
+static __device__ __align__(256) int g_noalloc_scratch[kNoAllocInts];
+
+constexpr int kMaxDevices = 64;
+int* g_noalloc_ptr[kMaxDevices] = {nullptr};
+std::mutex g_noalloc_mutex;
+
+__global__ void noalloc_setup_kernel(int* hdr, int n_rows, int n_pinned, int target) {
+  hdr[0] = n_rows;    // plays the role of the per-sequence length array (one sequence)
+  hdr[1] = n_pinned;
+  hdr[2] = target;
+  hdr[3] = 0;         // status word
+}
+
+}  // namespace
+
+extern "C" {
+
+dynts_status_t dynts_evict_noalloc(void* K, void* V, int* pos, float* score, int n_slabs, int head_dim, int dtype,
+                                   int capacity, int n_rows, int n_pinned, int window, int target, void* stream) {
+  if (!K || !V || !pos || !score) return fail(DYNTS_ERR_INVALID_ARG, "NULL tensor pointer");
+  if (!aligned16(K) || !aligned16(V)) return fail(DYNTS_ERR_INVALID_ARG, "K and V must be 16-byte aligned");
+  if (dtype != DYNTS_BF16 && dtype != DYNTS_FP32) return fail(DYNTS_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+  if (n_slabs < 1 || head_dim < 8 || head_dim % 8 || head_dim > 256 || capacity < 1)
+    return fail(DYNTS_ERR_INVALID_ARG, "bad shape: n_slabs %d head_dim %d capacity %d", n_slabs, head_dim, capacity);
+  if (n_rows < 0 || n_rows > capacity || n_pinned < 0 || n_pinned > n_rows || window < 0 || target < 1)
+    return fail(DYNTS_ERR_INVALID_ARG, "bad lengths: n_rows %d n_pinned %d window %d target %d", n_rows, n_pinned,
+                window, target);
+  const size_t hdr_ints = align_up((size_t)n_slabs * 4, 64);
+  const size_t need = kNoAllocHeaderInts + hdr_ints + (size_t)n_slabs * capacity;
+  if (need > kNoAllocInts)
+    return fail(DYNTS_ERR_CAPACITY,
+                "n_slabs * capacity = %zu rows need %zu scratch ints; the built-in scratch holds %zu (about %zu rows)",
+                (size_t)n_slabs * capacity, need, kNoAllocInts, kNoAllocInts - kNoAllocHeaderInts - hdr_ints);
+  if ((size_t)capacity * 8 > 200 * 1024)
+    return fail(DYNTS_ERR_CAPACITY, "capacity %d exceeds the selection kernel's shared memory", capacity);
+  if (n_rows <= target) return DYNTS_OK;  // nothing to evict
+  if (n_pinned + window > target)
+    return fail(DYNTS_ERR_BUDGET, "question window %d + local window %d exceed target %d", n_pinned, window, target);
+
+  int dev = -1;
+  CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return fail(DYNTS_ERR_INVALID_ARG, "device index %d not supported", dev);
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);  // the scratch is shared: one call at a time
+  if (!g_noalloc_ptr[dev]) {
+    // Once per device, with that device current: the array's name is only a host-side stand-in,
+    // the kernels need its device address.
+    int* ptr = nullptr;
+    CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_noalloc_scratch));
+    CUDA_TRY(cudaFuncSetAttribute(dynts::evict_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    g_noalloc_ptr[dev] = ptr;
+  }
+  int* base = g_noalloc_ptr[dev];
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  dynts::EvictParams p;
+  p.K = K;
+  p.V = V;
+  p.pos = pos;
+  p.score = score;
+  p.len = base + 0;
+  p.pinned = base + 1;
+  p.target = base + 2;
+  p.err = base + 3;
+  p.hdr = base + kNoAllocHeaderInts;
+  p.src = base + kNoAllocHeaderInts + hdr_ints;
+  p.L = 1;
+  p.Nb = 1;
+  p.Hkv = n_slabs;
+  p.d = head_dim;
+  p.cap = capacity;
+  p.window = window;
+  p.elt_bytes = elt_bytes_of(dtype);
+  noalloc_setup_kernel<<<1, 1, 0, st>>>(base, n_rows, n_pinned, target);
+  CUDA_TRY(cudaGetLastError());
+  dynts::evict_select_kernel<<<(unsigned)n_slabs, dynts::kSelectThreads, (size_t)capacity * 8, st>>>(p);
+  CUDA_TRY(cudaGetLastError());
+  const int pieces = head_dim * p.elt_bytes / 16;
+  const unsigned groups = (unsigned)((pieces + 3) / 4);
+  dynts::evict_compact_kernel<<<dim3(2 * groups, (unsigned)n_slabs, 1), dynts::kCompactThreads, 0, st>>>(p);
+  CUDA_TRY(cudaGetLastError());
+  return DYNTS_OK;
+}
+
 }  // extern "C"
+
