@@ -80,22 +80,25 @@ class OracleCache:
         self.group = q_heads // kv_heads
         self.window = window
         self.capacity = capacity
-        self.slabs = [[[Slab(capacity, head_dim) for _ in range(kv_heads)]
-                       for _ in range(batch)] for _ in range(layers)]
+        self._slabs = {}                 # (layer, seq, head) -> Slab, storage created on first use
         self.n_pinned = [0] * batch      # M: question rows, immune to eviction
         self.next_pos = [0] * batch      # position id given to the next appended token
 
     def slab(self, layer: int, seq: int, head: int) -> Slab:
-        return self.slabs[layer][seq][head]
+        key = (layer, seq, head)
+        s = self._slabs.get(key)
+        if s is None:
+            s = self._slabs[key] = Slab(self.capacity, self.head_dim)
+        return s
 
     def length(self, seq: int) -> int:
-        return self.slabs[0][seq][0].n
+        return self.slab(0, seq, 0).n
 
     def units(self):
         for l in range(self.layers):
             for b in range(self.batch):
                 for h in range(self.kv_heads):
-                    yield l, b, h, self.slabs[l][b][h]
+                    yield l, b, h, self.slab(l, b, h)
 
 
 def prefill(cache: OracleCache, k: np.ndarray, v: np.ndarray, n_pinned: Optional[int] = None,
@@ -112,7 +115,7 @@ def prefill(cache: OracleCache, k: np.ndarray, v: np.ndarray, n_pinned: Optional
         assert 0 <= m <= T <= cache.capacity
         for l in range(cache.layers):
             for h in range(cache.kv_heads):
-                s = cache.slabs[l][b][h]
+                s = cache.slab(l, b, h)
                 src_k = k[l, b, h] if seq is None else k[l, h]
                 src_v = v[l, b, h] if seq is None else v[l, h]
                 s.K[:T] = src_k
