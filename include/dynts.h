@@ -196,9 +196,11 @@ dynts_status_t dynts_poll_error(dynts_cache_t* c);
 /* Wait for the cache's stream. */
 dynts_status_t dynts_synchronize(dynts_cache_t* c);
 
-/* Launch configuration of the decode kernel, for tuning: cluster size (1, 2, 4, 8 or 16; 0 =>
- * automatic) and kernel variant (0 => automatic, 1 => generic FMA kernel, 2 => tensor-core kernel;
- * the tensor-core kernel needs bf16, d = 128, G <= 8). */
+/* Launch configuration of the decode kernel, for tuning.  variant: 0 => automatic, 1 => generic
+ * FMA kernel (any supported shape), 2 => tensor-core kernel with one thread-block cluster per
+ * slab, 3 => persistent streaming tensor-core kernel (TMA ring, the default where it applies);
+ * 2 and 3 need bf16, d = 128, G <= 8.  cluster: for variants 1 and 2 the cluster size (1, 2, 4,
+ * 8 or 16; 0 => automatic); for variant 3 the CTAs per SM (1 or 2; anything else => 2). */
 dynts_status_t dynts_cache_set_launch(dynts_cache_t* c, int cluster, int variant);
 
 /* Number of kernels this library has launched on behalf of the cache so far. */

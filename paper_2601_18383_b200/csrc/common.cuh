@@ -11,6 +11,8 @@ constexpr int kMaxGroup = 8;        // query heads per KV head handled by the ke
 constexpr int kErrTileOverflow = 1; // device status bits
 constexpr int kErrLenOverflow = 2;
 constexpr int kErrEvictSmem = 4;
+constexpr int kErrTimeout = 8;           // a bounded wait on a shared-memory barrier gave up
+constexpr int kErrStreamBounds = 16; // the streaming kernel's chunk list left the slab bounds
 
 // One decode launch covers `n_layers` layers starting at `layer0`.
 struct DecodeParams {
@@ -28,6 +30,10 @@ struct DecodeParams {
   const int* active;  // [Nb]
   unsigned int* ticket;
   int* err;           // pinned host status word
+  float* logit;       // streaming kernel: scaled logits of the step, [L, Nb, Hkv, G, cap]
+  float* part;        // streaming kernel: per-CTA partials, [CTAs][2][O 8x128 | m 8 | l 8]
+  int* arrive;        // streaming kernel: per-slab arrival counters, zero between launches
+  int* dbg;           // streaming kernel: 32 ints describing the first failed self-check
   int layer0, n_layers, Nb, Hkv, G, d, cap;
   int advance;        // 1: the last CTA to finish increments len/tot of active sequences
   int tile_tokens;    // rows of logits a CTA can hold in shared memory

@@ -1,0 +1,564 @@
+// Persistent streaming variant of the fused decode attention + importance accumulation
+// (Eq. 4-6) for sm_100a: bf16 slabs, head_dim 128, G <= 8.
+//
+// Work decomposition.  Every slab (layer, sequence, KV head) of n rows is cut into chunks of 32
+// rows; the chunks of all slabs of the launch form one list, ordered slab by slab, and the
+// persistent grid (two CTAs per SM) cuts that list into equal contiguous pieces, one per CTA
+// ("stream-K": a CTA usually starts in the middle of one slab, covers some slabs completely and
+// stops in the middle of another).  Inside a CTA one producer thread walks the piece and issues
+// TMA tile loads (cp.async.bulk.tensor, 128-byte swizzle, no multicast) of the K and V rows of
+// each chunk into a 6-stage shared-memory ring guarded by mbarriers, running ahead of the four
+// consumer warps across chunk and slab boundaries, so the HBM stream never pauses for an
+// epilogue.  Chunk i of a CTA goes to stage i mod 6 and to the warp pair i mod 2; with an even
+// stage count every stage is always consumed by the same two warps, which is what makes the
+// parity wait on its barrier unambiguous (a waiter is never two phases away from the barrier).
+// The consumer warps take 16 rows each: QK^T and PV run on the tensor pipe
+// (mma.sync m16n8k16, bf16 in, fp32 accumulate) with operands fetched by ldmatrix from the
+// swizzled tiles, online softmax in registers.
+//
+// The final softmax normaliser of a slab is known only when all its chunks are done, and the
+// importance score needs the normalised weights (Eq. 6).  So every row's scaled logits go to a
+// scratch array (fp32, [slab][head][row], 4*G bytes per row beside the 512 bytes of K and V), and
+// each CTA that finishes its part of a slab publishes a partial (max, sum, unnormalised output)
+// and takes a ticket on the slab's arrival counter.  Whoever arrives last combines the partials,
+// writes the output and then walks the slab's logits once to do the single read-modify-write of
+// every score row.  Nobody ever waits for another CTA: there is no inter-CTA spin, no float
+// atomic, one writer per score row and per output element.
+#pragma once
+
+#include <cuda.h>
+#include <math_constants.h>
+
+#include "common.cuh"
+#include "decode_attn.cuh"
+
+namespace dynts {
+
+constexpr int kStRows = 32;                      // rows per chunk = per ring stage
+constexpr int kStStages = 6;                     // even: chunk i of a CTA goes to stage i % 6 and to the warp pair i % 2,
+                                                 // so every stage is always consumed by the same two warps
+constexpr int kStConsumerWarps = 4;
+constexpr int kStConsumers = kStConsumerWarps * 32;
+constexpr int kStThreads = kStConsumers + 32;    // + one producer warp
+constexpr int kStBoxBytes = kStRows * 128;       // one TMA box: 32 rows x 64 bf16
+constexpr int kStStageBytes = 4 * kStBoxBytes;   // K low/high half of head_dim, V low/high
+constexpr int kStCombFloats = kStConsumerWarps * 4 * 128;
+constexpr int kStMaxCtas = 320;                  // partial slots exist for this many CTAs
+constexpr int kStPartStride = 8 * 128 + 16;      // floats per partial: O[8][128], m[8], l[8]
+constexpr int kStMaxBatch = 512;                 // sequences whose chunk prefix fits shared memory
+constexpr uint32_t kStSpinLimit = 1u << 22;      // bounded mbarrier polling
+
+__host__ __device__ inline size_t stream_smem_bytes(int Nb) {
+  return 1024 /* alignment slack */ + (size_t)kStStages * kStStageBytes + sizeof(float) * kStCombFloats +
+         sizeof(float) * (2 * kStConsumerWarps * 8 + kStConsumerWarps * 8 + 4 * 8) + 16 * kStStages + 64 +
+         sizeof(int) * (2 * (size_t)Nb + 2);
+}
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Polls with an iteration limit.  On expiry the status word gets the timeout bit and the CTA-wide
+// abort flag is raised; every later wait of the CTA then returns at once, so the kernel ends (its
+// results are void, which the status word says).
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err) {
+  if (*abort_flag) return;
+  for (uint32_t i = 0; i < kStSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return;
+    if ((i & 1023u) == 1023u && *abort_flag) return;
+  }
+  *abort_flag = 1;
+  atomicOr(err, kErrTimeout);
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
+                                                  uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kStConsumers) : "memory"); }
+
+// ---- the chunk list ---------------------------------------------------------------------------
+// Chunk index g (within the launch) -> layer-major, then sequence, KV head, chunk of the slab.
+// s_cnt[b] = chunks of one slab of sequence b (0 if inactive); s_off[b] = Hkv * sum of s_cnt
+// below b; s_off[Nb] = chunks per layer.
+struct StCursor {
+  int lrel, b, h, chunk, cb;
+};
+
+__device__ __forceinline__ void cursor_seek(StCursor& c, long long g, const int* s_off, const int* s_cnt, int Nb) {
+  const int per_layer = s_off[Nb];
+  c.lrel = (int)(g / per_layer);
+  int r = (int)(g % per_layer);
+  int lo = 0, hi = Nb;  // largest b with s_off[b] <= r and s_cnt[b] > 0
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (s_off[mid] <= r) lo = mid; else hi = mid;
+  }
+  c.b = lo;
+  c.cb = s_cnt[lo];
+  r -= s_off[lo];
+  c.h = r / c.cb;
+  c.chunk = r % c.cb;
+}
+
+// Moves to chunk 0 of the next slab in list order.
+__device__ __forceinline__ void cursor_next_slab(StCursor& c, const int* s_cnt, int Nb, int Hkv) {
+  c.chunk = 0;
+  if (++c.h < Hkv) return;
+  c.h = 0;
+  do {
+    if (++c.b == Nb) {
+      c.b = 0;
+      ++c.lrel;
+    }
+  } while (s_cnt[c.b] == 0);
+  c.cb = s_cnt[c.b];
+}
+
+__global__ void __launch_bounds__(kStThreads, 2)
+decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmK,
+                          const __grid_constant__ CUtensorMap tmV) {
+  constexpr int d = 128;
+  const int G = p.G, Nb = p.Nb, Hkv = p.Hkv;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  extern __shared__ uint8_t st_smem_raw[];
+  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(st_smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* s_stage = sm;                                             // [stages][4 boxes]
+  float* s_comb = reinterpret_cast<float*>(s_stage + kStStages * kStStageBytes);  // [warps][4 heads][128]
+  float* s_wm = s_comb + kStCombFloats;                              // [warps][8]
+  float* s_wl = s_wm + kStConsumerWarps * 8;
+  float* s_sc = s_wl + kStConsumerWarps * 8;                         // [warps][8] rescale of each warp's partial
+  float* s_cm = s_sc + kStConsumerWarps * 8;                         // [8] CTA partial max
+  float* s_cl = s_cm + 8;                                            // [8] CTA partial sum
+  float* s_finM = s_cl + 8;                                          // [8] slab max
+  float* s_finf = s_finM + 8;                                        // [8] 1 / slab sum
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_finf + 8);         // full[stages], empty[stages]
+  int* s_flags = reinterpret_cast<int*>(s_bar + 2 * kStStages);      // [0] abort, [1] last arriver, [2+s] armed phase
+  int* s_cnt = s_flags + 16;                                         // [Nb]
+  int* s_off = s_cnt + Nb;                                           // [Nb + 1]
+  volatile int* s_abort = s_flags;
+
+  const uint32_t bar_full = smem_u32(s_bar), bar_empty = smem_u32(s_bar + kStStages);
+
+  // ---- per-CTA set-up: barriers and the chunk prefix of the sequences -------------------------
+  if (tid == 0) {
+    for (int s = 0; s < kStStages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 2);  // the two warps that consume the stage
+    }
+    for (int i = 0; i < 16; ++i) s_flags[i] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    int carry = 0;
+    for (int b0 = 0; b0 < Nb; b0 += 32) {
+      const int b = b0 + lane;
+      int c = 0;
+      if (b < Nb && p.active[b]) c = (p.len[b] + 1 + kStRows - 1) / kStRows;
+      int incl = c;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      if (b < Nb) {
+        s_cnt[b] = c;
+        s_off[b] = (carry + incl - c) * Hkv;
+      }
+      carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) s_off[Nb] = carry * Hkv;
+  }
+  __syncthreads();
+
+  const long long per_layer = s_off[Nb];
+  const long long total = per_layer * p.n_layers;
+  const long long per_cta = (total + gridDim.x - 1) / gridDim.x;
+  const long long g_begin = per_cta * blockIdx.x;
+  long long g_end = g_begin + per_cta;
+  if (g_end > total) g_end = total;
+  const int cnt = g_end > g_begin ? (int)(g_end - g_begin) : 0;
+
+  if (cnt > 0 && warp == kStConsumerWarps) {
+    // =========================== producer: one thread feeds the ring ===========================
+    if (lane == 0) {
+      StCursor c;
+      cursor_seek(c, g_begin, s_off, s_cnt, Nb);
+      for (int it = 0; it < cnt; ++it) {
+        const int stage = it % kStStages;
+        const uint32_t ph = (uint32_t)(it / kStStages) & 1u;
+        mbar_wait(bar_empty + 8 * stage, ph ^ 1u, s_abort, p.err);
+        if (*s_abort) break;
+        const size_t slab = ((size_t)(p.layer0 + c.lrel) * Nb + c.b) * Hkv + c.h;
+        const int n_old = p.len[c.b];
+        if (c.lrel >= p.n_layers || c.b >= Nb || c.h >= Hkv || n_old + 1 > p.cap || (c.chunk + 1) * kStRows > p.cap + kStRows ||
+            (smem_u32(s_stage + (size_t)stage * kStStageBytes) & 1023u) != 0u) {
+          // the chunk list and the slab bounds disagree: record, stop feeding, let the waits expire
+          atomicOr(p.err, kErrStreamBounds);
+          p.dbg[0] = c.lrel; p.dbg[1] = c.b; p.dbg[2] = c.h; p.dbg[3] = c.chunk; p.dbg[4] = n_old; p.dbg[5] = it;
+          p.dbg[6] = (int)blockIdx.x; p.dbg[7] = (int)smem_u32(s_stage);
+          *s_abort = 1;
+          break;
+        }
+        const uint32_t full = bar_full + 8 * stage;
+        const uint32_t dst = smem_u32(s_stage + (size_t)stage * kStStageBytes);
+        mbar_arrive_expect_tx(full, kStStageBytes);
+        s_flags[2 + stage] = 1 + (int)ph;  // phase of the loads now in flight, for the drain below
+        const int row = (int)(slab * (size_t)p.cap) + c.chunk * kStRows;
+        tma_load_2d(dst, &tmK, 0, row, full);
+        tma_load_2d(dst + kStBoxBytes, &tmK, 64, row, full);
+        tma_load_2d(dst + 2 * kStBoxBytes, &tmV, 0, row, full);
+        tma_load_2d(dst + 3 * kStBoxBytes, &tmV, 64, row, full);
+        if (++c.chunk == c.cb) cursor_next_slab(c, s_cnt, Nb, Hkv);
+      }
+    }
+  } else if (cnt > 0) {
+    // ================================== consumers ============================================
+    const int gid = lane >> 2, tig = lane & 3;
+    const int pair = warp >> 1, u16 = (warp & 1) * 16;  // pair: parity of the chunks (items) this warp takes
+    // ldmatrix lane address inside a box: row of the warp's 16-row unit, 16-byte chunk parity
+    const int lrow = u16 + ((lane >> 4) << 3) + (lane & 7);
+    const int lchk = (lane >> 3) & 1;
+    StCursor c;
+    cursor_seek(c, g_begin, s_off, s_cnt, Nb);
+    int it = 0;
+    while (it < cnt) {
+      // ---- one segment: chunks [c.chunk, c.chunk + seg) of one slab -----------------------------
+      const int seg = min(c.cb - c.chunk, cnt - it);
+      const size_t unit = ((size_t)c.lrel * Nb + c.b) * Hkv + c.h;
+      const size_t slab = ((size_t)(p.layer0 + c.lrel) * Nb + c.b) * Hkv + c.h;
+      const int n_old = p.len[c.b];
+      const int n = n_old + 1;
+      float* lg = p.logit + slab * (size_t)G * p.cap;  // [G][cap]
+      if (c.lrel >= p.n_layers || c.b >= Nb || c.h >= Hkv || n > p.cap || seg < 1 || c.chunk + seg > c.cb) {
+        if (tid == 0) {
+          atomicOr(p.err, kErrStreamBounds);
+          p.dbg[8] = c.lrel; p.dbg[9] = c.b; p.dbg[10] = c.h; p.dbg[11] = c.chunk; p.dbg[12] = n; p.dbg[13] = it;
+          p.dbg[14] = (int)blockIdx.x; p.dbg[15] = seg;
+          *s_abort = 1;
+        }
+        break;  // uniform over the consumer warps
+      }
+
+      // Query fragments of the group, straight from global memory (2 KB at most, L2-resident):
+      // a0 = Q[head gid][16kk + 2tig, +1], a2 = Q[head gid][16kk + 8 + 2tig, +1].
+      uint32_t qa[8][2];
+      {
+        const uint32_t* hq = reinterpret_cast<const uint32_t*>(reinterpret_cast<const __nv_bfloat16*>(p.q) + unit * (size_t)G * d);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          qa[kk][0] = gid < G ? __ldg(hq + gid * 64 + 8 * kk + tig) : 0u;
+          qa[kk][1] = gid < G ? __ldg(hq + gid * 64 + 8 * kk + 4 + tig) : 0u;
+        }
+      }
+
+      float o[8][4];
+#pragma unroll
+      for (int mb = 0; mb < 8; ++mb)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[mb][e] = 0.f;
+      float m_run = -CUDART_INF_F, l_part = 0.f;
+
+      for (int k = (pair ^ it) & 1; k < seg; k += 2) {
+        const int item = it + k;  // item & 1 == pair
+        const int stage = item % kStStages;
+        const int row0 = (c.chunk + k) * kStRows;
+        mbar_wait(bar_full + 8 * stage, (uint32_t)(item / kStStages) & 1u, s_abort, p.err);
+        __syncwarp();
+        uint8_t* st = s_stage + (size_t)stage * kStStageBytes;
+        const int t0 = row0 + u16;  // first row of this warp's unit
+        if (t0 < n) {
+          if (n_old >= t0 && n_old < t0 + 16) {
+            // a1: the appended row.  The tile holds whatever the slab had at row n_old; overwrite
+            // it in shared memory with k_new / v_new and store the row to the slab.
+            const int r = n_old - row0, ch = lane & 15, isv = lane >> 4;
+            const __nv_bfloat16* nrow = reinterpret_cast<const __nv_bfloat16*>(isv ? p.v_new : p.k_new) + unit * d;
+            const uint4 val = __ldg(reinterpret_cast<const uint4*>(nrow) + ch);
+            uint8_t* box = st + (2 * isv + (ch >> 3)) * kStBoxBytes;
+            *reinterpret_cast<uint4*>(box + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = val;
+            __nv_bfloat16* grow = reinterpret_cast<__nv_bfloat16*>(isv ? p.V : p.K) + (slab * (size_t)p.cap + n_old) * d;
+            reinterpret_cast<uint4*>(grow)[ch] = val;
+            if (lane == 0) p.pos[slab * (size_t)p.cap + n_old] = p.tot[c.b];
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+          }
+          // a2: S^T[head][token] = Q K^T for two blocks of 8 tokens
+          // (all fragment loads of a phase are issued before its mma chain, so their shared-memory
+          // latency overlaps; the V fragments are fetched before the softmax arithmetic)
+          float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+          const uint32_t kbase = smem_u32(st) + lrow * 128;
+          const uint32_t vbase = kbase + 2 * kStBoxBytes;
+          uint32_t fr[8][4];
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const int chk = ((2 * kk) & 7) + lchk;
+            ldmatrix_x4(kbase + (kk >> 2) * kStBoxBytes + ((chk ^ (lrow & 7)) << 4), fr[kk][0], fr[kk][1], fr[kk][2], fr[kk][3]);
+          }
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            mma_bf16_m16n8k16(s0, qa[kk][0], 0u, qa[kk][1], 0u, fr[kk][0], fr[kk][1]);
+            mma_bf16_m16n8k16(s1, qa[kk][0], 0u, qa[kk][1], 0u, fr[kk][2], fr[kk][3]);
+          }
+#pragma unroll
+          for (int mb = 0; mb < 8; ++mb) {
+            const int chk = ((2 * mb) & 7) + lchk;
+            ldmatrix_x4_trans(vbase + (mb >> 2) * kStBoxBytes + ((chk ^ (lrow & 7)) << 4), fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3]);
+          }
+          // a3: online softmax of head gid over the unit's 16 tokens
+          const int tk = t0 + 2 * tig;
+          float x[4];
+          x[0] = (gid < G && tk < n) ? s0[0] * p.scale_log2 : -CUDART_INF_F;
+          x[1] = (gid < G && tk + 1 < n) ? s0[1] * p.scale_log2 : -CUDART_INF_F;
+          x[2] = (gid < G && tk + 8 < n) ? s1[0] * p.scale_log2 : -CUDART_INF_F;
+          x[3] = (gid < G && tk + 9 < n) ? s1[1] * p.scale_log2 : -CUDART_INF_F;
+          if (gid < G) {
+            float* t = lg + (size_t)gid * p.cap + tk;
+            if (tk < n) t[0] = x[0];
+            if (tk + 1 < n) t[1] = x[1];
+            if (tk + 8 < n) t[8] = x[2];
+            if (tk + 9 < n) t[9] = x[3];
+          }
+          float um = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+          um = fmaxf(um, __shfl_xor_sync(0xffffffffu, um, 1));
+          um = fmaxf(um, __shfl_xor_sync(0xffffffffu, um, 2));
+          const float m_new = fmaxf(m_run, um);
+          const float m_safe = (m_new == -CUDART_INF_F) ? 0.f : m_new;
+          const float corr = fast_exp2(m_run - m_safe);
+          const float p0 = fast_exp2(x[0] - m_safe), p1 = fast_exp2(x[1] - m_safe);
+          const float p2 = fast_exp2(x[2] - m_safe), p3 = fast_exp2(x[3] - m_safe);
+          l_part = l_part * corr + ((p0 + p1) + (p2 + p3));
+          m_run = m_new;
+          const uint32_t pb0 = pack_bf16x2(p0, p1);  // B fragment: tokens 2tig, 2tig+1 of head gid
+          const uint32_t pb1 = pack_bf16x2(p2, p3);  // tokens 2tig+8, 2tig+9
+          const float c_even = __shfl_sync(0xffffffffu, corr, 8 * tig);      // head 2tig
+          const float c_odd = __shfl_sync(0xffffffffu, corr, 8 * tig + 4);   // head 2tig+1
+          // a4: O^T[d][head] += V^T P; accumulator mb covers d = 16mb + gid (+8), heads 2tig, 2tig+1
+#pragma unroll
+          for (int mb = 0; mb < 8; ++mb) {
+            o[mb][0] *= c_even;
+            o[mb][1] *= c_odd;
+            o[mb][2] *= c_even;
+            o[mb][3] *= c_odd;
+            mma_bf16_m16n8k16(o[mb], fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3], pb0, pb1);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_empty + 8 * stage);
+      }
+
+      // ---- segment end: warp partials -> CTA partial ---------------------------------------------
+      l_part += __shfl_xor_sync(0xffffffffu, l_part, 1);
+      l_part += __shfl_xor_sync(0xffffffffu, l_part, 2);
+      if (tig == 0) {
+        s_wm[warp * 8 + gid] = m_run;
+        s_wl[warp * 8 + gid] = l_part;
+      }
+      consumer_sync();
+      if (tid < 8) {
+        float mc = -CUDART_INF_F;
+#pragma unroll
+        for (int w = 0; w < kStConsumerWarps; ++w) mc = fmaxf(mc, s_wm[w * 8 + tid]);
+        const float ms = (mc == -CUDART_INF_F) ? 0.f : mc;
+        float l = 0.f;
+#pragma unroll
+        for (int w = 0; w < kStConsumerWarps; ++w) {
+          const float f = fast_exp2(s_wm[w * 8 + tid] - ms);
+          s_sc[w * 8 + tid] = f;
+          l += s_wl[w * 8 + tid] * f;
+        }
+        s_cm[tid] = mc;
+        s_cl[tid] = l;
+      }
+      // Who else works on this slab?  Chunk g0 is its first one.
+      const long long g0 = g_begin + it - c.chunk;
+      const int p_first = (int)(g0 / per_cta), p_last = (int)((g0 + c.cb - 1) / per_cta);
+      const bool exclusive = p_first == p_last;
+      if (p_first < 0 || p_last >= (int)gridDim.x || (int)blockIdx.x < p_first || (int)blockIdx.x > p_last) {
+        if (tid == 0) {
+          atomicOr(p.err, kErrStreamBounds);
+          p.dbg[16] = p_first; p.dbg[17] = p_last; p.dbg[18] = (int)blockIdx.x; p.dbg[19] = (int)g0;
+          *s_abort = 1;
+        }
+        break;
+      }
+      const int my_slot = (g0 <= g_begin) ? 0 : 1;  // 0: the slab is the first of this CTA's piece
+      float* my_part = p.part + ((size_t)blockIdx.x * 2 + my_slot) * kStPartStride;
+      __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + unit * (size_t)G * d;
+
+      for (int rd = 0; rd * 4 < G; ++rd) {
+        if ((tig >> 1) == rd) {
+          float* c0 = s_comb + ((size_t)warp * 4 + 2 * (tig & 1)) * d;
+#pragma unroll
+          for (int mb = 0; mb < 8; ++mb) {
+            c0[16 * mb + gid] = o[mb][0];
+            c0[d + 16 * mb + gid] = o[mb][1];
+            c0[16 * mb + 8 + gid] = o[mb][2];
+            c0[d + 16 * mb + 8 + gid] = o[mb][3];
+          }
+        }
+        consumer_sync();  // also orders s_sc / s_cm / s_cl
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int e = tid + kStConsumers * i;  // [4 heads][128]
+          const int g = 4 * rd + (e >> 7);
+          if (g < G) {
+            float acc = 0.f;
+#pragma unroll
+            for (int w = 0; w < kStConsumerWarps; ++w) acc += s_comb[(size_t)w * 4 * d + e] * s_sc[w * 8 + g];
+            if (exclusive) out[(size_t)g * d + (e & 127)] = __float2bfloat16_rn(acc / s_cl[g]);
+            else my_part[(size_t)g * d + (e & 127)] = acc;
+          }
+        }
+        consumer_sync();
+      }
+
+      bool finish = exclusive;
+      if (exclusive) {
+        if (tid < 8) {
+          s_finM[tid] = s_cm[tid];
+          s_finf[tid] = 1.0f / s_cl[tid];
+        }
+      } else {
+        if (tid < 8) {
+          my_part[8 * d + tid] = s_cm[tid];
+          my_part[8 * d + 8 + tid] = s_cl[tid];
+        }
+        __threadfence();  // partial and logits before the ticket
+        consumer_sync();
+        if (tid == 0) {
+          const int k = p_last - p_first + 1;
+          const int t = atomicAdd(p.arrive + slab, 1);
+          const int last = t == k - 1;
+          if (last) {
+            p.arrive[slab] = 0;
+            __threadfence();
+          }
+          s_flags[1] = last;
+        }
+        consumer_sync();
+        finish = s_flags[1] != 0;
+        if (finish) {
+          // Last arriver: combine the partials of CTAs p_first..p_last.
+          if (tid < G) {
+            float M = -CUDART_INF_F;
+            for (int q = p_first; q <= p_last; ++q) {
+              const int slot = (g0 <= per_cta * q) ? 0 : 1;
+              M = fmaxf(M, __ldcg(p.part + ((size_t)q * 2 + slot) * kStPartStride + 8 * d + tid));
+            }
+            float L = 0.f;
+            for (int q = p_first; q <= p_last; ++q) {
+              const int slot = (g0 <= per_cta * q) ? 0 : 1;
+              const float* pp = p.part + ((size_t)q * 2 + slot) * kStPartStride + 8 * d;
+              L += __ldcg(pp + 8 + tid) * fast_exp2(__ldcg(pp + tid) - M);
+            }
+            s_finM[tid] = M;
+            s_finf[tid] = 1.0f / L;
+          }
+          consumer_sync();
+          for (int e = tid; e < G * d; e += kStConsumers) {
+            const int g = e >> 7;
+            const float M = s_finM[g];
+            float acc = 0.f;
+            for (int q = p_first; q <= p_last; ++q) {
+              const int slot = (g0 <= per_cta * q) ? 0 : 1;
+              const float* pp = p.part + ((size_t)q * 2 + slot) * kStPartStride;
+              acc += __ldcg(pp + e) * fast_exp2(__ldcg(pp + 8 * d + g) - M);
+            }
+            out[e] = __float2bfloat16_rn(acc * s_finf[g]);
+          }
+        }
+      }
+      if (finish) {
+        // a5: final weights of every row of the slab, summed over the group's heads (Eq. 6)
+        consumer_sync();  // s_finM / s_finf, and this CTA's own logits
+        float M[kMaxGroup], f[kMaxGroup];
+#pragma unroll
+        for (int g = 0; g < kMaxGroup; ++g) {
+          M[g] = g < G ? s_finM[g] : 0.f;
+          f[g] = g < G ? s_finf[g] : 0.f;
+        }
+        float* score = p.score + slab * (size_t)p.cap;
+        float* dout = p.delta_out ? p.delta_out + slab * (size_t)p.cap : nullptr;
+        for (int j0 = tid; j0 < n; j0 += 4 * kStConsumers) {
+          float sc[4], dl[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int j = j0 + i * kStConsumers;
+            sc[i] = (j < n && j != n_old) ? score[j] : 0.f;
+            dl[i] = 0.f;
+          }
+#pragma unroll
+          for (int g = 0; g < kMaxGroup; ++g) {
+            if (g < G) {
+              float e[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const int j = j0 + i * kStConsumers;
+                e[i] = j < n ? __ldcg(lg + (size_t)g * p.cap + j) : -CUDART_INF_F;
+              }
+#pragma unroll
+              for (int i = 0; i < 4; ++i) dl[i] += fast_exp2(e[i] - M[g]) * f[g];
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int j = j0 + i * kStConsumers;
+            if (j < n) {
+              score[j] = sc[i] + dl[i];
+              if (dout) dout[j] = dl[i];
+            }
+          }
+        }
+      }
+      consumer_sync();  // shared scratch is reused by the next segment
+      it += seg;
+      if (it < cnt) cursor_next_slab(c, s_cnt, Nb, Hkv);
+    }
+  }
+
+  // Every tile load this CTA issued has been waited for by its consumers unless a wait gave up;
+  // then give the loads in flight a bounded time to land before the shared memory is released.
+  __syncthreads();
+  if (*s_abort && tid == 0) {
+    for (int s = 0; s < kStStages; ++s) {
+      const int armed = s_flags[2 + s];
+      if (armed == 0) continue;
+      for (uint32_t i = 0; i < kStSpinLimit; ++i)
+        if (mbar_try_wait(bar_full + 8 * s, (uint32_t)(armed - 1))) break;
+    }
+  }
+  finish_ticket(p);
+}
+
+}  // namespace dynts

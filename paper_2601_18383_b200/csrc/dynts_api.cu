@@ -17,6 +17,7 @@
 
 #include "common.cuh"
 #include "decode_attn.cuh"
+#include "decode_stream.cuh"
 #include "evict.cuh"
 
 namespace {
@@ -40,8 +41,13 @@ dynts_status_t fail(dynts_status_t st, const char* fmt, ...) {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  size_t K, V, pos, score, src, hdr, len, tot, pinned, target, active, ticket, total;
+  size_t K, V, pos, score, src, hdr, len, tot, pinned, target, active, ticket, logit, part, arrive, total;
 };
+
+// The streaming decode kernel covers bf16 slabs with head_dim 128.
+bool stream_capable(const dynts_config_t* c) {
+  return c->dtype == DYNTS_BF16 && c->head_dim == 128 && c->batch <= dynts::kStMaxBatch;
+}
 
 int elt_bytes_of(int dtype) { return dtype == DYNTS_FP32 ? 4 : 2; }
 
@@ -87,6 +93,12 @@ Layout make_layout(const dynts_config_t* c, int cap) {
   L.target = take((size_t)c->batch * 4);
   L.active = take((size_t)c->batch * 4);
   L.ticket = take(256);
+  L.logit = L.part = L.arrive = off;
+  if (stream_capable(c)) {
+    L.logit = take(slabs * (size_t)(c->q_heads / c->kv_heads) * cap * 4);
+    L.part = take((size_t)dynts::kStMaxCtas * 2 * dynts::kStPartStride * 4);
+    L.arrive = take(slabs * 4);
+  }
   L.total = off;
   return L;
 }
@@ -113,6 +125,10 @@ struct dynts_cache {
   char* stage_dev = nullptr;
   size_t stage_bytes = 0;
   bool attr_generic_f32 = false, attr_generic_bf16 = false, attr_mma = false, attr_select = false;
+  bool attr_stream = false;
+  bool have_maps = false;    // tensor maps of the K and V slabs for the streaming kernel
+  CUtensorMap map_K, map_V;
+  int sm_count = 0;
 
   void* K() const { return base + lay.K; }
   void* V() const { return base + lay.V; }
@@ -126,12 +142,48 @@ struct dynts_cache {
   int* target() const { return reinterpret_cast<int*>(base + lay.target); }
   int* active() const { return reinterpret_cast<int*>(base + lay.active); }
   unsigned int* ticket() const { return reinterpret_cast<unsigned int*>(base + lay.ticket); }
+  float* logit() const { return reinterpret_cast<float*>(base + lay.logit); }
+  float* part() const { return reinterpret_cast<float*>(base + lay.part); }
+  int* arrive() const { return reinterpret_cast<int*>(base + lay.arrive); }
   size_t slabs() const { return (size_t)cfg.layers * cfg.batch * cfg.kv_heads; }
 };
 
 namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Tensor maps (TMA descriptors) over all K rows and all V rows: a [slabs * cap][128] bf16 matrix
+// read in boxes of 32 rows x 64 columns with the 128-byte shared-memory swizzle.
+typedef CUresult (*tensor_map_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                         const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                         CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+dynts_status_t make_slab_maps(dynts_cache* c) {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+  if (!fn || qres != cudaDriverEntryPointSuccess) return fail(DYNTS_ERR_CUDA, "the driver has no cuTensorMapEncodeTiled");
+  tensor_map_encode_fn encode = reinterpret_cast<tensor_map_encode_fn>(fn);
+  const cuuint64_t rows = (cuuint64_t)c->slabs() * c->cap;
+  if (rows >= ((cuuint64_t)1 << 31)) return DYNTS_OK;  // row coordinates are 32-bit: keep the cluster kernels
+  const cuuint64_t dims[2] = {128, rows};
+  const cuuint64_t strides[1] = {256};
+  const cuuint32_t box[2] = {64, (cuuint32_t)dynts::kStRows};
+  const cuuint32_t estr[2] = {1, 1};
+  CUresult r1 = encode(&c->map_K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c->K(), dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r2 = encode(&c->map_V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c->V(), dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r1 != CUDA_SUCCESS || r2 != CUDA_SUCCESS)
+    return fail(DYNTS_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d, %d)", (int)r1, (int)r2);
+  int dev = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  CUDA_TRY(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev));
+  c->have_maps = true;
+  return DYNTS_OK;
+}
 
 dynts_status_t materialise(dynts_cache* c) {
   if (c->ready) return DYNTS_OK;
@@ -162,6 +214,11 @@ dynts_status_t materialise(dynts_cache* c) {
     CUDA_TRY(cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->err_dev), c->err_host, 0));
   }
   CUDA_TRY(cudaMemsetAsync(c->base, 0, c->lay.total, c->stream));
+  c->have_maps = false;
+  if (stream_capable(&c->cfg)) {
+    dynts_status_t ms = make_slab_maps(c);
+    if (ms != DYNTS_OK) return ms;
+  }
   const int Nb = c->cfg.batch;
   c->seq_budget.assign(Nb, c->cfg.budget);
   if (c->cfg.seq_budgets)
@@ -193,7 +250,7 @@ int pick_cluster(const dynts_cache* c, int units, int n_max) {
   if (c->cluster > 0) return c->cluster;
   // Enough CTAs to fill 148 SMs several times over, but at least ~64 rows per CTA.
   int s = 1;
-  while (s < 8 && (long long)units * s < 148 * 12 && n_max / (2 * s) >= 64) s *= 2;
+  while (s < 8 && (long long)units * s < 148 * 6 && n_max / (2 * s) >= 64) s *= 2;
   return s;
 }
 
@@ -232,6 +289,10 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
   p.active = c->active();
   p.ticket = c->ticket();
   p.err = c->err_dev;
+  p.logit = c->logit();
+  p.part = c->part();
+  p.arrive = c->arrive();
+  p.dbg = reinterpret_cast<int*>(c->ticket()) + 8;  // spare words of the ticket block
   p.layer0 = layer0;
   p.n_layers = n_layers;
   p.Nb = Nb;
@@ -244,9 +305,31 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
   p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)f.head_dim));
 
   const bool mma_ok = f.dtype == DYNTS_BF16 && f.head_dim == 128 && c->G <= 8;
+  const bool stream_ok = mma_ok && c->have_maps;
   int variant = c->variant;
-  if (variant == 0) variant = mma_ok ? 2 : 1;
+  if (variant == 0) variant = stream_ok ? 3 : (mma_ok ? 2 : 1);
   if (variant == 2 && !mma_ok) return fail(DYNTS_ERR_INVALID_ARG, "tensor-core variant needs bf16, head_dim 128, G <= 8");
+  if (variant == 3 && !stream_ok)
+    return fail(DYNTS_ERR_INVALID_ARG, "streaming variant needs bf16, head_dim 128, G <= 8, batch <= %d", dynts::kStMaxBatch);
+
+  if (variant == 3) {
+    const size_t smem = dynts::stream_smem_bytes(Nb);
+    if (!c->attr_stream) {
+      CUDA_TRY(cudaFuncSetAttribute(dynts::decode_attn_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)dynts::stream_smem_bytes(dynts::kStMaxBatch)));
+      c->attr_stream = true;
+    }
+    int ctas = ((c->cluster == 1 || c->cluster == 2) ? c->cluster : 2) * c->sm_count;
+    ctas = std::max(1, std::min(ctas, dynts::kStMaxCtas));
+    dynts::decode_attn_stream_kernel<<<ctas, dynts::kStThreads, smem, c->stream>>>(p, c->map_K, c->map_V);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(DYNTS_ERR_CUDA, "decode launch (streaming, %d CTAs): %s", ctas, cudaGetErrorString(e));
+    c->launches += 1;
+    if (advance)
+      for (int b = 0; b < Nb; ++b)
+        if (c->active_h[b]) c->len_h[b] += 1;
+    return DYNTS_OK;
+  }
 
   cudaLaunchConfig_t lc;
   memset(&lc, 0, sizeof(lc));
@@ -651,8 +734,17 @@ dynts_status_t dynts_cache_import(dynts_cache_t* c, int layer, int seq, int head
 
 dynts_status_t dynts_poll_error(dynts_cache_t* c) {
   if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
-  if (c->err_host && *reinterpret_cast<volatile int*>(c->err_host) != 0)
-    return fail(DYNTS_ERR_DEVICE, "device status word 0x%x", *reinterpret_cast<volatile int*>(c->err_host));
+  if (c->err_host && *reinterpret_cast<volatile int*>(c->err_host) != 0) {
+    const int word = *reinterpret_cast<volatile int*>(c->err_host);
+    int dbg[24] = {0};
+    if (c->ready && (word & dynts::kErrStreamBounds))
+      cudaMemcpy(dbg, reinterpret_cast<int*>(c->ticket()) + 8, sizeof(dbg), cudaMemcpyDeviceToHost);
+    return fail(DYNTS_ERR_DEVICE,
+                "device status word 0x%x (producer: layer %d seq %d head %d chunk %d len %d item %d cta %d smem 0x%x; "
+                "consumer: layer %d seq %d head %d chunk %d n %d item %d cta %d seg %d; sharers %d..%d cta %d first chunk %d)",
+                word, dbg[0], dbg[1], dbg[2], dbg[3], dbg[4], dbg[5], dbg[6], dbg[7], dbg[8], dbg[9], dbg[10], dbg[11],
+                dbg[12], dbg[13], dbg[14], dbg[15], dbg[16], dbg[17], dbg[18], dbg[19]);
+  }
   return DYNTS_OK;
 }
 
@@ -666,7 +758,7 @@ dynts_status_t dynts_cache_set_launch(dynts_cache_t* c, int cluster, int variant
   if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
   if (!(cluster == 0 || cluster == 1 || cluster == 2 || cluster == 4 || cluster == 8 || cluster == 16))
     return fail(DYNTS_ERR_INVALID_ARG, "cluster size must be 0, 1, 2, 4, 8 or 16");
-  if (variant < 0 || variant > 2) return fail(DYNTS_ERR_INVALID_ARG, "variant must be 0, 1 or 2");
+  if (variant < 0 || variant > 3) return fail(DYNTS_ERR_INVALID_ARG, "variant must be 0, 1, 2 or 3");
   c->cluster = cluster;
   c->variant = variant;
   return DYNTS_OK;

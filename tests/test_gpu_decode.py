@@ -58,7 +58,7 @@ def test_fp32_generic_small(cluster):
     assert ed <= H.TOL_DELTA and es <= H.TOL_DELTA, (ed, es)
 
 
-@pytest.mark.parametrize("variant,cluster", [(1, 1), (1, 4), (2, 1), (2, 2), (2, 4), (2, 8), (0, 0)])
+@pytest.mark.parametrize("variant,cluster", [(1, 1), (1, 4), (2, 1), (2, 2), (2, 4), (2, 8), (3, 1), (3, 2), (0, 0)])
 def test_bf16_llama_shape_small(variant, cluster):
     """Llama-like group (G = 4, d = 128), several tiles and a ragged tail, both kernels."""
     cfg = W.get_config("c2_llama8b").scaled(layers=2, batch=2, prompt=37, budget=512, window=16, evict_interval=64)
@@ -67,7 +67,7 @@ def test_bf16_llama_shape_small(variant, cluster):
     assert ed <= H.TOL_DELTA and es <= H.TOL_DELTA, (ed, es)
 
 
-@pytest.mark.parametrize("variant,cluster", [(1, 2), (2, 1), (2, 8), (0, 0)])
+@pytest.mark.parametrize("variant,cluster", [(1, 2), (2, 1), (2, 8), (3, 2), (0, 0)])
 def test_bf16_qwen_shape_small(variant, cluster):
     """Qwen-like group (G = 7)."""
     cfg = W.get_config("c3_qwen7b").scaled(layers=1, batch=3, prompt=200, budget=512, window=16, evict_interval=64)
@@ -77,7 +77,7 @@ def test_bf16_qwen_shape_small(variant, cluster):
 
 
 @pytest.mark.parametrize("G", [1, 2, 3, 5, 8])
-@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("variant", [1, 2, 3])
 def test_group_sizes(G, variant):
     cfg = W.get_config("c2_llama8b").scaled(layers=1, batch=1, kv_heads=2, q_heads=2 * G, prompt=50, budget=256,
                                              window=8, evict_interval=32)
@@ -85,7 +85,7 @@ def test_group_sizes(G, variant):
     assert eo <= H.TOL_OUT["bf16"] and ed <= H.TOL_DELTA and es <= H.TOL_DELTA, (eo, ed, es)
 
 
-@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("variant", [1, 2, 3])
 def test_empty_cache_first_token_attends_to_itself(variant):
     """Degenerate case: no prompt.  Step 1 has a single row; alpha = 1, out = v_new, mass = G."""
     cfg = W.get_config("c2_llama8b").scaled(layers=1, batch=1, prompt=0, budget=64, window=4, evict_interval=16)
@@ -113,10 +113,30 @@ def test_head_dim_64_bf16_and_256_fp32_generic():
         assert eo <= H.TOL_OUT[dtype] and ed <= H.TOL_DELTA and es <= H.TOL_DELTA, (dtype, d, eo, ed, es)
 
 
-def test_unpinned_prompt_rows_and_partial_pin():
+@pytest.mark.parametrize("variant", [2, 3])
+def test_unpinned_prompt_rows_and_partial_pin(variant):
     cfg = W.get_config("c2_llama8b").scaled(layers=1, batch=1, prompt=40, budget=256, window=8, evict_interval=32)
-    eo, ed, es = _lockstep_steps(cfg, 10, seed=41, cluster=2, variant=2, prompt_rows=90, n_pinned=40)
+    eo, ed, es = _lockstep_steps(cfg, 10, seed=41, cluster=2, variant=variant, prompt_rows=90, n_pinned=40)
     assert eo <= H.TOL_OUT["bf16"] and ed <= H.TOL_DELTA and es <= H.TOL_DELTA
+
+
+@pytest.mark.parametrize("ctas_per_sm", [1, 2])
+def test_stream_kernel_many_slabs_per_cta(ctas_per_sm):
+    """Streaming kernel with far more slabs than CTAs: a CTA's piece of the chunk list holds
+    slabs it finishes alone and, at both ends, slabs it shares with its neighbours; the row
+    counts cross a 32-row chunk boundary during the run."""
+    cfg = W.get_config("c2_llama8b").scaled(layers=24, batch=5, prompt=57, budget=256, window=8, evict_interval=32)
+    eo, ed, es = _lockstep_steps(cfg, 9, seed=51, cluster=ctas_per_sm, variant=3)
+    assert eo <= H.TOL_OUT["bf16"] and ed <= H.TOL_DELTA and es <= H.TOL_DELTA, (eo, ed, es)
+
+
+def test_stream_kernel_one_slab_many_ctas():
+    """One KV head, one layer, a long slab: every chunk goes to a different CTA and the last
+    arriver combines dozens of partials."""
+    cfg = W.get_config("c3_qwen7b").scaled(layers=1, batch=1, kv_heads=1, q_heads=7, prompt=1500, budget=2048,
+                                            window=16, evict_interval=64)
+    eo, ed, es = _lockstep_steps(cfg, 5, seed=52, cluster=2, variant=3)
+    assert eo <= H.TOL_OUT["bf16"] and ed <= H.TOL_DELTA and es <= H.TOL_DELTA, (eo, ed, es)
 
 
 def test_layer_by_layer_matches_all_layers():
