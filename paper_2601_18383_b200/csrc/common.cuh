@@ -37,6 +37,7 @@ struct DecodeParams {
   int layer0, n_layers, Nb, Hkv, G, d, cap;
   int advance;        // 1: the last CTA to finish increments len/tot of active sequences
   int tile_tokens;    // rows of logits a CTA can hold in shared memory
+  int slabs_per_cta;  // streaming kernel: > 0 => every CTA takes this many whole slabs
   float scale_log2;   // log2(e) / sqrt(d)
 };
 

@@ -87,10 +87,19 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
   *abort_flag = 1;
   atomicOr(err, kErrTimeout);
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+// K and V rows are read once per step: their L2 lines are marked evict-first so that the stream
+// does not push the scores and the logit scratch (which are re-read soon) out of L2.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar,
+                                            uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
@@ -144,6 +153,132 @@ __device__ __forceinline__ void cursor_next_slab(StCursor& c, const int* s_cnt, 
   c.cb = s_cnt[c.b];
 }
 
+
+// a5 for one slab: score[j] += sum over the group's heads of exp2(logit[g][j] - M[g]) / L[g], the
+// appended row n_old starting from zero.  GG is the group size at compile time so that every load
+// of a pass is issued before the first use (one memory round trip per pass).
+template <int GG, int VB>
+__device__ __forceinline__ void score_pass_vec(float* __restrict__ score, float* __restrict__ dout,
+                                               const float* __restrict__ lg, int cap, int n, int n_old,
+                                               const float* s_finM, const float* s_finf, int tid) {
+  float M[GG], f[GG];
+#pragma unroll
+  for (int g = 0; g < GG; ++g) {
+    M[g] = s_finM[g];
+    f[g] = s_finf[g];
+  }
+  for (int v0 = tid; 4 * v0 < n; v0 += VB * kStConsumers) {
+    float4 sc[VB], e[VB][GG];
+#pragma unroll
+    for (int i = 0; i < VB; ++i) {
+      const int j = min(4 * (v0 + i * kStConsumers), cap - 4);  // clamped: always a valid address
+      sc[i] = *reinterpret_cast<const float4*>(score + j);
+#pragma unroll
+      for (int g = 0; g < GG; ++g) e[i][g] = __ldcg(reinterpret_cast<const float4*>(lg + (size_t)g * cap + j));
+    }
+#pragma unroll
+    for (int i = 0; i < VB; ++i) {
+      const int j = 4 * (v0 + i * kStConsumers);
+      if (j >= n) continue;
+      float4 dl = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int g = 0; g < GG; ++g) {
+        dl.x += fast_exp2(e[i][g].x - M[g]) * f[g];
+        dl.y += fast_exp2(e[i][g].y - M[g]) * f[g];
+        dl.z += fast_exp2(e[i][g].z - M[g]) * f[g];
+        dl.w += fast_exp2(e[i][g].w - M[g]) * f[g];
+      }
+      const int z = n_old - j;  // the appended row starts from zero
+      if (z == 0) sc[i].x = 0.f;
+      if (z == 1) sc[i].y = 0.f;
+      if (z == 2) sc[i].z = 0.f;
+      if (z == 3) sc[i].w = 0.f;
+      const float4 r = make_float4(sc[i].x + dl.x, sc[i].y + dl.y, sc[i].z + dl.z, sc[i].w + dl.w);
+      if (j + 4 <= n) {
+        *reinterpret_cast<float4*>(score + j) = r;
+        if (dout) *reinterpret_cast<float4*>(dout + j) = dl;
+      } else {  // rows past the end are left alone
+        score[j] = r.x;
+        if (j + 1 < n) score[j + 1] = r.y;
+        if (j + 2 < n) score[j + 2] = r.z;
+        if (dout) {
+          dout[j] = dl.x;
+          if (j + 1 < n) dout[j + 1] = dl.y;
+          if (j + 2 < n) dout[j + 2] = dl.z;
+        }
+      }
+    }
+  }
+}
+
+template <int GG>
+__device__ __forceinline__ void score_pass(float* score, float* dout, const float* lg, int cap, int n, int n_old,
+                                           const float* s_finM, const float* s_finf, int tid) {
+  if ((cap & 3) == 0 && cap >= 4) {
+    score_pass_vec<GG, (GG <= 4 ? 4 : 2)>(score, dout, lg, cap, n, n_old, s_finM, s_finf, tid);
+  } else {
+    for (int j = tid; j < n; j += kStConsumers) {
+      float dl = 0.f;
+#pragma unroll
+      for (int g = 0; g < GG; ++g) dl += fast_exp2(__ldcg(lg + (size_t)g * cap + j) - s_finM[g]) * s_finf[g];
+      score[j] = (j == n_old ? 0.f : score[j]) + dl;
+      if (dout) dout[j] = dl;
+    }
+  }
+}
+
+// The slab's last arriver combines the partials of the k <= 4 CTAs that worked on it; thread tid
+// produces output column tid of every head.  pp[i] = partial of contributor i (clamped copies
+// beyond k).  All loads are issued before the first use.
+template <int GG>
+__device__ __forceinline__ void combine_partials(const float* const (&pp)[4], int k, __nv_bfloat16* out,
+                                                 float* s_finM, float* s_finf, int tid) {
+  constexpr int d = 128;
+  float pm[4][GG], pl[4][GG], po[4][GG];
+#pragma unroll
+  for (int qi = 0; qi < 4; ++qi) {
+#pragma unroll
+    for (int g = 0; g < GG; ++g) {
+      pm[qi][g] = __ldcg(pp[qi] + 8 * d + g);
+      pl[qi][g] = __ldcg(pp[qi] + 8 * d + 8 + g);
+      po[qi][g] = __ldcg(pp[qi] + (size_t)g * d + tid);
+    }
+  }
+#pragma unroll
+  for (int g = 0; g < GG; ++g) {
+    float M = -CUDART_INF_F;
+#pragma unroll
+    for (int qi = 0; qi < 4; ++qi)
+      if (qi < k) M = fmaxf(M, pm[qi][g]);
+    float L = 0.f, acc = 0.f;
+#pragma unroll
+    for (int qi = 0; qi < 4; ++qi) {
+      if (qi < k) {
+        const float w = fast_exp2(pm[qi][g] - M);
+        L += pl[qi][g] * w;
+        acc += po[qi][g] * w;
+      }
+    }
+    out[(size_t)g * d + tid] = __float2bfloat16_rn(acc / L);
+    if (tid == 0) {
+      s_finM[g] = M;
+      s_finf[g] = 1.0f / L;
+    }
+  }
+}
+
+#define DYNTS_DISPATCH_GROUP(G, CALL) \
+  switch (G) {                        \
+    case 1: { constexpr int GG = 1; CALL; } break; \
+    case 2: { constexpr int GG = 2; CALL; } break; \
+    case 3: { constexpr int GG = 3; CALL; } break; \
+    case 4: { constexpr int GG = 4; CALL; } break; \
+    case 5: { constexpr int GG = 5; CALL; } break; \
+    case 6: { constexpr int GG = 6; CALL; } break; \
+    case 7: { constexpr int GG = 7; CALL; } break; \
+    default: { constexpr int GG = 8; CALL; } break; \
+  }
+
 __global__ void __launch_bounds__(kStThreads, 2)
 decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmK,
                           const __grid_constant__ CUtensorMap tmV) {
@@ -176,16 +311,20 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, 2);  // the two warps that consume the stage
     }
-    for (int i = 0; i < 16; ++i) s_flags[i] = 0;
+    for (int i = 0; i < 8; ++i) s_flags[i] = 0;  // (s_flags[8] belongs to the prefix warp below)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    int carry = 0;
+    int carry = 0, cmin = 0x7fffffff, cmax = 0;
     for (int b0 = 0; b0 < Nb; b0 += 32) {
       const int b = b0 + lane;
       int c = 0;
       if (b < Nb && p.active[b]) c = (p.len[b] + 1 + kStRows - 1) / kStRows;
+      if (c > 0) {
+        cmin = min(cmin, c);
+        cmax = max(cmax, c);
+      }
       int incl = c;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -198,13 +337,24 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
       }
       carry += __shfl_sync(0xffffffffu, incl, 31);
     }
-    if (lane == 0) s_off[Nb] = carry * Hkv;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      cmin = min(cmin, __shfl_xor_sync(0xffffffffu, cmin, o));
+      cmax = max(cmax, __shfl_xor_sync(0xffffffffu, cmax, o));
+    }
+    if (lane == 0) {
+      s_off[Nb] = carry * Hkv;
+      s_flags[8] = (cmin == cmax) ? cmax : 0;  // chunks per slab if all slabs are equally long
+    }
   }
   __syncthreads();
 
   const long long per_layer = s_off[Nb];
   const long long total = per_layer * p.n_layers;
-  const long long per_cta = (total + gridDim.x - 1) / gridDim.x;
+  // Piece length: whole slabs per CTA where the host asked for it and the slabs are equally long
+  // (no slab is then shared between CTAs), else an equal share of the chunk list.
+  const long long per_cta = (p.slabs_per_cta > 0 && s_flags[8] > 0) ? (long long)p.slabs_per_cta * s_flags[8]
+                                                                   : (total + gridDim.x - 1) / gridDim.x;
   const long long g_begin = per_cta * blockIdx.x;
   long long g_end = g_begin + per_cta;
   if (g_end > total) g_end = total;
@@ -215,6 +365,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
     if (lane == 0) {
       StCursor c;
       cursor_seek(c, g_begin, s_off, s_cnt, Nb);
+      const uint64_t pol = l2_evict_first_policy();
       for (int it = 0; it < cnt; ++it) {
         const int stage = it % kStStages;
         const uint32_t ph = (uint32_t)(it / kStStages) & 1u;
@@ -236,10 +387,10 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         mbar_arrive_expect_tx(full, kStStageBytes);
         s_flags[2 + stage] = 1 + (int)ph;  // phase of the loads now in flight, for the drain below
         const int row = (int)(slab * (size_t)p.cap) + c.chunk * kStRows;
-        tma_load_2d(dst, &tmK, 0, row, full);
-        tma_load_2d(dst + kStBoxBytes, &tmK, 64, row, full);
-        tma_load_2d(dst + 2 * kStBoxBytes, &tmV, 0, row, full);
-        tma_load_2d(dst + 3 * kStBoxBytes, &tmV, 64, row, full);
+        tma_load_2d(dst, &tmK, 0, row, full, pol);
+        tma_load_2d(dst + kStBoxBytes, &tmK, 64, row, full, pol);
+        tma_load_2d(dst + 2 * kStBoxBytes, &tmV, 0, row, full, pol);
+        tma_load_2d(dst + 3 * kStBoxBytes, &tmV, 64, row, full, pol);
         if (++c.chunk == c.cb) cursor_next_slab(c, s_cnt, Nb, Hkv);
       }
     }
@@ -343,11 +494,16 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           x[2] = (gid < G && tk + 8 < n) ? s1[0] * p.scale_log2 : -CUDART_INF_F;
           x[3] = (gid < G && tk + 9 < n) ? s1[1] * p.scale_log2 : -CUDART_INF_F;
           if (gid < G) {
-            float* t = lg + (size_t)gid * p.cap + tk;
-            if (tk < n) t[0] = x[0];
-            if (tk + 1 < n) t[1] = x[1];
-            if (tk + 8 < n) t[8] = x[2];
-            if (tk + 9 < n) t[9] = x[3];
+            float* t = lg + (size_t)gid * p.cap + tk;  // tk is even: 8-byte stores when the row base allows
+            if ((p.cap & 1) == 0 && tk + 9 < n) {
+              *reinterpret_cast<float2*>(t) = make_float2(x[0], x[1]);
+              *reinterpret_cast<float2*>(t + 8) = make_float2(x[2], x[3]);
+            } else {
+              if (tk < n) t[0] = x[0];
+              if (tk + 1 < n) t[1] = x[1];
+              if (tk + 8 < n) t[8] = x[2];
+              if (tk + 9 < n) t[9] = x[3];
+            }
           }
           float um = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
           um = fmaxf(um, __shfl_xor_sync(0xffffffffu, um, 1));
@@ -384,22 +540,6 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         s_wm[warp * 8 + gid] = m_run;
         s_wl[warp * 8 + gid] = l_part;
       }
-      consumer_sync();
-      if (tid < 8) {
-        float mc = -CUDART_INF_F;
-#pragma unroll
-        for (int w = 0; w < kStConsumerWarps; ++w) mc = fmaxf(mc, s_wm[w * 8 + tid]);
-        const float ms = (mc == -CUDART_INF_F) ? 0.f : mc;
-        float l = 0.f;
-#pragma unroll
-        for (int w = 0; w < kStConsumerWarps; ++w) {
-          const float f = fast_exp2(s_wm[w * 8 + tid] - ms);
-          s_sc[w * 8 + tid] = f;
-          l += s_wl[w * 8 + tid] * f;
-        }
-        s_cm[tid] = mc;
-        s_cl[tid] = l;
-      }
       // Who else works on this slab?  Chunk g0 is its first one.
       const long long g0 = g_begin + it - c.chunk;
       const int p_first = (int)(g0 / per_cta), p_last = (int)((g0 + c.cb - 1) / per_cta);
@@ -415,8 +555,10 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
       const int my_slot = (g0 <= g_begin) ? 0 : 1;  // 0: the slab is the first of this CTA's piece
       float* my_part = p.part + ((size_t)blockIdx.x * 2 + my_slot) * kStPartStride;
       __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + unit * (size_t)G * d;
-
+      float* score = p.score + slab * (size_t)p.cap;
+      // Thread tid owns output column tid of the four heads of a round.
       for (int rd = 0; rd * 4 < G; ++rd) {
+        if (rd > 0) consumer_sync();  // the previous round's sums have been read
         if ((tig >> 1) == rd) {
           float* c0 = s_comb + ((size_t)warp * 4 + 2 * (tig & 1)) * d;
 #pragma unroll
@@ -427,33 +569,41 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
             c0[d + 16 * mb + 8 + gid] = o[mb][3];
           }
         }
-        consumer_sync();  // also orders s_sc / s_cm / s_cl
+        consumer_sync();  // also orders s_wm / s_wl
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const int e = tid + kStConsumers * i;  // [4 heads][128]
-          const int g = 4 * rd + (e >> 7);
+          const int g = 4 * rd + i;
           if (g < G) {
-            float acc = 0.f;
+            float mc = -CUDART_INF_F;
 #pragma unroll
-            for (int w = 0; w < kStConsumerWarps; ++w) acc += s_comb[(size_t)w * 4 * d + e] * s_sc[w * 8 + g];
-            if (exclusive) out[(size_t)g * d + (e & 127)] = __float2bfloat16_rn(acc / s_cl[g]);
-            else my_part[(size_t)g * d + (e & 127)] = acc;
+            for (int w = 0; w < kStConsumerWarps; ++w) mc = fmaxf(mc, s_wm[w * 8 + g]);
+            const float ms = (mc == -CUDART_INF_F) ? 0.f : mc;
+            float acc = 0.f, l = 0.f;
+#pragma unroll
+            for (int w = 0; w < kStConsumerWarps; ++w) {
+              const float f = fast_exp2(s_wm[w * 8 + g] - ms);
+              acc += s_comb[((size_t)w * 4 + i) * d + tid] * f;
+              l += s_wl[w * 8 + g] * f;
+            }
+            if (exclusive) {
+              out[(size_t)g * d + tid] = __float2bfloat16_rn(acc / l);
+              if (tid == 0) {
+                s_finM[g] = mc;
+                s_finf[g] = 1.0f / l;
+              }
+            } else {
+              my_part[(size_t)g * d + tid] = acc;
+              if (tid == 0) {
+                my_part[8 * d + g] = mc;
+                my_part[8 * d + 8 + g] = l;
+              }
+            }
           }
         }
-        consumer_sync();
       }
 
       bool finish = exclusive;
-      if (exclusive) {
-        if (tid < 8) {
-          s_finM[tid] = s_cm[tid];
-          s_finf[tid] = 1.0f / s_cl[tid];
-        }
-      } else {
-        if (tid < 8) {
-          my_part[8 * d + tid] = s_cm[tid];
-          my_part[8 * d + 8 + tid] = s_cl[tid];
-        }
+      if (!exclusive) {
         __threadfence();  // partial and logits before the ticket
         consumer_sync();
         if (tid == 0) {
@@ -469,77 +619,49 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         consumer_sync();
         finish = s_flags[1] != 0;
         if (finish) {
-          // Last arriver: combine the partials of CTAs p_first..p_last.
-          if (tid < G) {
-            float M = -CUDART_INF_F;
-            for (int q = p_first; q <= p_last; ++q) {
+          // Last arriver: combine the partials of CTAs p_first..p_last; thread tid does column tid.
+          const int k = p_last - p_first + 1;
+          if (k <= 4) {
+            const float* pp[4];
+#pragma unroll
+            for (int qi = 0; qi < 4; ++qi) {
+              const int q = min(p_first + qi, p_last);
               const int slot = (g0 <= per_cta * q) ? 0 : 1;
-              M = fmaxf(M, __ldcg(p.part + ((size_t)q * 2 + slot) * kStPartStride + 8 * d + tid));
+              pp[qi] = p.part + ((size_t)q * 2 + slot) * kStPartStride;
             }
-            float L = 0.f;
-            for (int q = p_first; q <= p_last; ++q) {
-              const int slot = (g0 <= per_cta * q) ? 0 : 1;
-              const float* pp = p.part + ((size_t)q * 2 + slot) * kStPartStride + 8 * d;
-              L += __ldcg(pp + 8 + tid) * fast_exp2(__ldcg(pp + tid) - M);
+            DYNTS_DISPATCH_GROUP(G, combine_partials<GG>(pp, k, out, s_finM, s_finf, tid));
+          } else {
+#pragma unroll
+            for (int g = 0; g < kMaxGroup; ++g) {
+              if (g < G) {
+                float M = -CUDART_INF_F;
+                for (int q = p_first; q <= p_last; ++q) {
+                  const int slot = (g0 <= per_cta * q) ? 0 : 1;
+                  M = fmaxf(M, __ldcg(p.part + ((size_t)q * 2 + slot) * kStPartStride + 8 * d + g));
+                }
+                float L = 0.f, acc = 0.f;
+                for (int q = p_first; q <= p_last; ++q) {
+                  const int slot = (g0 <= per_cta * q) ? 0 : 1;
+                  const float* pq = p.part + ((size_t)q * 2 + slot) * kStPartStride;
+                  const float f = fast_exp2(__ldcg(pq + 8 * d + g) - M);
+                  L += __ldcg(pq + 8 * d + 8 + g) * f;
+                  acc += __ldcg(pq + (size_t)g * d + tid) * f;
+                }
+                out[(size_t)g * d + tid] = __float2bfloat16_rn(acc / L);
+                if (tid == 0) {
+                  s_finM[g] = M;
+                  s_finf[g] = 1.0f / L;
+                }
+              }
             }
-            s_finM[tid] = M;
-            s_finf[tid] = 1.0f / L;
-          }
-          consumer_sync();
-          for (int e = tid; e < G * d; e += kStConsumers) {
-            const int g = e >> 7;
-            const float M = s_finM[g];
-            float acc = 0.f;
-            for (int q = p_first; q <= p_last; ++q) {
-              const int slot = (g0 <= per_cta * q) ? 0 : 1;
-              const float* pp = p.part + ((size_t)q * 2 + slot) * kStPartStride;
-              acc += __ldcg(pp + e) * fast_exp2(__ldcg(pp + 8 * d + g) - M);
-            }
-            out[e] = __float2bfloat16_rn(acc * s_finf[g]);
           }
         }
       }
       if (finish) {
         // a5: final weights of every row of the slab, summed over the group's heads (Eq. 6)
         consumer_sync();  // s_finM / s_finf, and this CTA's own logits
-        float M[kMaxGroup], f[kMaxGroup];
-#pragma unroll
-        for (int g = 0; g < kMaxGroup; ++g) {
-          M[g] = g < G ? s_finM[g] : 0.f;
-          f[g] = g < G ? s_finf[g] : 0.f;
-        }
-        float* score = p.score + slab * (size_t)p.cap;
         float* dout = p.delta_out ? p.delta_out + slab * (size_t)p.cap : nullptr;
-        for (int j0 = tid; j0 < n; j0 += 4 * kStConsumers) {
-          float sc[4], dl[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int j = j0 + i * kStConsumers;
-            sc[i] = (j < n && j != n_old) ? score[j] : 0.f;
-            dl[i] = 0.f;
-          }
-#pragma unroll
-          for (int g = 0; g < kMaxGroup; ++g) {
-            if (g < G) {
-              float e[4];
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const int j = j0 + i * kStConsumers;
-                e[i] = j < n ? __ldcg(lg + (size_t)g * p.cap + j) : -CUDART_INF_F;
-              }
-#pragma unroll
-              for (int i = 0; i < 4; ++i) dl[i] += fast_exp2(e[i] - M[g]) * f[g];
-            }
-          }
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int j = j0 + i * kStConsumers;
-            if (j < n) {
-              score[j] = sc[i] + dl[i];
-              if (dout) dout[j] = dl[i];
-            }
-          }
-        }
+        DYNTS_DISPATCH_GROUP(G, score_pass<GG>(score, dout, lg, p.cap, n, n_old, s_finM, s_finf, tid));
       }
       consumer_sync();  // shared scratch is reused by the next segment
       it += seg;

@@ -171,10 +171,10 @@ dynts_status_t make_slab_maps(dynts_cache* c) {
   const cuuint32_t box[2] = {64, (cuuint32_t)dynts::kStRows};
   const cuuint32_t estr[2] = {1, 1};
   CUresult r1 = encode(&c->map_K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c->K(), dims, strides, box, estr,
-                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   CUresult r2 = encode(&c->map_V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c->V(), dims, strides, box, estr,
-                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r1 != CUDA_SUCCESS || r2 != CUDA_SUCCESS)
     return fail(DYNTS_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d, %d)", (int)r1, (int)r2);
@@ -302,6 +302,7 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
   p.cap = c->cap;
   p.advance = advance ? 1 : 0;
   p.tile_tokens = tile_tokens;
+  p.slabs_per_cta = 0;
   p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)f.head_dim));
 
   const bool mma_ok = f.dtype == DYNTS_BF16 && f.head_dim == 128 && c->G <= 8;
@@ -321,6 +322,26 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
     }
     int ctas = ((c->cluster == 1 || c->cluster == 2) ? c->cluster : 2) * c->sm_count;
     ctas = std::max(1, std::min(ctas, dynts::kStMaxCtas));
+    // Equally long slabs and at least about as many slabs as CTAs: give every CTA whole slabs, so
+    // that no slab needs the cross-CTA combine.  Otherwise the chunk list is cut into equal pieces.
+    p.slabs_per_cta = 0;
+    {
+      bool uniform = true;
+      int n_active = 0, len0 = -1;
+      for (int b = 0; b < Nb; ++b) {
+        if (!c->active_h[b]) continue;
+        ++n_active;
+        if (len0 < 0) len0 = c->len_h[b];
+        uniform = uniform && c->len_h[b] == len0;
+      }
+      const long long slabs = (long long)n_layers * n_active * f.kv_heads;
+      const long long per = (slabs + ctas - 1) / ctas;
+      const long long used = (slabs + per - 1) / per;
+      if (uniform && used * 5 >= (long long)ctas * 4) {
+        p.slabs_per_cta = (int)per;
+        ctas = (int)used;
+      }
+    }
     dynts::decode_attn_stream_kernel<<<ctas, dynts::kStThreads, smem, c->stream>>>(p, c->map_K, c->map_V);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(DYNTS_ERR_CUDA, "decode launch (streaming, %d CTAs): %s", ctas, cudaGetErrorString(e));
