@@ -175,7 +175,9 @@ int dynts_cache_capacity(const dynts_cache_t* c);
 
 /* Device [L, Nb, Hkv, cap] fp32 score accumulator.  The caller may overwrite it on the cache's
  * stream to drive the eviction with external scores (e.g. a predictor's).  NULL before storage
- * exists. */
+ * exists.  (The decode step adds each step's mass with compensated summation; the compensation
+ * terms live beside the scores inside the cache, move with them at an eviction, and are at most
+ * one ulp of the score, so overwriting the scores needs no further call.) */
 float* dynts_cache_scores(dynts_cache_t* c);
 
 /* Copy one slab to host buffers (any may be NULL): K, V [n][d] in the cache dtype, pos [n] int32,

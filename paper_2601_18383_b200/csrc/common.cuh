@@ -25,6 +25,7 @@ struct DecodeParams {
   void* V;
   int* pos;           // full [L, Nb, Hkv, cap]
   float* score;       // full [L, Nb, Hkv, cap]
+  float* comp;        // full [L, Nb, Hkv, cap]: rounding error of the score sums (compensated summation)
   int* len;           // [Nb] rows per slab of each sequence
   int* tot;           // [Nb] tokens seen so far (next position id)
   const int* active;  // [Nb]
@@ -46,6 +47,7 @@ struct EvictParams {
   void* V;
   int* pos;
   float* score;
+  float* comp;        // NULL, or the score sums' compensation terms (moved with the scores)
   int* src;           // [slabs, cap] gather list: src[dst] = surviving row index
   int* hdr;           // [slabs, 4]: {first moved dst, rows kept, old length, unused}
   int* len;           // [Nb]
@@ -73,6 +75,21 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {
                : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
                : "l"(p));
   return r;
+}
+
+// Compensated (Kahan) addition of one step's mass x to a score s with running compensation c: the
+// rounding error of each fp32 addition is carried into the next one, so a score accumulated over
+// thousands of steps stays within about one ulp of the exact sum.  Pinned rows (score +inf) are
+// left alone.
+__device__ __forceinline__ void kahan_add(float& s, float& c, float x) {
+  if (s > 3.0e38f) {  // +inf
+    c = 0.f;
+    return;
+  }
+  const float y = __fsub_rn(x, c);
+  const float t = __fadd_rn(s, y);
+  c = __fsub_rn(__fsub_rn(t, s), y);
+  s = t;
 }
 
 // The last CTA of the grid to finish advances the per-sequence lengths: every other CTA has

@@ -124,6 +124,7 @@ __device__ __forceinline__ void cluster_epilogue(const DecodeParams& p, float* p
       }
     }
     float* score = p.score + u.slab * (size_t)p.cap;
+    float* comp = p.comp + u.slab * (size_t)p.cap;
     float* dout = p.delta_out ? p.delta_out + u.slab * (size_t)p.cap : nullptr;
     for (int j = t_begin + (int)threadIdx.x; j < t_end; j += (int)blockDim.x) {
       const float* t = tile + (size_t)(j - t_begin) * G;
@@ -132,8 +133,11 @@ __device__ __forceinline__ void cluster_epilogue(const DecodeParams& p, float* p
       for (int g = 0; g < kMaxGroup; ++g) {
         if (g < G) dl += TILE_IS_P ? t[g] * w[g] : fast_exp2(t[g] - M[g]) * w[g];
       }
-      const float s = (j == n_old) ? 0.f : score[j];
-      score[j] = s + dl;
+      float s = (j == n_old) ? 0.f : score[j];
+      float cc = (j == n_old) ? 0.f : comp[j];
+      kahan_add(s, cc, dl);
+      score[j] = s;
+      comp[j] = cc;
       if (dout) dout[j] = dl;
     }
   }

@@ -158,7 +158,7 @@ __device__ __forceinline__ void cursor_next_slab(StCursor& c, const int* s_cnt, 
 // appended row n_old starting from zero.  GG is the group size at compile time so that every load
 // of a pass is issued before the first use (one memory round trip per pass).
 template <int GG, int VB>
-__device__ __forceinline__ void score_pass_vec(float* __restrict__ score, float* __restrict__ dout,
+__device__ __forceinline__ void score_pass_vec(float* __restrict__ score, float* __restrict__ comp, float* __restrict__ dout,
                                                const float* __restrict__ lg, int cap, int n, int n_old,
                                                const float* s_finM, const float* s_finf, int tid) {
   float M[GG], f[GG];
@@ -168,11 +168,12 @@ __device__ __forceinline__ void score_pass_vec(float* __restrict__ score, float*
     f[g] = s_finf[g];
   }
   for (int v0 = tid; 4 * v0 < n; v0 += VB * kStConsumers) {
-    float4 sc[VB], e[VB][GG];
+    float4 sc[VB], cc[VB], e[VB][GG];
 #pragma unroll
     for (int i = 0; i < VB; ++i) {
       const int j = min(4 * (v0 + i * kStConsumers), cap - 4);  // clamped: always a valid address
       sc[i] = *reinterpret_cast<const float4*>(score + j);
+      cc[i] = *reinterpret_cast<const float4*>(comp + j);
 #pragma unroll
       for (int g = 0; g < GG; ++g) e[i][g] = __ldcg(reinterpret_cast<const float4*>(lg + (size_t)g * cap + j));
     }
@@ -189,18 +190,23 @@ __device__ __forceinline__ void score_pass_vec(float* __restrict__ score, float*
         dl.w += fast_exp2(e[i][g].w - M[g]) * f[g];
       }
       const int z = n_old - j;  // the appended row starts from zero
-      if (z == 0) sc[i].x = 0.f;
-      if (z == 1) sc[i].y = 0.f;
-      if (z == 2) sc[i].z = 0.f;
-      if (z == 3) sc[i].w = 0.f;
-      const float4 r = make_float4(sc[i].x + dl.x, sc[i].y + dl.y, sc[i].z + dl.z, sc[i].w + dl.w);
+      if (z == 0) sc[i].x = cc[i].x = 0.f;
+      if (z == 1) sc[i].y = cc[i].y = 0.f;
+      if (z == 2) sc[i].z = cc[i].z = 0.f;
+      if (z == 3) sc[i].w = cc[i].w = 0.f;
+      kahan_add(sc[i].x, cc[i].x, dl.x);
+      kahan_add(sc[i].y, cc[i].y, dl.y);
+      kahan_add(sc[i].z, cc[i].z, dl.z);
+      kahan_add(sc[i].w, cc[i].w, dl.w);
       if (j + 4 <= n) {
-        *reinterpret_cast<float4*>(score + j) = r;
+        *reinterpret_cast<float4*>(score + j) = sc[i];
+        *reinterpret_cast<float4*>(comp + j) = cc[i];
         if (dout) *reinterpret_cast<float4*>(dout + j) = dl;
       } else {  // rows past the end are left alone
-        score[j] = r.x;
-        if (j + 1 < n) score[j + 1] = r.y;
-        if (j + 2 < n) score[j + 2] = r.z;
+        score[j] = sc[i].x;
+        comp[j] = cc[i].x;
+        if (j + 1 < n) score[j + 1] = sc[i].y, comp[j + 1] = cc[i].y;
+        if (j + 2 < n) score[j + 2] = sc[i].z, comp[j + 2] = cc[i].z;
         if (dout) {
           dout[j] = dl.x;
           if (j + 1 < n) dout[j + 1] = dl.y;
@@ -212,16 +218,19 @@ __device__ __forceinline__ void score_pass_vec(float* __restrict__ score, float*
 }
 
 template <int GG>
-__device__ __forceinline__ void score_pass(float* score, float* dout, const float* lg, int cap, int n, int n_old,
-                                           const float* s_finM, const float* s_finf, int tid) {
+__device__ __forceinline__ void score_pass(float* score, float* comp, float* dout, const float* lg, int cap, int n,
+                                           int n_old, const float* s_finM, const float* s_finf, int tid) {
   if ((cap & 3) == 0 && cap >= 4) {
-    score_pass_vec<GG, (GG <= 4 ? 4 : 2)>(score, dout, lg, cap, n, n_old, s_finM, s_finf, tid);
+    score_pass_vec<GG, (GG <= 4 ? 4 : 2)>(score, comp, dout, lg, cap, n, n_old, s_finM, s_finf, tid);
   } else {
     for (int j = tid; j < n; j += kStConsumers) {
       float dl = 0.f;
 #pragma unroll
       for (int g = 0; g < GG; ++g) dl += fast_exp2(__ldcg(lg + (size_t)g * cap + j) - s_finM[g]) * s_finf[g];
-      score[j] = (j == n_old ? 0.f : score[j]) + dl;
+      float sj = j == n_old ? 0.f : score[j], cj = j == n_old ? 0.f : comp[j];
+      kahan_add(sj, cj, dl);
+      score[j] = sj;
+      comp[j] = cj;
       if (dout) dout[j] = dl;
     }
   }
@@ -661,7 +670,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         // a5: final weights of every row of the slab, summed over the group's heads (Eq. 6)
         consumer_sync();  // s_finM / s_finf, and this CTA's own logits
         float* dout = p.delta_out ? p.delta_out + slab * (size_t)p.cap : nullptr;
-        DYNTS_DISPATCH_GROUP(G, score_pass<GG>(score, dout, lg, p.cap, n, n_old, s_finM, s_finf, tid));
+        DYNTS_DISPATCH_GROUP(G, score_pass<GG>(score, p.comp + slab * (size_t)p.cap, dout, lg, p.cap, n, n_old, s_finM, s_finf, tid));
       }
       consumer_sync();  // shared scratch is reused by the next segment
       it += seg;

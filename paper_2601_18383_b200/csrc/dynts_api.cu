@@ -41,7 +41,7 @@ dynts_status_t fail(dynts_status_t st, const char* fmt, ...) {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  size_t K, V, pos, score, src, hdr, len, tot, pinned, target, active, ticket, logit, part, arrive, total;
+  size_t K, V, pos, score, comp, src, hdr, len, tot, pinned, target, active, ticket, logit, part, arrive, total;
 };
 
 // The streaming decode kernel covers bf16 slabs with head_dim 128.
@@ -85,6 +85,7 @@ Layout make_layout(const dynts_config_t* c, int cap) {
   L.V = take(kv);
   L.pos = take(slabs * cap * 4);
   L.score = take(slabs * cap * 4);
+  L.comp = take(slabs * cap * 4);
   L.src = take(slabs * cap * 4);
   L.hdr = take(slabs * 16);
   L.len = take((size_t)c->batch * 4);
@@ -134,6 +135,7 @@ struct dynts_cache {
   void* V() const { return base + lay.V; }
   int* pos() const { return reinterpret_cast<int*>(base + lay.pos); }
   float* score() const { return reinterpret_cast<float*>(base + lay.score); }
+  float* comp() const { return reinterpret_cast<float*>(base + lay.comp); }
   int* src() const { return reinterpret_cast<int*>(base + lay.src); }
   int* hdr() const { return reinterpret_cast<int*>(base + lay.hdr); }
   int* len() const { return reinterpret_cast<int*>(base + lay.len); }
@@ -284,6 +286,7 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
   p.V = c->V();
   p.pos = c->pos();
   p.score = c->score();
+  p.comp = c->comp();
   p.len = c->len();
   p.tot = c->tot();
   p.active = c->active();
@@ -422,6 +425,7 @@ dynts_status_t do_prefill(dynts_cache* c, int seq, const void* k, const void* v,
   p.V = c->V();
   p.pos = c->pos();
   p.score = c->score();
+  p.comp = c->comp();
   p.len = c->len();
   p.tot = c->tot();
   p.pinned = c->pinned();
@@ -473,6 +477,7 @@ dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validat
   p.V = c->V();
   p.pos = c->pos();
   p.score = c->score();
+  p.comp = c->comp();
   p.src = c->src();
   p.hdr = c->hdr();
   p.len = c->len();
@@ -486,7 +491,7 @@ dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validat
   p.cap = c->cap;
   p.window = c->cfg.window;
   p.elt_bytes = c->elt;
-  const size_t smem = (size_t)c->cap * 8;
+  const size_t smem = (size_t)c->cap * 12;
   dynts_status_t st = ensure_smem_attr(dynts::evict_select_kernel, smem, &c->attr_select, false);
   if (st != DYNTS_OK) return st;
   dynts::evict_select_kernel<<<(unsigned)c->slabs(), dynts::kSelectThreads, smem, c->stream>>>(p);
@@ -741,6 +746,7 @@ dynts_status_t dynts_cache_import(dynts_cache_t* c, int layer, int seq, int head
   CUDA_TRY(cudaMemcpy(static_cast<char*>(c->V()) + slab * c->cap * row_bytes, V, n * row_bytes, cudaMemcpyHostToDevice));
   CUDA_TRY(cudaMemcpy(c->pos() + slab * c->cap, pos, n * sizeof(int), cudaMemcpyHostToDevice));
   CUDA_TRY(cudaMemcpy(c->score() + slab * c->cap, score, n * sizeof(float), cudaMemcpyHostToDevice));
+  CUDA_TRY(cudaMemset(c->comp() + slab * c->cap, 0, n * sizeof(float)));
   int next = n > 0 ? pos[n - 1] + 1 : 0;
   int one = 1;
   CUDA_TRY(cudaMemcpy(c->len() + seq, &n, sizeof(int), cudaMemcpyHostToDevice));
@@ -857,6 +863,7 @@ dynts_status_t dynts_evict_noalloc(void* K, void* V, int* pos, float* score, int
   p.V = V;
   p.pos = pos;
   p.score = score;
+  p.comp = nullptr;
   p.len = base + 0;
   p.pinned = base + 1;
   p.target = base + 2;

@@ -75,6 +75,7 @@ __global__ void __launch_bounds__(kSelectThreads) evict_select_kernel(const Evic
   extern __shared__ __align__(16) uint32_t esm[];
   uint32_t* raw = esm;                                   // [cap] score bit patterns
   int* posbuf = reinterpret_cast<int*>(esm + p.cap);     // [cap]
+  uint32_t* compbuf = esm + 2 * (size_t)p.cap;           // [cap], only with p.comp
   __shared__ unsigned int hist[256];
   __shared__ int warp_tot[32];
   __shared__ uint32_t s_prefix;
@@ -83,9 +84,11 @@ __global__ void __launch_bounds__(kSelectThreads) evict_select_kernel(const Evic
   float* score = p.score + (size_t)slab * p.cap;
   int* pos = p.pos + (size_t)slab * p.cap;
   int* src = p.src + (size_t)slab * p.cap;
+  float* comp = p.comp ? p.comp + (size_t)slab * p.cap : nullptr;
   for (int j = tid; j < n; j += kSelectThreads) {
     raw[j] = __float_as_uint(score[j]);
     posbuf[j] = pos[j];
+    if (comp) compbuf[j] = __float_as_uint(comp[j]);
   }
   if (tid == 0) {
     s_prefix = 0u;
@@ -157,6 +160,7 @@ __global__ void __launch_bounds__(kSelectThreads) evict_select_kernel(const Evic
       src[dst] = j;
       score[dst] = __uint_as_float(raw[j]);
       pos[dst] = posbuf[j];
+      if (comp) comp[dst] = __uint_as_float(compbuf[j]);
     } else if (in) {
       atomicMin(&s_first, j);
     }
@@ -218,6 +222,7 @@ struct PrefillParams {
   void* V;
   int* pos;
   float* score;
+  float* comp;
   int* len;
   int* tot;
   int* pinned;
@@ -252,6 +257,7 @@ __global__ void __launch_bounds__(256) prefill_kernel(const PrefillParams p) {
   for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < p.T; t += gridDim.x * blockDim.x) {
     p.pos[slab * p.cap + t] = t;
     p.score[slab * p.cap + t] = t < p.n_pinned ? __int_as_float(0x7f800000) : 0.f;
+    p.comp[slab * p.cap + t] = 0.f;
   }
   if (blockIdx.x == 0 && threadIdx.x == 0 && l == 0 && h == 0) {
     p.len[b] = p.T;
