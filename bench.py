@@ -187,7 +187,9 @@ def run_ours(args, cfg, rank, world, device):
 
     # ---- per-kernel durations (separate pass: event pairs around every launch) -----------------
     Kp = min(K, 8 * E)
-    dec_events, ev_events, dec_bytes, ev_moved_bytes = [], [], [], []
+    elt = 2 if cfg.dtype == "bf16" else 4
+    row_move_bytes = 2 * (2 * cfg.head_dim * elt + 8)      # K row + V row + pos + score, read and written
+    dec_events, ev_events, dec_bytes = [], [], []
     for i in range(Kp):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         dec_bytes.append(BYTES_PER_SLOT * slots_in_step(cfg, [cache.len(bb) + 1 for bb in range(cfg.batch)]))
@@ -196,16 +198,12 @@ def run_ours(args, cfg, rank, world, device):
         b.record(stream)
         dec_events.append((a, b))
         if (i + 1) % E == 0:
-            need = any(cache.len(bb) > (cfg.seq_budgets[bb] if cfg.seq_budgets else cfg.budget) for bb in range(cfg.batch))
-            if need:
-                # moved rows are known only on the device: read the first-moved index per slab
-                pos_before = None
             a2, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            lens_before = [cache.len(bb) for bb in range(cfg.batch)]
             a2.record(stream)
             cache.evict(0)
             b2.record(stream)
-            ev_events.append((a2, b2, lens_before))
+            scanned, moved = cache.evict_stats()           # synchronises; outside the event pair
+            ev_events.append((a2, b2, 4 * scanned + row_move_bytes * moved))
     torch.cuda.synchronize(device)
     dec_ms = [a.elapsed_time(b) for a, b in dec_events]
     dec_avg_ms = sum(dec_ms) / len(dec_ms)
@@ -223,8 +221,12 @@ def run_ours(args, cfg, rank, world, device):
     evict = None
     if ev_events:
         ev_ms = [a.elapsed_time(b) for a, b, _ in ev_events]
-        evict = {"kernels": "evict_select + evict_compact", "avg_event_us": round(1e3 * sum(ev_ms) / len(ev_ms), 2),
-                 "events_timed": len(ev_ms)}
+        ev_bytes = sum(x for _, _, x in ev_events) / len(ev_events)
+        ev_avg = sum(ev_ms) / len(ev_ms)
+        ev_gbs = ev_bytes / (ev_avg * 1e-3) / 1e9 if ev_avg > 0 else 0.0
+        evict = {"kernels": "evict_select + evict_compact", "bound": "hbm", "achieved": round(ev_gbs, 1), "peak": peak,
+                 "unit": "GB/s", "frac": round(ev_gbs / peak, 4), "algorithmic_bytes_per_event": int(ev_bytes),
+                 "avg_event_us": round(1e3 * ev_avg, 2), "events_timed": len(ev_ms)}
 
     # ---- end to end through the host-buffer entry point ----------------------------------------
     e2e = None
@@ -290,10 +292,9 @@ def oracle_baseline(cfg, cache, q_ring, k_ring, v_ring, budget_s=20.0, slabs=Non
         threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
     except Exception:
         threads = os.cpu_count() or 1
-    # sample: the first `nl` layers, all sequences and heads
+    # sample: layer 0 of every sequence and KV head (exported from the device cache)
     total_slabs = cfg.layers * cfg.batch * cfg.kv_heads
     nl = 1
-    sub = cfg.scaled(layers=nl)
     orc = O.OracleCache(nl, cfg.batch, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.window, cache.capacity)
     for b in range(cfg.batch):
         for h in range(cfg.kv_heads):
@@ -310,7 +311,7 @@ def oracle_baseline(cfg, cache, q_ring, k_ring, v_ring, budget_s=20.0, slabs=Non
     v = v_ring[:, :nl].double().cpu().numpy()
     t0 = time.perf_counter()
     steps = 0
-    while time.perf_counter() - t0 < budget_s and steps < 4 * cfg.evict_interval:
+    while time.perf_counter() - t0 < budget_s and steps < 65536:
         if any(orc.slab(0, b, 0).n + 1 > cache.capacity for b in range(cfg.batch)):
             O.evict(orc, list(cfg.seq_budgets) if cfg.seq_budgets else cfg.budget)
         j = steps % q.shape[0]
@@ -320,7 +321,7 @@ def oracle_baseline(cfg, cache, q_ring, k_ring, v_ring, budget_s=20.0, slabs=Non
     frac = (nl * cfg.batch * cfg.kv_heads) / total_slabs
     value = cfg.batch * steps / dt * frac
     return {"value": round(value, 3), "unit": UNIT, "cores": int(threads), "kind": "oracle",
-            "sample": f"{steps} decode steps (+ evictions as they fall due) of layer 0 of {cfg.layers} "
+            "sample": f"{steps} decode steps (+ evictions as they fall due) over layer 0 of {cfg.layers} "
                       f"({nl * cfg.batch * cfg.kv_heads} of {total_slabs} slabs) in {dt:.1f} s; scaled by the slab fraction"}
 
 

@@ -205,6 +205,11 @@ dynts_status_t dynts_synchronize(dynts_cache_t* c);
  * 8 or 16; 0 => automatic); for variant 3 the CTAs per SM (1 or 2; anything else => 2). */
 dynts_status_t dynts_cache_set_launch(dynts_cache_t* c, int cluster, int variant);
 
+/* Bookkeeping of the most recent eviction, read back from the device (synchronises the stream):
+ * over the slabs that shrank, the rows whose scores were scanned and the rows that changed place
+ * during compaction (rows behind the first evicted one).  For traffic accounting. */
+dynts_status_t dynts_evict_stats(dynts_cache_t* c, long long* rows_scanned, long long* rows_moved);
+
 /* Number of kernels this library has launched on behalf of the cache so far. */
 long long dynts_cache_launch_count(const dynts_cache_t* c);
 

@@ -80,6 +80,7 @@ _sigs = {
     "dynts_synchronize": (C.c_int, [_P]),
     "dynts_cache_set_launch": (C.c_int, [_P, C.c_int, C.c_int]),
     "dynts_cache_launch_count": (C.c_longlong, [_P]),
+    "dynts_evict_stats": (C.c_int, [_P, C.POINTER(C.c_longlong), C.POINTER(C.c_longlong)]),
     "dynts_last_error": (C.c_char_p, []),
     "dynts_version": (C.c_char_p, []),
 }
@@ -233,6 +234,13 @@ def dynts_cache_set_launch(c, cluster=0, variant=0):
     return _check(lib.dynts_cache_set_launch(c, cluster, variant))
 
 
+def dynts_evict_stats(c):
+    """(rows scanned, rows moved) of the most recent eviction."""
+    a, b = C.c_longlong(0), C.c_longlong(0)
+    _check(lib.dynts_evict_stats(c, C.byref(a), C.byref(b)))
+    return a.value, b.value
+
+
 def dynts_cache_launch_count(c) -> int:
     return lib.dynts_cache_launch_count(c)
 
@@ -317,6 +325,9 @@ class Cache:
 
     def poll_error(self):
         return dynts_poll_error(self.handle)
+
+    def evict_stats(self):
+        return dynts_evict_stats(self.handle)
 
     def launch_count(self):
         return dynts_cache_launch_count(self.handle)

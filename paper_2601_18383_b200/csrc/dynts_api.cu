@@ -793,6 +793,24 @@ dynts_status_t dynts_cache_set_launch(dynts_cache_t* c, int cluster, int variant
 
 long long dynts_cache_launch_count(const dynts_cache_t* c) { return c ? c->launches : -1; }
 
+dynts_status_t dynts_evict_stats(dynts_cache_t* c, long long* rows_scanned, long long* rows_moved) {
+  if (!c || !c->ready) return fail(DYNTS_ERR_STATE, "cache holds nothing yet");
+  CUDA_TRY(cudaStreamSynchronize(c->stream));
+  std::vector<int> h(c->slabs() * 4);
+  CUDA_TRY(cudaMemcpy(h.data(), c->hdr(), h.size() * sizeof(int), cudaMemcpyDeviceToHost));
+  long long scanned = 0, moved = 0;
+  for (size_t s = 0; s < c->slabs(); ++s) {
+    const int first = h[4 * s], kept = h[4 * s + 1], old_len = h[4 * s + 2];
+    if (old_len > kept) {  // this slab was evicted by the last eviction
+      scanned += old_len;
+      moved += kept > first ? kept - first : 0;
+    }
+  }
+  if (rows_scanned) *rows_scanned = scanned;
+  if (rows_moved) *rows_moved = moved;
+  return DYNTS_OK;
+}
+
 /* ---- eviction for callers that cannot allocate -------------------------------------------- */
 
 }  // extern "C" (the scratch array and its helpers have internal linkage)
