@@ -126,7 +126,7 @@ struct dynts_cache {
   char* stage_dev = nullptr;
   size_t stage_bytes = 0;
   bool attr_generic_f32 = false, attr_generic_bf16 = false, attr_mma = false, attr_select = false;
-  bool attr_stream = false;
+  bool attr_stream = false, attr_fused = false;
   bool have_maps = false;    // tensor maps of the K and V slabs for the streaming kernel
   CUtensorMap map_K, map_V;
   int sm_count = 0;
@@ -491,16 +491,26 @@ dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validat
   p.cap = c->cap;
   p.window = c->cfg.window;
   p.elt_bytes = c->elt;
-  const size_t smem = (size_t)c->cap * 12;
-  dynts_status_t st = ensure_smem_attr(dynts::evict_select_kernel, smem, &c->attr_select, false);
-  if (st != DYNTS_OK) return st;
-  dynts::evict_select_kernel<<<(unsigned)c->slabs(), dynts::kSelectThreads, smem, c->stream>>>(p);
-  CUDA_TRY(cudaGetLastError());
-  const int pieces = c->cfg.head_dim * c->elt / 16;
-  const unsigned groups = (unsigned)((pieces + 3) / 4);
-  dynts::evict_compact_kernel<<<dim3(2 * groups, (unsigned)c->slabs(), 1), dynts::kCompactThreads, 0, c->stream>>>(p);
-  CUDA_TRY(cudaGetLastError());
-  c->launches += 2;
+  if (c->cap <= 12800) {
+    // one launch: selection and compaction of a slab by the same CTA
+    const size_t smem = (size_t)c->cap * 16;
+    dynts_status_t st = ensure_smem_attr(dynts::evict_fused_kernel, smem, &c->attr_fused, false);
+    if (st != DYNTS_OK) return st;
+    dynts::evict_fused_kernel<<<(unsigned)c->slabs(), dynts::kFusedThreads, smem, c->stream>>>(p, c->ticket() + 1);
+    CUDA_TRY(cudaGetLastError());
+    c->launches += 1;
+  } else {
+    const size_t smem = (size_t)c->cap * 12;
+    dynts_status_t st = ensure_smem_attr(dynts::evict_select_kernel, smem, &c->attr_select, false);
+    if (st != DYNTS_OK) return st;
+    dynts::evict_select_kernel<<<(unsigned)c->slabs(), dynts::kSelectThreads, smem, c->stream>>>(p);
+    CUDA_TRY(cudaGetLastError());
+    const int pieces = c->cfg.head_dim * c->elt / 16;
+    const unsigned groups = (unsigned)((pieces + 3) / 4);
+    dynts::evict_compact_kernel<<<dim3(2 * groups, (unsigned)c->slabs(), 1), dynts::kCompactThreads, 0, c->stream>>>(p);
+    CUDA_TRY(cudaGetLastError());
+    c->launches += 2;
+  }
   for (int b = 0; b < Nb; ++b)
     if (c->active_h[b]) c->len_h[b] = std::min(c->len_h[b], targets[b]);
   return DYNTS_OK;

@@ -213,6 +213,215 @@ __global__ void __launch_bounds__(kCompactThreads) evict_compact_kernel(const Ev
 }
 
 // ---------------------------------------------------------------------------------------------
+// Fused eviction: one CTA per slab selects the survivors (same integer-only rule as
+// evict_select_kernel) and then moves the slab's K and V rows itself, so the gather list never
+// leaves shared memory and one launch does the whole event.  The CTA walks the destination rows in
+// ascending blocks of whole rows; per block every source row is loaded into registers before any
+// destination row is stored, and since src[dst] >= dst with both increasing, a later block never
+// reads a row an earlier block has overwritten.  The new lengths are published by the last CTA of
+// the grid to finish (every CTA reads the old length before it takes its ticket).
+// ---------------------------------------------------------------------------------------------
+constexpr int kFusedThreads = 256;
+constexpr int kFusedUnroll = 8;  // 16-byte loads in flight per thread and tensor (K and V: 16 in total)
+
+// Exclusive prefix sum of one int per thread over the CTA (256 threads), plus the total.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot /* [8] shared */, int& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  int before = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < kFusedThreads / 32; ++w) {
+    const int t = warp_tot[w];
+    if (w < warp) before += t;
+    tot += t;
+  }
+  __syncthreads();  // warp_tot may be reused right after
+  total = tot;
+  return before + incl - v;
+}
+
+__global__ void __launch_bounds__(kFusedThreads) evict_fused_kernel(const EvictParams p, unsigned int* ticket) {
+  const int slab = blockIdx.x;
+  const int b = (slab / p.Hkv) % p.Nb;
+  const int tid = threadIdx.x;
+  const int n = p.len[b];
+  const int tgt = p.target[b];
+  int* hdr = p.hdr + (size_t)slab * 4;
+
+  extern __shared__ __align__(16) uint32_t esm[];
+  uint32_t* raw = esm;                                            // [cap] score bit patterns
+  int* posbuf = reinterpret_cast<int*>(esm + p.cap);              // [cap]
+  uint32_t* compbuf = esm + 2 * (size_t)p.cap;                    // [cap]
+  int* srcbuf = reinterpret_cast<int*>(esm + 3 * (size_t)p.cap);  // [cap] gather list: srcbuf[dst] = surviving row
+  __shared__ unsigned int hist[256];
+  __shared__ int warp_tot[kFusedThreads / 32];
+  __shared__ uint32_t s_prefix;
+  __shared__ int s_krem, s_first;
+
+  if (n > tgt) {  // uniform over the CTA
+    const int M = p.pinned[b];
+    const int lo = M, hi = n - p.window;  // selection window [lo, hi)
+    const int k = tgt - M - p.window;     // survivors wanted from it (host guarantees 0 <= k < hi - lo)
+    float* score = p.score + (size_t)slab * p.cap;
+    int* pos = p.pos + (size_t)slab * p.cap;
+    float* comp = p.comp ? p.comp + (size_t)slab * p.cap : nullptr;
+    for (int j = tid; j < n; j += kFusedThreads) {
+      raw[j] = __float_as_uint(score[j]);
+      posbuf[j] = pos[j];
+      compbuf[j] = comp ? __float_as_uint(comp[j]) : 0u;
+    }
+    if (tid == 0) {
+      s_prefix = 0u;
+      s_krem = k;
+      s_first = n;
+    }
+    __syncthreads();
+
+    // Radix select of the k-th largest key of the selection window (8 bits per pass).
+    uint32_t mask = 0u;
+    if (k > 0) {
+      for (int shift = 24; shift >= 0; shift -= 8) {
+        hist[tid] = 0u;
+        __syncthreads();
+        const uint32_t prefix = s_prefix;
+        const int krem = s_krem;
+        for (int j = lo + tid; j < hi; j += kFusedThreads) {
+          const uint32_t key = order_key(raw[j]);
+          if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (tid < 32) {
+          unsigned int mine = 0;
+          for (int i = 0; i < 8; ++i) mine += hist[255 - 8 * tid - i];
+          unsigned int incl = mine;
+          for (int o = 1; o < 32; o <<= 1) {
+            const unsigned int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (tid >= o) incl += v;
+          }
+          const unsigned int excl = incl - mine;
+          if ((int)excl < krem && krem <= (int)incl) {
+            unsigned int above = excl;
+            for (int i = 0; i < 8; ++i) {
+              const int bin = 255 - 8 * tid - i;
+              const unsigned int c = hist[bin];
+              if ((int)(above + c) >= krem) {
+                s_prefix = prefix | ((uint32_t)bin << shift);
+                s_krem = krem - (int)above;
+                break;
+              }
+              above += c;
+            }
+          }
+        }
+        mask |= 0xFFu << shift;
+        __syncthreads();
+      }
+    }
+    const uint32_t T = s_prefix;   // key of the k-th largest candidate
+    const int take_eq = s_krem;    // rows with key == T that survive (lowest indices first)
+
+    // Every thread owns a contiguous run of rows; two CTA-wide prefix sums give the rank of each
+    // row among the ties and its destination.
+    int run = (n + kFusedThreads - 1) / kFusedThreads;
+    run |= 1;  // odd stride: conflict-free shared-memory walks
+    const int j0 = min(tid * run, n), j1 = min(j0 + run, n);
+    int my_eq = 0;
+    for (int j = j0; j < j1; ++j)
+      if (k > 0 && j >= lo && j < hi && order_key(raw[j]) == T) ++my_eq;
+    int tot;
+    int eq_rank = block_exclusive_scan(my_eq, warp_tot, tot);
+    int my_keep = 0;
+    unsigned long long keepbits = 0ull;  // run <= 64 rows (the host limits the capacity)
+    int first_gone = n;
+    for (int j = j0; j < j1; ++j) {
+      const bool cand = j >= lo && j < hi;
+      bool keep = true;
+      if (cand) {
+        const uint32_t key = order_key(raw[j]);
+        keep = k > 0 && (key > T || (key == T && eq_rank < take_eq));
+        if (k > 0 && key == T) ++eq_rank;
+      }
+      if (keep) {
+        keepbits |= 1ull << (j - j0);
+        ++my_keep;
+      } else {
+        first_gone = min(first_gone, j);
+      }
+    }
+    int dst = block_exclusive_scan(my_keep, warp_tot, tot);
+    for (int j = j0; j < j1; ++j)
+      if ((keepbits >> (j - j0)) & 1ull) srcbuf[dst++] = j;
+    if (first_gone < n) atomicMin(&s_first, first_gone);
+    __syncthreads();
+    const int first = s_first, kept = tot;  // rows below `first` stay where they are; kept == tgt
+    if (tid == 0) {
+      hdr[0] = first;
+      hdr[1] = kept;
+      hdr[2] = n;
+    }
+    // score, pos, compensation of the moved rows (sources are in shared memory: in place is safe)
+    for (int dd = first + tid; dd < kept; dd += kFusedThreads) {
+      const int j = srcbuf[dd];
+      score[dd] = __uint_as_float(raw[j]);
+      pos[dd] = posbuf[j];
+      if (comp) comp[dd] = __uint_as_float(compbuf[j]);
+    }
+    // K and V rows
+    const int row_bytes = p.d * p.elt_bytes;
+    const int pieces = row_bytes >> 4;
+    const int rpp = kFusedThreads / pieces;  // rows per pass
+    const bool active = tid < rpp * pieces;
+    const int r_in = tid / pieces, piece = tid - r_in * pieces;
+    char* Kb = reinterpret_cast<char*>(p.K) + (size_t)slab * p.cap * row_bytes + (size_t)piece * 16;
+    char* Vb = reinterpret_cast<char*>(p.V) + (size_t)slab * p.cap * row_bytes + (size_t)piece * 16;
+    for (int c0 = first; c0 < kept; c0 += rpp * kFusedUnroll) {
+      uint4 kb[kFusedUnroll], vb[kFusedUnroll];
+#pragma unroll
+      for (int uu = 0; uu < kFusedUnroll; ++uu) {
+        const int dd = c0 + uu * rpp + r_in;
+        if (active && dd < kept) {
+          const size_t so = (size_t)srcbuf[dd] * row_bytes;
+          kb[uu] = *reinterpret_cast<const uint4*>(Kb + so);
+          vb[uu] = *reinterpret_cast<const uint4*>(Vb + so);
+        }
+      }
+      __syncthreads();  // every source row of the block is in registers before any row is overwritten
+#pragma unroll
+      for (int uu = 0; uu < kFusedUnroll; ++uu) {
+        const int dd = c0 + uu * rpp + r_in;
+        if (active && dd < kept) {
+          *reinterpret_cast<uint4*>(Kb + (size_t)dd * row_bytes) = kb[uu];
+          *reinterpret_cast<uint4*>(Vb + (size_t)dd * row_bytes) = vb[uu];
+        }
+      }
+    }
+  } else if (tid == 0) {
+    hdr[0] = n;
+    hdr[1] = n;
+    hdr[2] = n;
+  }
+
+  // The last CTA to finish publishes the new lengths.
+  __syncthreads();
+  if (tid == 0) {
+    __threadfence();
+    const unsigned int t = atomicAdd(ticket, 1u);
+    if (t == gridDim.x - 1) {
+      *ticket = 0u;
+      for (int bb = 0; bb < p.Nb; ++bb) p.len[bb] = min(p.len[bb], p.target[bb]);
+      __threadfence();
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Prompt load (question window, Section 4.2).  grid.x = row blocks, grid.y = slabs touched.
 // ---------------------------------------------------------------------------------------------
 struct PrefillParams {
