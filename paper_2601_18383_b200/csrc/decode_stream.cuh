@@ -167,6 +167,7 @@ __device__ __forceinline__ void score_pass_vec(float* __restrict__ score, float*
     M[g] = s_finM[g];
     f[g] = s_finf[g];
   }
+  const bool drop_lines = (cap & 31) == 0;  // then every head's row range starts on a 128-byte line
   for (int v0 = tid; 4 * v0 < n; v0 += VB * kStConsumers) {
     float4 sc[VB], cc[VB], e[VB][GG];
 #pragma unroll
@@ -188,6 +189,13 @@ __device__ __forceinline__ void score_pass_vec(float* __restrict__ score, float*
         dl.y += fast_exp2(e[i][g].y - M[g]) * f[g];
         dl.z += fast_exp2(e[i][g].z - M[g]) * f[g];
         dl.w += fast_exp2(e[i][g].w - M[g]) * f[g];
+      }
+      // The logits of these rows are dead now: drop their L2 lines instead of letting them be
+      // written back to DRAM (each 128-byte line was read by eight lanes of this warp in one load).
+      if (drop_lines && (threadIdx.x & 7) == 0) {
+#pragma unroll
+        for (int g = 0; g < GG; ++g)
+          asm volatile("discard.global.L2 [%0], 128;" ::"l"(lg + (size_t)g * cap + j) : "memory");
       }
       const int z = n_old - j;  // the appended row starts from zero
       if (z == 0) sc[i].x = cc[i].x = 0.f;
