@@ -97,7 +97,8 @@ __device__ __forceinline__ void kahan_add(float& s, float& c, float x) {
 __device__ __forceinline__ void finish_ticket(const DecodeParams& p) {
   __syncthreads();
   if (threadIdx.x == 0) {
-    __threadfence();
+    // (this CTA's reads of the lengths returned their values long ago; no fence is needed to
+    // order them before the ticket)
     unsigned int t = atomicAdd(p.ticket, 1u);
     if (t == gridDim.x - 1) {
       *p.ticket = 0u;

@@ -229,7 +229,7 @@ template <int GG>
 __device__ __forceinline__ void score_pass(float* score, float* comp, float* dout, const float* lg, int cap, int n,
                                            int n_old, const float* s_finM, const float* s_finf, int tid) {
   if ((cap & 3) == 0 && cap >= 4) {
-    score_pass_vec<GG, (GG <= 4 ? 4 : 2)>(score, comp, dout, lg, cap, n, n_old, s_finM, s_finf, tid);
+    score_pass_vec<GG, (GG <= 4 ? 5 : 2)>(score, comp, dout, lg, cap, n, n_old, s_finM, s_finf, tid);
   } else {
     for (int j = tid; j < n; j += kStConsumers) {
       float dl = 0.f;
@@ -332,6 +332,10 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  // The launch may overlap the tail of the kernel before it in the stream (programmatic dependent
+  // launch): nothing above touches global memory; everything below waits until that kernel has
+  // completed and its writes are visible.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (warp == 1) {
     int carry = 0, cmin = 0x7fffffff, cmax = 0;
     for (int b0 = 0; b0 < Nb; b0 += 32) {

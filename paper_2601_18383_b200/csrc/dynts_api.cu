@@ -345,8 +345,18 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
         ctas = (int)used;
       }
     }
-    dynts::decode_attn_stream_kernel<<<ctas, dynts::kStThreads, smem, c->stream>>>(p, c->map_K, c->map_V);
-    cudaError_t e = cudaGetLastError();
+    cudaLaunchConfig_t sc;
+    memset(&sc, 0, sizeof(sc));
+    cudaLaunchAttribute sattr[1];
+    sattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see griddepcontrol.wait in the kernel
+    sattr[0].val.programmaticStreamSerializationAllowed = 1;
+    sc.attrs = sattr;
+    sc.numAttrs = 1;
+    sc.stream = c->stream;
+    sc.gridDim = dim3((unsigned)ctas, 1, 1);
+    sc.blockDim = dim3(dynts::kStThreads, 1, 1);
+    sc.dynamicSmemBytes = smem;
+    cudaError_t e = cudaLaunchKernelEx(&sc, dynts::decode_attn_stream_kernel, p, c->map_K, c->map_V);
     if (e != cudaSuccess) return fail(DYNTS_ERR_CUDA, "decode launch (streaming, %d CTAs): %s", ctas, cudaGetErrorString(e));
     c->launches += 1;
     if (advance)
