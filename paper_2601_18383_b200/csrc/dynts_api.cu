@@ -506,8 +506,18 @@ dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validat
     const size_t smem = (size_t)c->cap * 16;
     dynts_status_t st = ensure_smem_attr(dynts::evict_fused_kernel, smem, &c->attr_fused, false);
     if (st != DYNTS_OK) return st;
-    dynts::evict_fused_kernel<<<(unsigned)c->slabs(), dynts::kFusedThreads, smem, c->stream>>>(p, c->ticket() + 1);
-    CUDA_TRY(cudaGetLastError());
+    cudaLaunchConfig_t fc;
+    memset(&fc, 0, sizeof(fc));
+    cudaLaunchAttribute fattr[1];
+    fattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see griddepcontrol.wait in the kernel
+    fattr[0].val.programmaticStreamSerializationAllowed = 1;
+    fc.attrs = fattr;
+    fc.numAttrs = 1;
+    fc.stream = c->stream;
+    fc.gridDim = dim3((unsigned)c->slabs(), 1, 1);
+    fc.blockDim = dim3(dynts::kFusedThreads, 1, 1);
+    fc.dynamicSmemBytes = smem;
+    CUDA_TRY(cudaLaunchKernelEx(&fc, dynts::evict_fused_kernel, p, c->ticket() + 1));
     c->launches += 1;
   } else {
     const size_t smem = (size_t)c->cap * 12;

@@ -251,6 +251,8 @@ __global__ void __launch_bounds__(kFusedThreads) evict_fused_kernel(const EvictP
   const int slab = blockIdx.x;
   const int b = (slab / p.Hkv) % p.Nb;
   const int tid = threadIdx.x;
+  // Launched with programmatic stream serialisation: wait here for the kernel before this one.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int n = p.len[b];
   const int tgt = p.target[b];
   int* hdr = p.hdr + (size_t)slab * 4;

@@ -104,3 +104,39 @@ def test_config4_full_size_ragged():
     assert [gpu.len(b) for b in range(cfg.batch)] == list(cfg.seq_budgets)
     gpu.close()
     torch.cuda.empty_cache()
+
+
+def test_config5_attention_shapes_layer_by_layer():
+    """The attention part of the full-model configuration (32 layers, 32/8 heads, batch 8, budget
+    3072), driven the way a model drives it: one call per layer.  Window 128 and interval 64 are
+    this build's reading (the configuration names neither)."""
+    cfg = W.get_config("c2_llama8b").scaled(name="c5_attn", batch=8, budget=3072, window=128, evict_interval=64,
+                                             prompt=256, density=0.03)
+    gpu = _steady_state(cfg, 5100, cfg.capacity - 2)
+    slabs = _sample_slabs(cfg, 10, 5)
+    ring = gen.torch_step_ring(cfg, 5100, 2, "cuda:0")
+    out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda:0")
+    delta = torch.zeros((cfg.layers, cfg.batch, cfg.kv_heads, gpu.capacity), dtype=torch.float32, device="cuda:0")
+    G = cfg.group
+    for s in range(2):
+        orc = H.oracle_from_gpu(gpu, cfg, slabs=slabs)
+        q, k, v = ring[0][s], ring[1][s], ring[2][s]
+        for l in range(cfg.layers):
+            gpu.decode_attn_layer(l, q[l], k[l], v[l], out[l], delta)
+        gpu.synchronize()
+        gpu.poll_error()
+        qh, kh, vh = q.double().cpu().numpy(), k.double().cpu().numpy(), v.double().cpu().numpy()
+        og, dh = out.float().cpu().numpy(), delta.cpu().numpy()
+        for (l, b, h) in slabs:
+            sl = orc.slab(l, b, h)
+            sl.K[sl.n], sl.V[sl.n] = kh[l, b, h], vh[l, b, h]
+            n = sl.n + 1
+            alpha = O.attention_weights(qh[l, b, h * G:(h + 1) * G], sl.K[:n])
+            o_ref = O.attention_output(alpha, sl.V[:n])
+            assert H.rel_err_vectors(og[l, b, h * G:(h + 1) * G], o_ref) <= H.TOL_OUT["bf16"]
+            assert float(np.abs(dh[l, b, h, :n] - alpha.sum(axis=0)).max()) <= H.TOL_DELTA
+    assert gpu.len(0) == cfg.capacity
+    H.check_evict_bit_exact(gpu, cfg, 0, slabs=slabs)
+    assert gpu.len(7) == cfg.budget
+    gpu.close()
+    torch.cuda.empty_cache()
