@@ -15,6 +15,9 @@ What each function follows in the paper:
 * ``select_keep`` / ``evict`` -- Section 4.2: the question window (the first M rows) and the local
   window (the last W rows) are always retained, the top-k of the selection window by score are
   retained, the rest are evicted.  Ties go to the lower index; retained rows keep their order.
+* ``set_new_scores`` / ``predictor_mlp`` / ``paper_target`` / ``run_paper_schedule`` -- Section 4.1
+  (Eq. 7: one predictor score per token) and Section 4.2 as written (select when the count reaches
+  the budget B, keep a ratio of the selection window).
 * ``eviction_count`` / ``effective_length`` -- Section 5, the closed form for the cache length.
 * ``attn_flops`` / ``predictor_flops`` / ``break_even_volume`` -- Appendix A and Eq. 9-10.
 
@@ -129,12 +132,15 @@ def prefill(cache: OracleCache, k: np.ndarray, v: np.ndarray, n_pinned: Optional
 
 
 def decode_step(cache: OracleCache, q: np.ndarray, k_new: np.ndarray, v_new: np.ndarray,
-                active: Optional[Sequence[bool]] = None):
+                active: Optional[Sequence[bool]] = None, accumulate: bool = True):
     """One decode step for every (layer, sequence, KV head).
 
     q [L, Nb, Hq, d]; k_new, v_new [L, Nb, Hkv, d].  For each slab: append the new row (its
     score starts at 0), attend over all n rows including the new one (Eq. 4-5), add each row's
     attention mass summed over the group's query heads to its score (Eq. 6).
+
+    With ``accumulate=False`` the scores are left alone (the new row's score stays 0): the
+    caller supplies them, as the paper does with its Importance Predictor (Section 4.1, Eq. 7).
 
     Returns (out [L, Nb, Hq, d] float64, delta) where delta[l][b][h] is this step's mass per
     row, an array of length n.
@@ -156,7 +162,8 @@ def decode_step(cache: OracleCache, q: np.ndarray, k_new: np.ndarray, v_new: np.
         alpha = attention_weights(qg, s.K[:n])                 # Eq. 4
         out[l, b, h * G:(h + 1) * G] = attention_output(alpha, s.V[:n])   # Eq. 5
         dl = alpha.sum(axis=0)                                 # Eq. 6, one more query row per head
-        s.score[:n] += dl
+        if accumulate:                                         # else: scores come from outside (Eq. 7)
+            s.score[:n] += dl
         delta[l][b][h] = dl
     for b in range(Nb):
         if active is None or active[b]:
@@ -213,6 +220,66 @@ def evict(cache: OracleCache, target, scores32=None):
         s.n = m
         kept_all[l][b][h] = kept
     return kept_all
+
+
+# ----------------------------------------------------------------------------------------------
+# Section 4.1-4.2: predictor scores and the paper's own trigger
+# ----------------------------------------------------------------------------------------------
+
+def set_new_scores(cache: OracleCache, s_new: Sequence[float], active: Optional[Sequence[bool]] = None) -> None:
+    """Section 4.2: a newly generated token's importance score is appended beside its KV.  The
+    paper's predictor emits one scalar per token (Eq. 7), so the row appended by the latest
+    decode step gets the same score s_new[b] in every layer and KV head of sequence b."""
+    for l, b, h, s in cache.units():
+        if active is not None and not active[b]:
+            continue
+        assert s.n > 0
+        s.score[s.n - 1] = np.float32(s_new[b])
+
+
+def predictor_mlp(h: np.ndarray, W1, b1, W2, b2, W3, b3, activation: str = "none") -> np.ndarray:
+    """Importance Predictor head (Section 4.1, Appendix A): a three-layer MLP d -> 2d -> d/2 -> 1 on
+    the final hidden state h [Nb, d]; returns one score per sequence, float64.  W_i is [out, in].
+    The paper calls the layers linear and names no activation; ``activation`` ("none" or "relu",
+    applied after the first two layers) is this build's parameter."""
+    act = (lambda x: x) if activation == "none" else (lambda x: np.maximum(x, 0.0))
+    x = np.asarray(h, dtype=np.float64)
+    y1 = act(x @ np.asarray(W1, dtype=np.float64).T + np.asarray(b1, dtype=np.float64))
+    y2 = act(y1 @ np.asarray(W2, dtype=np.float64).T + np.asarray(b2, dtype=np.float64))
+    y3 = y2 @ np.asarray(W3, dtype=np.float64).T + np.asarray(b3, dtype=np.float64)
+    return y3.reshape(-1)
+
+
+def paper_target(M: int, B: int, W_l: int, ratio: float) -> int:
+    """Rows kept by one selection of Section 4.2: the question window (M rows), the local window
+    (W_l rows) and the top ratio * W_s rows of the selection window, W_s = B - M - W_l.  The paper
+    does not say how ratio * W_s is rounded; this build rounds down."""
+    W_s = B - M - W_l
+    if W_s < 0:
+        raise ValueError("question window + local window exceed the budget")
+    return M + int(math.floor(ratio * W_s)) + W_l
+
+
+def run_paper_schedule(cache: OracleCache, prompt_k, prompt_v, stream, steps: int, B: int, ratio: float,
+                       new_scores=None, on_evict=None) -> List[int]:
+    """Section 4.2 as written: prefill (question pinned), decode; once the row count reaches the
+    budget B, select down to paper_target(...).  ``new_scores(s)`` -> [Nb] gives the predictor
+    scores of step s (then attention mass is not accumulated); None => Eq. 6 mass accumulates.
+    Returns the cache length after each step."""
+    prefill(cache, prompt_k, prompt_v)
+    M = cache.n_pinned[0]
+    lengths = []
+    for s in range(1, steps + 1):
+        q, k_new, v_new = stream.step(s)
+        decode_step(cache, q, k_new, v_new, accumulate=new_scores is None)
+        if new_scores is not None:
+            set_new_scores(cache, new_scores(s))
+        if cache.length(0) >= B:
+            kept = evict(cache, paper_target(M, B, cache.window, ratio))
+            if on_evict is not None:
+                on_evict(s, kept)
+        lengths.append(cache.length(0))
+    return lengths
 
 
 # ----------------------------------------------------------------------------------------------

@@ -1,0 +1,134 @@
+"""Pins of the oracle's predictor-score mode and of Section 4.2's own trigger (select when the row
+count reaches the budget B, keep a ratio of the selection window), against the paper's closed
+forms, brute force and algebraic special cases.  CPU only."""
+import math
+
+import numpy as np
+import pytest
+
+import workloads as W
+from oracle import dynts_oracle as O
+
+
+def _small_cfg(**kw):
+    base = dict(layers=2, batch=2, kv_heads=2, q_heads=4, head_dim=16, prompt=12, budget=64, window=8, evict_interval=16)
+    base.update(kw)
+    return W.get_config("c1_tiny_fp32").scaled(**base)
+
+
+def _score_stream(seed, batch):
+    def f(s):
+        return np.random.default_rng([seed, s]).standard_normal(batch).astype(np.float32)
+    return f
+
+
+@pytest.mark.parametrize("ratio", [0.3, 0.4, 0.75])
+def test_lengths_follow_the_closed_form_of_section_5(ratio):
+    """With the trigger at B and K rows leaving per event, the length after decode step i is
+    S_i = M + i - n_i K, n_i = max(0, floor((M + i - B) / K) + 1)."""
+    cfg = _small_cfg()
+    B, M = 64, cfg.prompt
+    W_s = B - M - cfg.window
+    K = W_s - math.floor(ratio * W_s)
+    assert O.paper_target(M, B, cfg.window, ratio) == B - K
+    orc = O.OracleCache(cfg.layers, cfg.batch, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.window, B + 1)
+    pk, pv = W.prompt_kv(cfg, 3)
+    lengths = O.run_paper_schedule(orc, pk.astype(np.float64), pv.astype(np.float64), W.DecodeStream(cfg, 3), 200, B,
+                                   ratio, new_scores=_score_stream(5, cfg.batch))
+    for i, n in enumerate(lengths, start=1):
+        assert n == O.effective_length(M, i, B, K), (i, n)
+        assert n < B
+    assert max(lengths) == B - 1 and O.eviction_count(M, 200, B, K) > 3
+
+
+def test_predictor_scores_give_one_retained_set_per_sequence():
+    """One scalar per token (Eq. 7) appended to every layer and head => every slab of a sequence
+    retains the same positions, and they are the brute-force top-k of the selection window."""
+    cfg = _small_cfg()
+    B, ratio = 64, 0.4
+    orc = O.OracleCache(cfg.layers, cfg.batch, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.window, B + 1)
+    pk, pv = W.prompt_kv(cfg, 4)
+    scores = _score_stream(9, cfg.batch)
+    history = {b: {} for b in range(cfg.batch)}          # position -> score, kept by the test itself
+
+    def new_scores(s):
+        v = scores(s)
+        for b in range(cfg.batch):
+            history[b][cfg.prompt + s - 1] = float(v[b])
+        return v
+
+    events = []
+    O.run_paper_schedule(orc, pk.astype(np.float64), pv.astype(np.float64), W.DecodeStream(cfg, 4), 150, B, ratio,
+                         new_scores=new_scores, on_evict=lambda s, kept: events.append(s))
+    assert len(events) >= 3
+    for b in range(cfg.batch):
+        ref = orc.slab(0, b, 0)
+        for l in range(cfg.layers):
+            for h in range(cfg.kv_heads):
+                sl = orc.slab(l, b, h)
+                assert np.array_equal(sl.pos[:sl.n], ref.pos[:ref.n])
+        # scores stored beside the rows are the predictor's, question rows are +inf
+        for j in range(ref.n):
+            p = int(ref.pos[j])
+            if p < cfg.prompt:
+                assert np.isinf(ref.score[j])
+            else:
+                assert ref.score[j] == np.float32(history[b][p])
+
+
+def test_one_selection_is_brute_force_top_k():
+    r = np.random.default_rng(11)
+    n, M, Wl, B, ratio = 40, 5, 6, 40, 0.5
+    sc = r.standard_normal(n).astype(np.float32)
+    sc[7] = sc[9] = sc[20]                               # ties go to the lower index
+    tgt = O.paper_target(M, B, Wl, ratio)
+    kept = O.select_keep(sc, n, M, Wl, tgt)
+    k = tgt - M - Wl
+    cand = list(range(M, n - Wl))
+    best = sorted(cand, key=lambda j: (-sc[j], j))[:k]
+    assert sorted(kept.tolist()) == sorted(list(range(M)) + best + list(range(n - Wl, n)))
+    # Table 2's "T-Bottom" ablation is the same call on negated scores: the complement of the
+    # top (W_s - k) when there are no ties
+    sc2 = r.standard_normal(n).astype(np.float32)
+    top = set(O.select_keep(sc2, n, M, Wl, tgt).tolist())
+    bottom = set(O.select_keep(-sc2, n, M, Wl, n - (tgt - M - Wl)).tolist())
+    assert (top & bottom) == set(range(M)) | set(range(n - Wl, n))
+
+
+def test_predictor_mlp_shapes_flops_and_linear_collapse():
+    d = 32
+    r = np.random.default_rng(2)
+    W1, b1 = r.standard_normal((2 * d, d)), r.standard_normal(2 * d)
+    W2, b2 = r.standard_normal((d // 2, 2 * d)), r.standard_normal(d // 2)
+    W3, b3 = r.standard_normal((1, d // 2)), r.standard_normal(1)
+    h = r.standard_normal((5, d))
+    # Appendix A counts 2 flops per weight: 6 d^2 + d
+    assert 2 * (W1.size + W2.size + W3.size) == O.predictor_flops(d) == 6 * d * d + d
+    assert O.predictor_flops(4096) == 6 * 4096 ** 2 + 4096
+    # without activation three linear layers collapse into one affine map
+    A = W3 @ W2 @ W1
+    c = W3 @ (W2 @ b1 + b2) + b3
+    np.testing.assert_allclose(O.predictor_mlp(h, W1, b1, W2, b2, W3, b3, "none"), (h @ A.T + c).reshape(-1), rtol=1e-12)
+    # ReLU is the identity on non-negative pre-activations
+    Wp = [np.abs(x) for x in (W1, b1, W2, b2)]
+    hp = np.abs(h)
+    np.testing.assert_allclose(O.predictor_mlp(hp, Wp[0], Wp[1], Wp[2], Wp[3], W3, b3, "relu"),
+                               O.predictor_mlp(hp, Wp[0], Wp[1], Wp[2], Wp[3], W3, b3, "none"), rtol=1e-12)
+    # and zeroes a unit whose pre-activation is negative: one hidden unit, by hand
+    assert O.predictor_mlp(np.array([[1.0, 0.0]]), np.array([[-2.0, 0.0], [3.0, 0.0], [0.0, 0.0], [0.0, 0.0]]), np.zeros(4),
+                           np.array([[1.0, 1.0, 0.0, 0.0]]), np.zeros(1), np.array([[2.0]]), np.array([0.5]), "relu")[0] == 6.5
+
+
+def test_accumulate_off_leaves_scores_alone():
+    cfg = _small_cfg(layers=1, batch=1)
+    orc = O.OracleCache(1, 1, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.window, 80)
+    pk, pv = W.prompt_kv(cfg, 6)
+    O.prefill(orc, pk.astype(np.float64), pv.astype(np.float64), n_pinned=4)
+    st = W.DecodeStream(cfg, 6)
+    before = orc.slab(0, 0, 0).score[:12].copy()
+    out_a, delta = O.decode_step(orc, *[x.astype(np.float64) for x in st.step(1)], accumulate=False)
+    sl = orc.slab(0, 0, 0)
+    assert np.array_equal(sl.score[:12], before) and sl.score[12] == 0.0 and sl.n == 13
+    assert abs(delta[0][0][0].sum() - cfg.group) < 1e-12       # the attention itself is unchanged
+    O.set_new_scores(orc, [0.25])
+    assert sl.score[12] == np.float32(0.25)
