@@ -44,6 +44,8 @@ typedef enum dynts_status {
 
 typedef enum dynts_dtype { DYNTS_BF16 = 0, DYNTS_FP32 = 1 } dynts_dtype_t;
 
+typedef enum dynts_score_source { DYNTS_SCORE_ATTENTION = 0, DYNTS_SCORE_EXTERNAL = 1 } dynts_score_source_t;
+
 typedef struct dynts_config {
   int layers, batch, q_heads, kv_heads, head_dim;
   int budget;         /* B: default eviction target (rows kept per slab) */
@@ -161,6 +163,30 @@ dynts_status_t dynts_evict_ex(dynts_cache_t* c, const int* seq_targets);
  *    current); make that first call before any stream capture begins. */
 dynts_status_t dynts_evict_noalloc(void* K, void* V, int* pos, float* score, int n_slabs, int head_dim, int dtype,
                                    int capacity, int n_rows, int n_pinned, int window, int target, void* stream);
+
+/* ---- predictor scores and the paper's own trigger ------------------------------------------ */
+
+/* Where the importance scores come from.  DYNTS_SCORE_ATTENTION (default): every decode step
+ * adds each retained row's attention mass to its score (Eq. 6 computed online).
+ * DYNTS_SCORE_EXTERNAL: the paper's inference mode (Section 4.1, Eq. 7) -- the decode step leaves
+ * the scores alone and gives the appended row score 0; the caller supplies the token's score with
+ * dynts_append_scores (or writes the accumulator directly, see dynts_cache_scores).  In this mode
+ * the `scores` argument of the decode calls still receives the step's attention mass if given. */
+dynts_status_t dynts_cache_set_score_source(dynts_cache_t* c, int source);
+
+/* Section 4.2: a newly generated token's importance score is stored beside its KV.  s_new: device
+ * [Nb] fp32, one predictor score per sequence (Eq. 7); it becomes the score of the row appended by
+ * the latest decode step in every layer and KV head of each active sequence, so all slabs of a
+ * sequence rank their rows alike and retain the same tokens.  Call after dynts_decode_attn (or
+ * after the last layer of a layer-by-layer step) and before the eviction. */
+dynts_status_t dynts_append_scores(dynts_cache_t* c, const float* s_new);
+
+/* Section 4.2's trigger: every active sequence whose row count has reached budget_B is reduced to
+ * M + floor(ratio * W_s) + W_l rows, W_s = budget_B - M - W_l (question window, top share of the
+ * selection window, local window); the others are left alone.  The paper does not say how
+ * ratio * W_s is rounded: down, here.  budget_B must not exceed the capacity; call it after every
+ * decode step.  DYNTS_ERR_BUDGET if M + W_l > budget_B. */
+dynts_status_t dynts_evict_at_budget(dynts_cache_t* c, int budget_B, double ratio);
 
 /* ---- sequence management and inspection ---------------------------------------------------- */
 

@@ -24,6 +24,8 @@ DYNTS_ERR_CUDA = 6
 DYNTS_ERR_DEVICE = 7
 DYNTS_BF16 = 0
 DYNTS_FP32 = 1
+DYNTS_SCORE_ATTENTION = 0
+DYNTS_SCORE_EXTERNAL = 1
 
 _STATUS_NAMES = {
     0: "DYNTS_OK", 1: "DYNTS_ERR_INVALID_ARG", 2: "DYNTS_ERR_OOM", 3: "DYNTS_ERR_CAPACITY",
@@ -80,6 +82,9 @@ _sigs = {
     "dynts_synchronize": (C.c_int, [_P]),
     "dynts_cache_set_launch": (C.c_int, [_P, C.c_int, C.c_int]),
     "dynts_cache_launch_count": (C.c_longlong, [_P]),
+    "dynts_cache_set_score_source": (C.c_int, [_P, C.c_int]),
+    "dynts_append_scores": (C.c_int, [_P, _P]),
+    "dynts_evict_at_budget": (C.c_int, [_P, C.c_int, C.c_double]),
     "dynts_evict_stats": (C.c_int, [_P, C.POINTER(C.c_longlong), C.POINTER(C.c_longlong)]),
     "dynts_last_error": (C.c_char_p, []),
     "dynts_version": (C.c_char_p, []),
@@ -234,6 +239,18 @@ def dynts_cache_set_launch(c, cluster=0, variant=0):
     return _check(lib.dynts_cache_set_launch(c, cluster, variant))
 
 
+def dynts_cache_set_score_source(c, source):
+    return _check(lib.dynts_cache_set_score_source(c, source))
+
+
+def dynts_append_scores(c, s_new):
+    return _check(lib.dynts_append_scores(c, _ptr(s_new)))
+
+
+def dynts_evict_at_budget(c, budget_B, ratio):
+    return _check(lib.dynts_evict_at_budget(c, budget_B, ratio))
+
+
 def dynts_evict_stats(c):
     """(rows scanned, rows moved) of the most recent eviction."""
     a, b = C.c_longlong(0), C.c_longlong(0)
@@ -325,6 +342,16 @@ class Cache:
 
     def poll_error(self):
         return dynts_poll_error(self.handle)
+
+    def set_score_source(self, source):
+        return dynts_cache_set_score_source(self.handle, source)
+
+    def append_scores(self, s_new):
+        return dynts_append_scores(self.handle, s_new)
+
+    def evict_at_budget(self, budget_B, ratio):
+        r = dynts_evict_at_budget(self.handle, budget_B, ratio)
+        return r
 
     def evict_stats(self):
         return dynts_evict_stats(self.handle)

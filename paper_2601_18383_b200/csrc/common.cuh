@@ -39,6 +39,7 @@ struct DecodeParams {
   int advance;        // 1: the last CTA to finish increments len/tot of active sequences
   int tile_tokens;    // rows of logits a CTA can hold in shared memory
   int slabs_per_cta;  // streaming kernel: > 0 => every CTA takes this many whole slabs
+  int accumulate;     // 1: add each row's attention mass to its score (Eq. 6); 0: scores come from the caller
   float scale_log2;   // log2(e) / sqrt(d)
 };
 

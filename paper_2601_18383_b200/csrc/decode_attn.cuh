@@ -133,11 +133,16 @@ __device__ __forceinline__ void cluster_epilogue(const DecodeParams& p, float* p
       for (int g = 0; g < kMaxGroup; ++g) {
         if (g < G) dl += TILE_IS_P ? t[g] * w[g] : fast_exp2(t[g] - M[g]) * w[g];
       }
-      float s = (j == n_old) ? 0.f : score[j];
-      float cc = (j == n_old) ? 0.f : comp[j];
-      kahan_add(s, cc, dl);
-      score[j] = s;
-      comp[j] = cc;
+      if (p.accumulate) {
+        float s = (j == n_old) ? 0.f : score[j];
+        float cc = (j == n_old) ? 0.f : comp[j];
+        kahan_add(s, cc, dl);
+        score[j] = s;
+        comp[j] = cc;
+      } else if (j == n_old) {  // external scores: the new row starts at 0 until the caller sets it
+        score[j] = 0.f;
+        comp[j] = 0.f;
+      }
       if (dout) dout[j] = dl;
     }
   }

@@ -158,7 +158,7 @@ __device__ __forceinline__ void cursor_next_slab(StCursor& c, const int* s_cnt, 
 // appended row n_old starting from zero.  GG is the group size at compile time so that every load
 // of a pass is issued before the first use (one memory round trip per pass).
 template <int GG, int VB>
-__device__ __forceinline__ void score_pass_vec(float* __restrict__ score, float* __restrict__ comp, float* __restrict__ dout,
+__device__ __forceinline__ void score_pass_vec(bool accumulate, float* __restrict__ score, float* __restrict__ comp, float* __restrict__ dout,
                                                const float* __restrict__ lg, int cap, int n, int n_old,
                                                const float* s_finM, const float* s_finf, int tid) {
   float M[GG], f[GG];
@@ -207,14 +207,18 @@ __device__ __forceinline__ void score_pass_vec(float* __restrict__ score, float*
       kahan_add(sc[i].z, cc[i].z, dl.z);
       kahan_add(sc[i].w, cc[i].w, dl.w);
       if (j + 4 <= n) {
-        *reinterpret_cast<float4*>(score + j) = sc[i];
-        *reinterpret_cast<float4*>(comp + j) = cc[i];
+        if (accumulate) {
+          *reinterpret_cast<float4*>(score + j) = sc[i];
+          *reinterpret_cast<float4*>(comp + j) = cc[i];
+        }
         if (dout) *reinterpret_cast<float4*>(dout + j) = dl;
       } else {  // rows past the end are left alone
-        score[j] = sc[i].x;
-        comp[j] = cc[i].x;
-        if (j + 1 < n) score[j + 1] = sc[i].y, comp[j + 1] = cc[i].y;
-        if (j + 2 < n) score[j + 2] = sc[i].z, comp[j + 2] = cc[i].z;
+        if (accumulate) {
+          score[j] = sc[i].x;
+          comp[j] = cc[i].x;
+          if (j + 1 < n) score[j + 1] = sc[i].y, comp[j + 1] = cc[i].y;
+          if (j + 2 < n) score[j + 2] = sc[i].z, comp[j + 2] = cc[i].z;
+        }
         if (dout) {
           dout[j] = dl.x;
           if (j + 1 < n) dout[j + 1] = dl.y;
@@ -226,19 +230,21 @@ __device__ __forceinline__ void score_pass_vec(float* __restrict__ score, float*
 }
 
 template <int GG>
-__device__ __forceinline__ void score_pass(float* score, float* comp, float* dout, const float* lg, int cap, int n,
-                                           int n_old, const float* s_finM, const float* s_finf, int tid) {
+__device__ __forceinline__ void score_pass(bool accumulate, float* score, float* comp, float* dout, const float* lg, int cap,
+                                           int n, int n_old, const float* s_finM, const float* s_finf, int tid) {
   if ((cap & 3) == 0 && cap >= 4) {
-    score_pass_vec<GG, (GG <= 4 ? 5 : 2)>(score, comp, dout, lg, cap, n, n_old, s_finM, s_finf, tid);
+    score_pass_vec<GG, (GG <= 4 ? 5 : 2)>(accumulate, score, comp, dout, lg, cap, n, n_old, s_finM, s_finf, tid);
   } else {
     for (int j = tid; j < n; j += kStConsumers) {
       float dl = 0.f;
 #pragma unroll
       for (int g = 0; g < GG; ++g) dl += fast_exp2(__ldcg(lg + (size_t)g * cap + j) - s_finM[g]) * s_finf[g];
-      float sj = j == n_old ? 0.f : score[j], cj = j == n_old ? 0.f : comp[j];
-      kahan_add(sj, cj, dl);
-      score[j] = sj;
-      comp[j] = cj;
+      if (accumulate) {
+        float sj = j == n_old ? 0.f : score[j], cj = j == n_old ? 0.f : comp[j];
+        kahan_add(sj, cj, dl);
+        score[j] = sj;
+        comp[j] = cj;
+      }
       if (dout) dout[j] = dl;
     }
   }
@@ -433,6 +439,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
       const int n_old = p.len[c.b];
       const int n = n_old + 1;
       float* lg = p.logit + slab * (size_t)G * p.cap;  // [G][cap]
+      const bool need_pass = p.accumulate || p.delta_out != nullptr;  // else the logits are not needed again
       if (c.lrel >= p.n_layers || c.b >= Nb || c.h >= Hkv || n > p.cap || seg < 1 || c.chunk + seg > c.cb) {
         if (tid == 0) {
           atomicOr(p.err, kErrStreamBounds);
@@ -481,7 +488,13 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
             *reinterpret_cast<uint4*>(box + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = val;
             __nv_bfloat16* grow = reinterpret_cast<__nv_bfloat16*>(isv ? p.V : p.K) + (slab * (size_t)p.cap + n_old) * d;
             reinterpret_cast<uint4*>(grow)[ch] = val;
-            if (lane == 0) p.pos[slab * (size_t)p.cap + n_old] = p.tot[c.b];
+            if (lane == 0) {
+              p.pos[slab * (size_t)p.cap + n_old] = p.tot[c.b];
+              if (!p.accumulate) {  // external scores: the new row starts at 0 until the caller sets it
+                p.score[slab * (size_t)p.cap + n_old] = 0.f;
+                p.comp[slab * (size_t)p.cap + n_old] = 0.f;
+              }
+            }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
           }
@@ -514,7 +527,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           x[1] = (gid < G && tk + 1 < n) ? s0[1] * p.scale_log2 : -CUDART_INF_F;
           x[2] = (gid < G && tk + 8 < n) ? s1[0] * p.scale_log2 : -CUDART_INF_F;
           x[3] = (gid < G && tk + 9 < n) ? s1[1] * p.scale_log2 : -CUDART_INF_F;
-          if (gid < G) {
+          if (gid < G && need_pass) {
             float* t = lg + (size_t)gid * p.cap + tk;  // tk is even: 8-byte stores when the row base allows
             if ((p.cap & 1) == 0 && tk + 9 < n) {
               *reinterpret_cast<float2*>(t) = make_float2(x[0], x[1]);
@@ -678,11 +691,11 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           }
         }
       }
-      if (finish) {
+      if (finish && need_pass) {
         // a5: final weights of every row of the slab, summed over the group's heads (Eq. 6)
         consumer_sync();  // s_finM / s_finf, and this CTA's own logits
         float* dout = p.delta_out ? p.delta_out + slab * (size_t)p.cap : nullptr;
-        DYNTS_DISPATCH_GROUP(G, score_pass<GG>(score, p.comp + slab * (size_t)p.cap, dout, lg, p.cap, n, n_old, s_finM, s_finf, tid));
+        DYNTS_DISPATCH_GROUP(G, score_pass<GG>(p.accumulate != 0, score, p.comp + slab * (size_t)p.cap, dout, lg, p.cap, n, n_old, s_finM, s_finf, tid));
       }
       consumer_sync();  // shared scratch is reused by the next segment
       it += seg;

@@ -121,6 +121,7 @@ struct dynts_cache {
   std::vector<int> seq_budget, len_h, pinned_h, target_h, active_h;
   int layer_cursor = 0;      // next layer expected by dynts_decode_attn_layer
   int cluster = 0, variant = 0;
+  int score_source = 0;      // 0: attention mass accumulates (Eq. 6); 1: the caller supplies scores (Eq. 7)
   long long launches = 0;
   // staging for the host-buffer entry point
   char* stage_dev = nullptr;
@@ -306,6 +307,7 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
   p.advance = advance ? 1 : 0;
   p.tile_tokens = tile_tokens;
   p.slabs_per_cta = 0;
+  p.accumulate = c->score_source == 0 ? 1 : 0;
   p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)f.head_dim));
 
   const bool mma_ok = f.dtype == DYNTS_BF16 && f.head_dim == 128 && c->G <= 8;
@@ -822,6 +824,47 @@ dynts_status_t dynts_cache_set_launch(dynts_cache_t* c, int cluster, int variant
 }
 
 long long dynts_cache_launch_count(const dynts_cache_t* c) { return c ? c->launches : -1; }
+
+dynts_status_t dynts_cache_set_score_source(dynts_cache_t* c, int source) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (source != DYNTS_SCORE_ATTENTION && source != DYNTS_SCORE_EXTERNAL)
+    return fail(DYNTS_ERR_INVALID_ARG, "score source must be DYNTS_SCORE_ATTENTION or DYNTS_SCORE_EXTERNAL");
+  if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "a layer-by-layer step is in progress");
+  c->score_source = source;
+  return DYNTS_OK;
+}
+
+dynts_status_t dynts_append_scores(dynts_cache_t* c, const float* s_new) {
+  if (!c || !s_new) return fail(DYNTS_ERR_INVALID_ARG, "NULL argument");
+  if (!c->ready) return fail(DYNTS_ERR_STATE, "cache holds nothing yet");
+  if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "a layer-by-layer step is in progress");
+  const int n_slabs = (int)c->slabs();
+  dynts::append_scores_kernel<<<(n_slabs + 255) / 256, 256, 0, c->stream>>>(c->score(), c->comp(), c->len(), c->active(), s_new,
+                                                                          n_slabs, c->cfg.batch, c->cfg.kv_heads, c->cap);
+  CUDA_TRY(cudaGetLastError());
+  c->launches += 1;
+  return DYNTS_OK;
+}
+
+dynts_status_t dynts_evict_at_budget(dynts_cache_t* c, int budget_B, double ratio) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (!c->ready) return fail(DYNTS_ERR_STATE, "cache holds nothing yet");
+  if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "evict in the middle of a layer-by-layer step");
+  if (budget_B < 1 || budget_B > c->cap || !(ratio >= 0.0 && ratio <= 1.0))
+    return fail(DYNTS_ERR_INVALID_ARG, "budget %d outside [1, capacity %d] or ratio %g outside [0, 1]", budget_B, c->cap, ratio);
+  const int Nb = c->cfg.batch;
+  std::vector<int> t(Nb);
+  for (int b = 0; b < Nb; ++b) {
+    t[b] = c->cap;  // no eviction for this sequence
+    if (!c->active_h[b] || c->len_h[b] < budget_B) continue;
+    const int w_s = budget_B - c->pinned_h[b] - c->cfg.window;
+    if (w_s < 0)
+      return fail(DYNTS_ERR_BUDGET, "sequence %d: question window %d + local window %d exceed the budget %d", b,
+                  c->pinned_h[b], c->cfg.window, budget_B);
+    t[b] = c->pinned_h[b] + (int)std::floor(ratio * (double)w_s) + c->cfg.window;
+  }
+  return do_evict(c, t.data());
+}
 
 dynts_status_t dynts_evict_stats(dynts_cache_t* c, long long* rows_scanned, long long* rows_moved) {
   if (!c || !c->ready) return fail(DYNTS_ERR_STATE, "cache holds nothing yet");

@@ -424,6 +424,21 @@ __global__ void __launch_bounds__(kFusedThreads) evict_fused_kernel(const EvictP
 }
 
 // ---------------------------------------------------------------------------------------------
+// Predictor scores (Section 4.1, Eq. 7; Section 4.2: a new token's score is appended beside its
+// KV): the row appended by the latest decode step gets s_new[b] in every slab of sequence b.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) append_scores_kernel(float* score, float* comp, const int* len, const int* active,
+                                                            const float* s_new, int n_slabs, int Nb, int Hkv, int cap) {
+  const int slab = blockIdx.x * blockDim.x + threadIdx.x;
+  if (slab >= n_slabs) return;
+  const int b = (slab / Hkv) % Nb;
+  const int n = len[b];
+  if (!active[b] || n < 1 || n > cap) return;
+  score[(size_t)slab * cap + n - 1] = s_new[b];
+  comp[(size_t)slab * cap + n - 1] = 0.f;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Prompt load (question window, Section 4.2).  grid.x = row blocks, grid.y = slabs touched.
 // ---------------------------------------------------------------------------------------------
 struct PrefillParams {
