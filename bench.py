@@ -139,10 +139,21 @@ def run_ours(args, cfg, rank, world, device):
     q_ring, k_ring, v_ring = gen.torch_step_ring(cfg, 77 + rank, ring_n, device)
     out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=q_ring.dtype, device=device)
     stream = torch.cuda.current_stream(device)
+    external = args.score_source == "external"
+    bytes_per_slot = BYTES_PER_SLOT - 8 if external else BYTES_PER_SLOT   # no score read-modify-write
+    if external:
+        import paper_2601_18383_b200 as D
+        cache.set_score_source(D.DYNTS_SCORE_EXTERNAL)
+        g = torch.Generator(device=device).manual_seed(4242 + rank)
+        s_ring = torch.randn((ring_n, cfg.batch), generator=g, device=device)   # stand-in for predictor outputs
+
+    def decode(j):
+        cache.decode_attn(q_ring[j], k_ring[j], v_ring[j], out)
+        if external:
+            cache.append_scores(s_ring[j])
 
     def step(i):
-        j = i % ring_n
-        cache.decode_attn(q_ring[j], k_ring[j], v_ring[j], out)
+        decode(i % ring_n)
         if (i + 1) % E == 0:
             cache.evict(0)
 
@@ -199,8 +210,8 @@ def run_ours(args, cfg, rank, world, device):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
         for j in range(i, i + run):
-            dec_bytes.append(BYTES_PER_SLOT * slots_in_step(cfg, [cache.len(bb) + 1 for bb in range(cfg.batch)]))
-            cache.decode_attn(q_ring[j % ring_n], k_ring[j % ring_n], v_ring[j % ring_n], out)
+            dec_bytes.append(bytes_per_slot * slots_in_step(cfg, [cache.len(bb) + 1 for bb in range(cfg.batch)]))
+            decode(j % ring_n)
         b.record(stream)
         dec_events.append((a, b, run))
         i += run
@@ -218,10 +229,11 @@ def run_ours(args, cfg, rank, world, device):
     peak, peak_kind = measured_peaks()
     algo_bytes = sum(dec_bytes) / len(dec_bytes)
     roofline = {
-        "kernel": "decode_attn (fused append + attention + importance accumulation)",
+        "kernel": "decode_attn (fused append + attention" + (" + append of the token's predictor score)" if external
+                                                                 else " + importance accumulation)"),
         "bound": "hbm", "achieved": round(dec_gbs, 1), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
         "frac": round(dec_gbs / peak, 4),
-        "traffic": None if NCU_TRAFFIC_RATIO is None else int(NCU_TRAFFIC_RATIO * algo_bytes),
+        "traffic": None if (NCU_TRAFFIC_RATIO is None or external or cfg.name != "c2_llama8b") else int(NCU_TRAFFIC_RATIO * algo_bytes),
         "algorithmic_bytes_per_launch": int(algo_bytes), "avg_launch_us": round(dec_avg_ms * 1e3, 2),
         "launches_timed": dec_launches,
     }
@@ -278,7 +290,7 @@ def run_ours(args, cfg, rank, world, device):
         "dtype": "bf16 inputs, fp32 accumulate" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": cfg.name, "layers": cfg.layers, "batch": cfg.batch, "q_heads": cfg.q_heads,
                    "kv_heads": cfg.kv_heads, "head_dim": cfg.head_dim, "budget": cfg.budget, "window": cfg.window,
-                   "evict_interval": E, "prompt_pinned": cfg.prompt, "dist": cfg.dist,
+                   "evict_interval": E, "prompt_pinned": cfg.prompt, "dist": cfg.dist, "score_source": args.score_source,
                    "cache_bytes": cache.nbytes, "l2_policy": "inputs larger than L2 (KV cache %.0f MB vs 126 MB L2)" % (cache.nbytes / 1e6),
                    "replicas": world},
         "hbm_gbs_decode": round(dec_gbs, 1), "roofline": roofline, "evict": evict, "e2e": e2e,
@@ -405,6 +417,8 @@ def main():
     ap.add_argument("--workload", default="c2_llama8b", choices=sorted(W.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--score-source", default="attention", choices=["attention", "external"],
+                    help="attention: Eq. 6 mass accumulated online (default); external: one predictor score per token (Eq. 7)")
     ap.add_argument("--cluster", type=int, default=0)
     ap.add_argument("--variant", type=int, default=0)
     args = ap.parse_args()
