@@ -133,6 +133,14 @@ dynts_status_t dynts_decode_attn_host(dynts_cache_t* c, const void* q, const voi
  * must shrink. */
 dynts_status_t dynts_evict(dynts_cache_t* c, int budget);
 
+/* Eviction with one selection per sequence (Appendix B.1 aggregates a token's importance across
+ * all layers and heads): the scores of all slabs of a sequence are summed row by row (float32,
+ * layer-major then KV head) and every slab ranks its selection window by that sum, so all
+ * layers and heads keep the same tokens.  Requires that all slabs of a sequence hold the same
+ * tokens, i.e. that every eviction of this cache is of this kind (or driven by shared external
+ * scores).  Otherwise as dynts_evict.  Up to 10000 rows per slab. */
+dynts_status_t dynts_evict_global(dynts_cache_t* c, int budget);
+
 /* Eviction with one target per sequence; seq_targets: host [Nb]. */
 dynts_status_t dynts_evict_ex(dynts_cache_t* c, const int* seq_targets);
 

@@ -70,6 +70,7 @@ _sigs = {
     "dynts_decode_attn_layer": (C.c_int, [_P, C.c_int, _P, _P, _P, _P, _P]),
     "dynts_decode_attn_host": (C.c_int, [_P, _P, _P, _P, _P]),
     "dynts_evict": (C.c_int, [_P, C.c_int]),
+    "dynts_evict_global": (C.c_int, [_P, C.c_int]),
     "dynts_evict_ex": (C.c_int, [_P, C.POINTER(C.c_int)]),
     "dynts_evict_noalloc": (C.c_int, [_P, _P, _P, _P] + [C.c_int] * 8 + [_P]),
     "dynts_seq_reset": (C.c_int, [_P, C.c_int]),
@@ -187,6 +188,10 @@ def dynts_decode_attn_host(c, q, k_new, v_new, out):
 
 def dynts_evict(c, budget=0):
     return _check(lib.dynts_evict(c, budget))
+
+
+def dynts_evict_global(c, budget=0):
+    return _check(lib.dynts_evict_global(c, budget))
 
 
 def dynts_evict_ex(c, seq_targets: Sequence[int]):
@@ -321,6 +326,9 @@ class Cache:
 
     def evict(self, budget=0):
         return dynts_evict(self.handle, budget)
+
+    def evict_global(self, budget=0):
+        return dynts_evict_global(self.handle, budget)
 
     def evict_ex(self, targets):
         return dynts_evict_ex(self.handle, targets)

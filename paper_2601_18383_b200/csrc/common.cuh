@@ -49,6 +49,7 @@ struct EvictParams {
   int* pos;
   float* score;
   float* comp;        // NULL, or the score sums' compensation terms (moved with the scores)
+  const float* key;   // NULL, or [Nb, cap] selection keys shared by all slabs of a sequence (fused kernel only)
   int* src;           // [slabs, cap] gather list: src[dst] = surviving row index
   int* hdr;           // [slabs, 4]: {first moved dst, rows kept, old length, unused}
   int* len;           // [Nb]

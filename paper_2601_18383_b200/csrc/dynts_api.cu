@@ -41,7 +41,7 @@ dynts_status_t fail(dynts_status_t st, const char* fmt, ...) {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  size_t K, V, pos, score, comp, src, hdr, len, tot, pinned, target, active, ticket, logit, part, arrive, total;
+  size_t K, V, pos, score, comp, agg, src, hdr, len, tot, pinned, target, active, ticket, logit, part, arrive, total;
 };
 
 // The streaming decode kernel covers bf16 slabs with head_dim 128.
@@ -86,6 +86,7 @@ Layout make_layout(const dynts_config_t* c, int cap) {
   L.pos = take(slabs * cap * 4);
   L.score = take(slabs * cap * 4);
   L.comp = take(slabs * cap * 4);
+  L.agg = take((size_t)c->batch * cap * 4);
   L.src = take(slabs * cap * 4);
   L.hdr = take(slabs * 16);
   L.len = take((size_t)c->batch * 4);
@@ -137,6 +138,7 @@ struct dynts_cache {
   int* pos() const { return reinterpret_cast<int*>(base + lay.pos); }
   float* score() const { return reinterpret_cast<float*>(base + lay.score); }
   float* comp() const { return reinterpret_cast<float*>(base + lay.comp); }
+  float* agg() const { return reinterpret_cast<float*>(base + lay.agg); }
   int* src() const { return reinterpret_cast<int*>(base + lay.src); }
   int* hdr() const { return reinterpret_cast<int*>(base + lay.hdr); }
   int* len() const { return reinterpret_cast<int*>(base + lay.len); }
@@ -466,7 +468,7 @@ dynts_status_t do_prefill(dynts_cache* c, int seq, const void* k, const void* v,
   return DYNTS_OK;
 }
 
-dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validated */) {
+dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validated */, bool global = false) {
   const int Nb = c->cfg.batch;
   bool any = false;
   for (int b = 0; b < Nb; ++b) {
@@ -490,6 +492,7 @@ dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validat
   p.pos = c->pos();
   p.score = c->score();
   p.comp = c->comp();
+  p.key = nullptr;
   p.src = c->src();
   p.hdr = c->hdr();
   p.len = c->len();
@@ -503,9 +506,18 @@ dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validat
   p.cap = c->cap;
   p.window = c->cfg.window;
   p.elt_bytes = c->elt;
+  if (global) {
+    // one score per token: sum the slab scores of each sequence, every slab then ranks by the sum
+    if (c->cap > 10000) return fail(DYNTS_ERR_CAPACITY, "sequence-wide selection supports up to 10000 rows per slab");
+    dynts::aggregate_scores_kernel<<<dim3((unsigned)((c->cap + 255) / 256), (unsigned)Nb, 1), 256, 0, c->stream>>>(
+        c->score(), c->agg(), c->len(), c->active(), c->cfg.layers, Nb, c->cfg.kv_heads, c->cap);
+    CUDA_TRY(cudaGetLastError());
+    c->launches += 1;
+    p.key = c->agg();
+  }
   if (c->cap <= 12800) {
     // one launch: selection and compaction of a slab by the same CTA
-    const size_t smem = (size_t)c->cap * 16;
+    const size_t smem = (size_t)c->cap * (global ? 20 : 16);
     dynts_status_t st = ensure_smem_attr(dynts::evict_fused_kernel, smem, &c->attr_fused, false);
     if (st != DYNTS_OK) return st;
     cudaLaunchConfig_t fc;
@@ -703,6 +715,15 @@ dynts_status_t dynts_evict(dynts_cache_t* c, int budget) {
   std::vector<int> t(c->cfg.batch);
   for (int b = 0; b < c->cfg.batch; ++b) t[b] = budget > 0 ? budget : c->seq_budget[b];
   return do_evict(c, t.data());
+}
+
+dynts_status_t dynts_evict_global(dynts_cache_t* c, int budget) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (!c->ready) return fail(DYNTS_ERR_STATE, "cache holds nothing yet");
+  if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "evict in the middle of a layer-by-layer step");
+  std::vector<int> t(c->cfg.batch);
+  for (int b = 0; b < c->cfg.batch; ++b) t[b] = budget > 0 ? budget : c->seq_budget[b];
+  return do_evict(c, t.data(), true);
 }
 
 dynts_status_t dynts_evict_ex(dynts_cache_t* c, const int* seq_targets) {
@@ -955,6 +976,7 @@ dynts_status_t dynts_evict_noalloc(void* K, void* V, int* pos, float* score, int
   p.pos = pos;
   p.score = score;
   p.comp = nullptr;
+  p.key = nullptr;
   p.len = base + 0;
   p.pinned = base + 1;
   p.target = base + 2;

@@ -262,6 +262,7 @@ __global__ void __launch_bounds__(kFusedThreads) evict_fused_kernel(const EvictP
   int* posbuf = reinterpret_cast<int*>(esm + p.cap);              // [cap]
   uint32_t* compbuf = esm + 2 * (size_t)p.cap;                    // [cap]
   int* srcbuf = reinterpret_cast<int*>(esm + 3 * (size_t)p.cap);  // [cap] gather list: srcbuf[dst] = surviving row
+  uint32_t* sel = p.key ? esm + 4 * (size_t)p.cap : raw;          // [cap] bit patterns the selection ranks by
   __shared__ unsigned int hist[256];
   __shared__ int warp_tot[kFusedThreads / 32];
   __shared__ uint32_t s_prefix;
@@ -278,6 +279,7 @@ __global__ void __launch_bounds__(kFusedThreads) evict_fused_kernel(const EvictP
       raw[j] = __float_as_uint(score[j]);
       posbuf[j] = pos[j];
       compbuf[j] = comp ? __float_as_uint(comp[j]) : 0u;
+      if (p.key) sel[j] = __float_as_uint(p.key[(size_t)b * p.cap + j]);
     }
     if (tid == 0) {
       s_prefix = 0u;
@@ -295,7 +297,7 @@ __global__ void __launch_bounds__(kFusedThreads) evict_fused_kernel(const EvictP
         const uint32_t prefix = s_prefix;
         const int krem = s_krem;
         for (int j = lo + tid; j < hi; j += kFusedThreads) {
-          const uint32_t key = order_key(raw[j]);
+          const uint32_t key = order_key(sel[j]);
           if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
         }
         __syncthreads();
@@ -336,7 +338,7 @@ __global__ void __launch_bounds__(kFusedThreads) evict_fused_kernel(const EvictP
     const int j0 = min(tid * run, n), j1 = min(j0 + run, n);
     int my_eq = 0;
     for (int j = j0; j < j1; ++j)
-      if (k > 0 && j >= lo && j < hi && order_key(raw[j]) == T) ++my_eq;
+      if (k > 0 && j >= lo && j < hi && order_key(sel[j]) == T) ++my_eq;
     int tot;
     int eq_rank = block_exclusive_scan(my_eq, warp_tot, tot);
     int my_keep = 0;
@@ -346,7 +348,7 @@ __global__ void __launch_bounds__(kFusedThreads) evict_fused_kernel(const EvictP
       const bool cand = j >= lo && j < hi;
       bool keep = true;
       if (cand) {
-        const uint32_t key = order_key(raw[j]);
+        const uint32_t key = order_key(sel[j]);
         keep = k > 0 && (key > T || (key == T && eq_rank < take_eq));
         if (k > 0 && key == T) ++eq_rank;
       }
@@ -421,6 +423,22 @@ __global__ void __launch_bounds__(kFusedThreads) evict_fused_kernel(const EvictP
       __threadfence();
     }
   }
+}
+
+// ---------------------------------------------------------------------------------------------
+// One importance score per token, aggregated across all layers and KV heads (Appendix B.1):
+// agg[b][j] = sum over (layer, head) of score[layer][b][head][j], added in float32 in that order
+// (the order is part of the result: it decides a ranking).  grid = (row blocks, sequences).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) aggregate_scores_kernel(const float* score, float* agg, const int* len,
+                                                               const int* active, int L, int Nb, int Hkv, int cap) {
+  const int b = blockIdx.y;
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (!active[b] || j >= len[b] || j >= cap) return;
+  float acc = 0.f;
+  for (int l = 0; l < L; ++l)
+    for (int h = 0; h < Hkv; ++h) acc = __fadd_rn(acc, score[(((size_t)l * Nb + b) * Hkv + h) * cap + j]);
+  agg[(size_t)b * cap + j] = acc;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -104,3 +104,51 @@ def test_external_mode_without_delta_output_and_argument_checks():
     gpu.evict_at_budget(40, 0.5)                        # 31 rows < 40: nothing happens
     assert gpu.len(0) == 31
     gpu.close()
+
+
+@pytest.mark.parametrize("name", ["c2_llama8b", "c3_qwen7b", "c1_tiny_fp32"])
+def test_sequence_wide_selection_on_aggregated_scores(name):
+    """Attention mass accumulates per slab; at every eviction the slab scores of a sequence are
+    summed (Appendix B.1) and one selection per sequence is applied to all layers and heads.  The
+    oracle repeats the decision from the device's own float32 scores: the compacted state of every
+    slab must then be bit-identical."""
+    extra = {"kv_heads": 2, "q_heads": 14} if name == "c3_qwen7b" else {}
+    cfg = W.get_config(name).scaled(layers=3, batch=2, prompt=24, budget=96, window=16, evict_interval=32, **extra)
+    gpu, orc = H.make_gpu(cfg), H.make_oracle(cfg)
+    pk, pv = W.prompt_kv(cfg, 31)
+    gpu.prefill(H.dev(pk, cfg), H.dev(pv, cfg))
+    O.prefill(orc, pk.astype(np.float64), pv.astype(np.float64))
+    stream = W.DecodeStream(cfg, 31)
+    out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=H.tdtype(cfg), device="cuda:0")
+    events = moved = 0
+    worst_score = 0.0
+    for s in range(1, 225):
+        q, k, v = stream.step(s)
+        gpu.decode_attn(H.dev(q, cfg), H.dev(k, cfg), H.dev(v, cfg), out)
+        O.decode_step(orc, q.astype(np.float64), k.astype(np.float64), v.astype(np.float64))
+        if s % cfg.evict_interval:
+            continue
+        sc = gpu.scores_tensor().cpu().numpy()
+        pre = H.export_all(gpu, cfg)
+        for l, b, h, sl in orc.units():
+            fin = np.isfinite(sl.score[:sl.n])
+            worst_score = max(worst_score, float(np.abs(sc[l, b, h, :sl.n][fin] - sl.score[:sl.n][fin]).max()))
+        n_before = gpu.len(0)
+        gpu.evict_global(0)
+        gpu.synchronize()
+        gpu.poll_error()
+        kept = O.evict_global(orc, cfg.budget, scores32=lambda l, b, h: sc[l, b, h])
+        for l, b, h, sl in orc.units():
+            K0, V0, p0, s0 = pre[(l, b, h)]
+            K1, V1, p1, s1 = gpu.export_slab(l, b, h)
+            idx = torch.from_numpy(kept[b])
+            assert K1.shape[0] == sl.n == len(kept[b])
+            assert torch.equal(p1, p0[idx]) and torch.equal(H.bits(s1), H.bits(s0[idx]))
+            assert torch.equal(H.bits(K1), H.bits(K0[idx])) and torch.equal(H.bits(V1), H.bits(V0[idx]))
+            assert np.array_equal(p1.numpy(), sl.pos[:sl.n])
+            sl.score[:sl.n] = s1.numpy().astype(np.float64)       # re-synchronise
+        if n_before > cfg.budget:
+            events += 1
+            moved += sum(int((kk != np.arange(len(kk))).sum()) for kk in kept)
+    assert events >= 3 and moved > 0 and worst_score <= H.TOL_DELTA, (events, moved, worst_score)
+    gpu.close()
