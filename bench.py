@@ -147,6 +147,8 @@ def run_ours(args, cfg, rank, world, device):
         g = torch.Generator(device=device).manual_seed(4242 + rank)
         s_ring = torch.randn((ring_n, cfg.batch), generator=g, device=device)   # stand-in for predictor outputs
 
+    evict_call = cache.evict_global if args.selection == "global" else cache.evict
+
     def decode(j):
         cache.decode_attn(q_ring[j], k_ring[j], v_ring[j], out)
         if external:
@@ -155,7 +157,7 @@ def run_ours(args, cfg, rank, world, device):
     def step(i):
         decode(i % ring_n)
         if (i + 1) % E == 0:
-            cache.evict(0)
+            evict_call(0)
 
     def barrier():
         if world > 1:
@@ -218,7 +220,7 @@ def run_ours(args, cfg, rank, world, device):
         if i % E == 0:
             a2, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a2.record(stream)
-            cache.evict(0)
+            evict_call(0)
             b2.record(stream)
             scanned, moved = cache.evict_stats()           # synchronises; outside the event pair
             ev_events.append((a2, b2, 4 * scanned + row_move_bytes * moved))
@@ -259,13 +261,13 @@ def run_ours(args, cfg, rank, world, device):
             cache.decode_attn_host(hq[i], hk[i], hv[i], hout)
         # re-align to the eviction cycle
         while cache.len(0) % 1 == 0 and any(cache.len(bb) >= cache.capacity for bb in range(cfg.batch)):
-            cache.evict(0)
+            evict_call(0)
         barrier()
         t0 = time.perf_counter()
         steps_done = 0
         for i in range(Ke):
             if any(cache.len(bb) + 1 > cache.capacity for bb in range(cfg.batch)):
-                cache.evict(0)
+                evict_call(0)
             cache.decode_attn_host(hq[i % ring_n], hk[i % ring_n], hv[i % ring_n], hout)
             steps_done += 1
         torch.cuda.synchronize(device)
@@ -290,7 +292,7 @@ def run_ours(args, cfg, rank, world, device):
         "dtype": "bf16 inputs, fp32 accumulate" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": cfg.name, "layers": cfg.layers, "batch": cfg.batch, "q_heads": cfg.q_heads,
                    "kv_heads": cfg.kv_heads, "head_dim": cfg.head_dim, "budget": cfg.budget, "window": cfg.window,
-                   "evict_interval": E, "prompt_pinned": cfg.prompt, "dist": cfg.dist, "score_source": args.score_source,
+                   "evict_interval": E, "prompt_pinned": cfg.prompt, "dist": cfg.dist, "score_source": args.score_source, "selection": args.selection,
                    "cache_bytes": cache.nbytes, "l2_policy": "inputs larger than L2 (KV cache %.0f MB vs 126 MB L2)" % (cache.nbytes / 1e6),
                    "replicas": world},
         "hbm_gbs_decode": round(dec_gbs, 1), "roofline": roofline, "evict": evict, "e2e": e2e,
@@ -419,6 +421,8 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--score-source", default="attention", choices=["attention", "external"],
                     help="attention: Eq. 6 mass accumulated online (default); external: one predictor score per token (Eq. 7)")
+    ap.add_argument("--selection", default="slab", choices=["slab", "global"],
+                    help="slab: every (layer, KV head) selects on its own scores; global: one selection per sequence")
     ap.add_argument("--cluster", type=int, default=0)
     ap.add_argument("--variant", type=int, default=0)
     args = ap.parse_args()

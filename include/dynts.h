@@ -196,6 +196,20 @@ dynts_status_t dynts_append_scores(dynts_cache_t* c, const float* s_new);
  * decode step.  DYNTS_ERR_BUDGET if M + W_l > budget_B. */
 dynts_status_t dynts_evict_at_budget(dynts_cache_t* c, int budget_B, double ratio);
 
+/* Importance Predictor head (Section 4.1, Eq. 7; Appendix A): scores[n] = MLP(h[n]) with layers
+ * d -> 2d -> d/2 -> 1.  The paper calls the layers linear and names no activation: activation 0
+ * applies none, 1 applies ReLU after the first two layers.
+ *   h: device [batch][d] bf16 (final hidden states);  W1 [2d][d], W2 [d/2][2d], W3 [1][d/2]: device
+ *   bf16, row-major [out][in];  b1 [2d], b2 [d/2], b3 [1]: device fp32 or NULL;  scores: device
+ *   [batch] fp32 (ready for dynts_append_scores).  Accumulation and the hidden activations are fp32.
+ *   scratch: device memory of dynts_predictor_mlp_scratch_bytes(d, batch) bytes, 16-byte aligned,
+ *   caller-owned (holds partial sums between the layers; contents need not be preserved).
+ * d must be a multiple of 512.  Three launches on `stream`; allocates nothing. */
+size_t dynts_predictor_mlp_scratch_bytes(int d, int batch);
+dynts_status_t dynts_predictor_mlp(const void* h, const void* W1, const float* b1, const void* W2, const float* b2,
+                                   const void* W3, const float* b3, int d, int batch, int activation, void* scratch,
+                                   size_t scratch_bytes, float* scores, void* stream);
+
 /* ---- sequence management and inspection ---------------------------------------------------- */
 
 /* Ragged batches: mark a sequence finished (length 0, inactive) until its next prefill_seq. */

@@ -86,6 +86,8 @@ _sigs = {
     "dynts_cache_set_score_source": (C.c_int, [_P, C.c_int]),
     "dynts_append_scores": (C.c_int, [_P, _P]),
     "dynts_evict_at_budget": (C.c_int, [_P, C.c_int, C.c_double]),
+    "dynts_predictor_mlp_scratch_bytes": (C.c_size_t, [C.c_int, C.c_int]),
+    "dynts_predictor_mlp": (C.c_int, [_P] * 7 + [C.c_int, C.c_int, C.c_int, _P, C.c_size_t, _P, _P]),
     "dynts_evict_stats": (C.c_int, [_P, C.POINTER(C.c_longlong), C.POINTER(C.c_longlong)]),
     "dynts_last_error": (C.c_char_p, []),
     "dynts_version": (C.c_char_p, []),
@@ -254,6 +256,15 @@ def dynts_append_scores(c, s_new):
 
 def dynts_evict_at_budget(c, budget_B, ratio):
     return _check(lib.dynts_evict_at_budget(c, budget_B, ratio))
+
+
+def dynts_predictor_mlp_scratch_bytes(d, batch) -> int:
+    return lib.dynts_predictor_mlp_scratch_bytes(d, batch)
+
+
+def dynts_predictor_mlp(h, W1, b1, W2, b2, W3, b3, d, batch, activation, scratch, scratch_bytes, scores, stream=None):
+    return _check(lib.dynts_predictor_mlp(_ptr(h), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(W3), _ptr(b3), d, batch,
+                                          activation, _ptr(scratch), scratch_bytes, _ptr(scores), stream))
 
 
 def dynts_evict_stats(c):

@@ -19,6 +19,7 @@
 #include "decode_attn.cuh"
 #include "decode_stream.cuh"
 #include "evict.cuh"
+#include "predictor.cuh"
 
 namespace {
 
@@ -902,6 +903,96 @@ dynts_status_t dynts_evict_stats(dynts_cache_t* c, long long* rows_scanned, long
   }
   if (rows_scanned) *rows_scanned = scanned;
   if (rows_moved) *rows_moved = moved;
+  return DYNTS_OK;
+}
+
+/* ---- Importance Predictor head ------------------------------------------------------------ */
+
+}  // extern "C"
+
+namespace {
+
+// K-slices of a layer with `rows` outputs and K inputs: enough CTAs to fill the GPU (about 256),
+// slices that are multiples of 256 elements and fit shared memory for a tile of 8 sequences.
+int mlp_k_slices(int rows, int K) {
+  const int units = K / 256;
+  const int row_blocks = (rows + dynts::kMlpRowsPerCta - 1) / dynts::kMlpRowsPerCta;
+  int best = units;  // finest split as a fallback
+  for (int ks = 1; ks <= units; ++ks) {
+    if (units % ks) continue;
+    if ((size_t)(K / ks) * dynts::kMlpBatchTile * 4 > 160 * 1024) continue;
+    if (row_blocks * ks >= 256) return ks;
+    best = ks;
+  }
+  return best;
+}
+
+bool g_mlp_attr = false;
+
+}  // namespace
+
+extern "C" {
+
+size_t dynts_predictor_mlp_scratch_bytes(int d, int batch) {
+  if (d < 512 || d % 512 || batch < 1) return 0;
+  const size_t p1 = (size_t)mlp_k_slices(2 * d, d) * batch * (2 * d);
+  const size_t p2 = (size_t)mlp_k_slices(d / 2, 2 * d) * batch * (d / 2);
+  return (p1 + p2) * sizeof(float);
+}
+
+dynts_status_t dynts_predictor_mlp(const void* h, const void* W1, const float* b1, const void* W2, const float* b2,
+                                   const void* W3, const float* b3, int d, int batch, int activation, void* scratch,
+                                   size_t scratch_bytes, float* scores, void* stream) {
+  if (!h || !W1 || !W2 || !W3 || !scratch || !scores) return fail(DYNTS_ERR_INVALID_ARG, "NULL tensor pointer");
+  if (!aligned16(h) || !aligned16(W1) || !aligned16(W2) || !aligned16(W3) || !aligned16(scratch))
+    return fail(DYNTS_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+  if (d < 512 || d % 512 || batch < 1) return fail(DYNTS_ERR_INVALID_ARG, "d must be a multiple of 512, batch >= 1");
+  if (activation != 0 && activation != 1) return fail(DYNTS_ERR_INVALID_ARG, "activation must be 0 (none) or 1 (ReLU)");
+  const size_t need = dynts_predictor_mlp_scratch_bytes(d, batch);
+  if (scratch_bytes < need) return fail(DYNTS_ERR_OOM, "scratch too small: %zu < %zu bytes", scratch_bytes, need);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!g_mlp_attr) {
+    CUDA_TRY(cudaFuncSetAttribute(dynts::mlp_layer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+    g_mlp_attr = true;
+  }
+  const int ks1 = mlp_k_slices(2 * d, d), ks2 = mlp_k_slices(d / 2, 2 * d);
+  float* parts1 = static_cast<float*>(scratch);
+  float* parts2 = parts1 + (size_t)ks1 * batch * (2 * d);
+  const unsigned tiles = (unsigned)((batch + dynts::kMlpBatchTile - 1) / dynts::kMlpBatchTile);
+
+  dynts::MlpLayerParams p;
+  p.W = static_cast<const __nv_bfloat16*>(W1);
+  p.xh = static_cast<const __nv_bfloat16*>(h);
+  p.xparts = nullptr;
+  p.xbias = nullptr;
+  p.yparts = parts1;
+  p.rows = 2 * d;
+  p.K = d;
+  p.Nb = batch;
+  p.n_parts = 0;
+  p.act = 0;
+  p.k_slice = d / ks1;
+  size_t smem = (size_t)std::min(batch, dynts::kMlpBatchTile) * p.k_slice * sizeof(float);
+  dynts::mlp_layer_kernel<<<dim3((unsigned)((p.rows + 63) / 64), (unsigned)ks1, tiles), dynts::kMlpThreads, smem, st>>>(p);
+  CUDA_TRY(cudaGetLastError());
+
+  p.W = static_cast<const __nv_bfloat16*>(W2);
+  p.xh = nullptr;
+  p.xparts = parts1;
+  p.xbias = b1;
+  p.yparts = parts2;
+  p.rows = d / 2;
+  p.K = 2 * d;
+  p.n_parts = ks1;
+  p.act = activation;
+  p.k_slice = 2 * d / ks2;
+  smem = (size_t)std::min(batch, dynts::kMlpBatchTile) * p.k_slice * sizeof(float);
+  dynts::mlp_layer_kernel<<<dim3((unsigned)((p.rows + 63) / 64), (unsigned)ks2, tiles), dynts::kMlpThreads, smem, st>>>(p);
+  CUDA_TRY(cudaGetLastError());
+
+  dynts::mlp_head_kernel<<<(unsigned)batch, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(W3), parts2, b2, b3, scores, d / 2,
+                                                        batch, ks2, activation);
+  CUDA_TRY(cudaGetLastError());
   return DYNTS_OK;
 }
 
