@@ -281,6 +281,11 @@ def run_ours(args, cfg, rank, world, device):
                "d2h_bytes_per_step": int(hout.numel() * hout.element_size()), "steps": steps_done,
                "api": "dynts_decode_attn_host + dynts_evict"}
 
+    # ---- Importance Predictor head (Section 4.1): d -> 2d -> d/2 -> 1 at Llama-8B width -----------
+    predictor = None
+    if rank == 0 and world == 1:
+        predictor = time_predictor(cfg.batch, device, peak)
+
     # ---- CPU baseline: the oracle, as it stands, on this machine's host cores (rank 0, N = 1) ------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -296,10 +301,43 @@ def run_ours(args, cfg, rank, world, device):
                    "cache_bytes": cache.nbytes, "l2_policy": "inputs larger than L2 (KV cache %.0f MB vs 126 MB L2)" % (cache.nbytes / 1e6),
                    "replicas": world},
         "hbm_gbs_decode": round(dec_gbs, 1), "roofline": roofline, "evict": evict, "e2e": e2e,
-        "cpu_baseline": cpu, "clocks": clocks, "gpu_launches": int(launches),
+        "predictor_mlp": predictor, "cpu_baseline": cpu, "clocks": clocks, "gpu_launches": int(launches),
     }
     cache.close()
     return result
+
+
+def time_predictor(batch, device, peak, d=4096, iters=40):
+    """Times dynts_predictor_mlp (three launches) on random bf16 weights; two weight sets alternate so
+    that the 101 MB of weights are not served from L2."""
+    import torch
+    import paper_2601_18383_b200 as D
+    g = torch.Generator(device=device).manual_seed(99)
+    mk = lambda *shape: (torch.randn(shape, generator=g, device=device) / shape[-1] ** 0.5).to(torch.bfloat16)
+    sets = [(mk(2 * d, d), mk(d // 2, 2 * d), mk(1, d // 2)) for _ in range(2)]
+    h = torch.randn((batch, d), generator=g, device=device).to(torch.bfloat16)
+    nbytes = D.dynts_predictor_mlp_scratch_bytes(d, batch)
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    scores = torch.empty(batch, dtype=torch.float32, device=device)
+    st = torch.cuda.current_stream(device)
+
+    def run(i):
+        W1, W2, W3 = sets[i % 2]
+        D.dynts_predictor_mlp(h, W1, None, W2, None, W3, None, d, batch, 1, scratch, nbytes, scores, st.cuda_stream)
+
+    for i in range(4):
+        run(i)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(st)
+    for i in range(iters):
+        run(i)
+    b.record(st)
+    torch.cuda.synchronize(device)
+    us = a.elapsed_time(b) * 1e3 / iters
+    wbytes = 2 * (2 * d * d + d * d + d // 2)            # the bf16 weights, read once
+    gbs = wbytes / (us * 1e-6) / 1e9
+    return {"d": d, "batch": batch, "us_per_call": round(us, 2), "weight_bytes": wbytes, "bound": "hbm",
+            "achieved": round(gbs, 1), "peak": peak, "unit": "GB/s", "frac": round(gbs / peak, 4)}
 
 
 def oracle_baseline(cfg, cache, q_ring, k_ring, v_ring, budget_s=20.0, slabs=None):

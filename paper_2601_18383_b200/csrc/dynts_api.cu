@@ -920,7 +920,7 @@ int mlp_k_slices(int rows, int K) {
   int best = units;  // finest split as a fallback
   for (int ks = 1; ks <= units; ++ks) {
     if (units % ks) continue;
-    if ((size_t)(K / ks) * dynts::kMlpBatchTile * 4 > 160 * 1024) continue;
+    if ((size_t)(K / ks) * dynts::kMlpBatchTile * 4 > 100 * 1024) continue;
     if (row_blocks * ks >= 256) return ks;
     best = ks;
   }
@@ -952,13 +952,17 @@ dynts_status_t dynts_predictor_mlp(const void* h, const void* W1, const float* b
   if (scratch_bytes < need) return fail(DYNTS_ERR_OOM, "scratch too small: %zu < %zu bytes", scratch_bytes, need);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (!g_mlp_attr) {
-    CUDA_TRY(cudaFuncSetAttribute(dynts::mlp_layer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+    CUDA_TRY(cudaFuncSetAttribute(dynts::mlp_layer_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+    CUDA_TRY(cudaFuncSetAttribute(dynts::mlp_layer_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+    CUDA_TRY(cudaFuncSetAttribute(dynts::mlp_layer_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+    CUDA_TRY(cudaFuncSetAttribute(dynts::mlp_layer_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
     g_mlp_attr = true;
   }
+  const int NT = batch >= 8 ? 8 : (batch >= 3 ? 4 : batch);  // sequences per batch tile
   const int ks1 = mlp_k_slices(2 * d, d), ks2 = mlp_k_slices(d / 2, 2 * d);
   float* parts1 = static_cast<float*>(scratch);
   float* parts2 = parts1 + (size_t)ks1 * batch * (2 * d);
-  const unsigned tiles = (unsigned)((batch + dynts::kMlpBatchTile - 1) / dynts::kMlpBatchTile);
+  const unsigned tiles = (unsigned)((batch + NT - 1) / NT);
 
   dynts::MlpLayerParams p;
   p.W = static_cast<const __nv_bfloat16*>(W1);
@@ -972,9 +976,18 @@ dynts_status_t dynts_predictor_mlp(const void* h, const void* W1, const float* b
   p.n_parts = 0;
   p.act = 0;
   p.k_slice = d / ks1;
-  size_t smem = (size_t)std::min(batch, dynts::kMlpBatchTile) * p.k_slice * sizeof(float);
-  dynts::mlp_layer_kernel<<<dim3((unsigned)((p.rows + 63) / 64), (unsigned)ks1, tiles), dynts::kMlpThreads, smem, st>>>(p);
-  CUDA_TRY(cudaGetLastError());
+  auto launch_layer = [&](const dynts::MlpLayerParams& q, int ks) -> cudaError_t {
+    const size_t smem = (size_t)NT * q.k_slice * sizeof(float);
+    const dim3 grid(tiles, (unsigned)((q.rows + 63) / 64), (unsigned)ks);
+    switch (NT) {
+      case 1: dynts::mlp_layer_kernel<1><<<grid, dynts::kMlpThreads, smem, st>>>(q); break;
+      case 2: dynts::mlp_layer_kernel<2><<<grid, dynts::kMlpThreads, smem, st>>>(q); break;
+      case 4: dynts::mlp_layer_kernel<4><<<grid, dynts::kMlpThreads, smem, st>>>(q); break;
+      default: dynts::mlp_layer_kernel<8><<<grid, dynts::kMlpThreads, smem, st>>>(q); break;
+    }
+    return cudaGetLastError();
+  };
+  CUDA_TRY(launch_layer(p, ks1));
 
   p.W = static_cast<const __nv_bfloat16*>(W2);
   p.xh = nullptr;
@@ -986,9 +999,7 @@ dynts_status_t dynts_predictor_mlp(const void* h, const void* W1, const float* b
   p.n_parts = ks1;
   p.act = activation;
   p.k_slice = 2 * d / ks2;
-  smem = (size_t)std::min(batch, dynts::kMlpBatchTile) * p.k_slice * sizeof(float);
-  dynts::mlp_layer_kernel<<<dim3((unsigned)((p.rows + 63) / 64), (unsigned)ks2, tiles), dynts::kMlpThreads, smem, st>>>(p);
-  CUDA_TRY(cudaGetLastError());
+  CUDA_TRY(launch_layer(p, ks2));
 
   dynts::mlp_head_kernel<<<(unsigned)batch, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(W3), parts2, b2, b3, scores, d / 2,
                                                         batch, ks2, activation);

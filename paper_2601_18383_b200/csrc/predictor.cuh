@@ -5,7 +5,7 @@
 // is shaped into a GEMM.
 //
 //   mlp_layer_kernel   y_part[ks][n][r] = sum over the K-slice ks of W[r][k] * x[n][k].
-//                      grid = (row blocks of 64, K slices, batch tiles); 8 warps x 8 rows.  The
+//                      grid = (batch tiles, row blocks of 64, K slices); 8 warps x 8 rows.  The
 //                      input slice of the batch tile sits in shared memory as fp32.  The input is
 //                      either the bf16 hidden state, or the previous layer's partial sums, which
 //                      are reduced (fixed order), biased and activated while they are loaded -- so
@@ -33,72 +33,114 @@ struct MlpLayerParams {
 
 __device__ __forceinline__ float mlp_act(float x, int act) { return act == 1 ? fmaxf(x, 0.f) : x; }
 
-__global__ void __launch_bounds__(kMlpThreads) mlp_layer_kernel(const MlpLayerParams p) {
+// NT = sequences of the batch tile (1, 2, 4 or 8): the accumulators are [8 rows][NT] registers.
+// grid = (batch tiles, row blocks, K slices): the tiles of one weight block run side by side and
+// share its lines in L2.
+template <int NT>
+__global__ void __launch_bounds__(kMlpThreads, NT >= 4 ? 1 : 2) mlp_layer_kernel(const MlpLayerParams p) {
   extern __shared__ __align__(16) float sx[];  // [tile sequences][k_slice]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int ks = blockIdx.y;
-  const int n0 = blockIdx.z * kMlpBatchTile;
-  const int nt = min(kMlpBatchTile, p.Nb - n0);
+  const int ks = blockIdx.z;
+  const int n0 = blockIdx.x * NT;
+  const int nt = min(NT, p.Nb - n0);
   const int k0 = ks * p.k_slice;
+  const int r0 = blockIdx.y * kMlpRowsPerCta + warp * kMlpRowsPerWarp;
+  const int n_chunks = p.k_slice >> 3;  // 16-byte pieces of a row's K-slice; lane owns lane, lane + 32, ...
 
-  // input slice -> shared memory (fp32)
-  for (int e = tid; e < nt * p.k_slice; e += kMlpThreads) {
-    const int n = e / p.k_slice, k = e - n * p.k_slice;
-    float v;
-    if (p.xh) {
-      v = __bfloat162float(p.xh[(size_t)(n0 + n) * p.K + k0 + k]);
-    } else {
-      v = 0.f;
-      for (int q = 0; q < p.n_parts; ++q) v += p.xparts[((size_t)q * p.Nb + n0 + n) * p.K + k0 + k];
-      if (p.xbias) v += p.xbias[k0 + k];
-      v = mlp_act(v, p.act);
-    }
-    sx[e] = v;
-  }
-  __syncthreads();
-
-  const int r0 = blockIdx.x * kMlpRowsPerCta + warp * kMlpRowsPerWarp;
-  float acc[kMlpRowsPerWarp][kMlpBatchTile];
-#pragma unroll
-  for (int r = 0; r < kMlpRowsPerWarp; ++r)
-#pragma unroll
-    for (int n = 0; n < kMlpBatchTile; ++n) acc[r][n] = 0.f;
-
-  // lane owns the 16-byte pieces lane, lane + 32, ... of the K-slice
-  for (int c = lane; c * 8 < p.k_slice; c += 32) {
-    uint4 w[kMlpRowsPerWarp];
+  auto load_w = [&](uint4 (&w)[kMlpRowsPerWarp], int c) {
 #pragma unroll
     for (int r = 0; r < kMlpRowsPerWarp; ++r) {
       const int row = min(r0 + r, p.rows - 1);  // clamped: rows past the end are computed and dropped
       w[r] = ldg_stream(p.W + (size_t)row * p.K + k0 + c * 8);
     }
+  };
+  // The first weight pieces are requested before the input slice is staged: their latency overlaps it.
+  uint4 wa[kMlpRowsPerWarp], wb[kMlpRowsPerWarp];
+  if (lane < n_chunks) load_w(wa, lane);
+  if (lane + 32 < n_chunks) load_w(wb, lane + 32);
+
+  // input slice -> shared memory (fp32), eight elements per thread and step.  Piece c of sequence n
+  // is stored as two float4: sxa[n * n_chunks + c] (elements 0-3) and sxb[...] (elements 4-7), so that
+  // the lanes of a warp, which own consecutive pieces, read consecutive 16-byte words.  Sequences
+  // past the end of the batch are zero.
+  float4* sxa = reinterpret_cast<float4*>(sx);
+  float4* sxb = sxa + (size_t)NT * n_chunks;
+#pragma unroll 2
+  for (int g = tid; g < NT * n_chunks; g += kMlpThreads) {
+    const int n = g / n_chunks, c = g - n * n_chunks;
+    float v[8];
 #pragma unroll
-    for (int n = 0; n < kMlpBatchTile; ++n) {
-      if (n < nt) {
-        const float4 xa = *reinterpret_cast<const float4*>(sx + (size_t)n * p.k_slice + c * 8);
-        const float4 xb = *reinterpret_cast<const float4*>(sx + (size_t)n * p.k_slice + c * 8 + 4);
-#pragma unroll
-        for (int r = 0; r < kMlpRowsPerWarp; ++r) {
-          // a bf16 is the upper half of an fp32
-          float a = acc[r][n];
-          a = fmaf(__uint_as_float(w[r].x << 16), xa.x, a);
-          a = fmaf(__uint_as_float(w[r].x & 0xffff0000u), xa.y, a);
-          a = fmaf(__uint_as_float(w[r].y << 16), xa.z, a);
-          a = fmaf(__uint_as_float(w[r].y & 0xffff0000u), xa.w, a);
-          a = fmaf(__uint_as_float(w[r].z << 16), xb.x, a);
-          a = fmaf(__uint_as_float(w[r].z & 0xffff0000u), xb.y, a);
-          a = fmaf(__uint_as_float(w[r].w << 16), xb.z, a);
-          a = fmaf(__uint_as_float(w[r].w & 0xffff0000u), xb.w, a);
-          acc[r][n] = a;
+    for (int i = 0; i < 8; ++i) v[i] = 0.f;
+    if (n < nt) {
+      const size_t off = (size_t)(n0 + n) * p.K + k0 + c * 8;
+      if (p.xh) {
+        const uint4 w = *reinterpret_cast<const uint4*>(p.xh + off);
+        v[0] = __uint_as_float(w.x << 16); v[1] = __uint_as_float(w.x & 0xffff0000u);
+        v[2] = __uint_as_float(w.y << 16); v[3] = __uint_as_float(w.y & 0xffff0000u);
+        v[4] = __uint_as_float(w.z << 16); v[5] = __uint_as_float(w.z & 0xffff0000u);
+        v[6] = __uint_as_float(w.w << 16); v[7] = __uint_as_float(w.w & 0xffff0000u);
+      } else {
+        for (int q = 0; q < p.n_parts; ++q) {
+          const float4 a4 = *reinterpret_cast<const float4*>(p.xparts + (size_t)q * p.Nb * p.K + off);
+          const float4 b4 = *reinterpret_cast<const float4*>(p.xparts + (size_t)q * p.Nb * p.K + off + 4);
+          v[0] += a4.x; v[1] += a4.y; v[2] += a4.z; v[3] += a4.w;
+          v[4] += b4.x; v[5] += b4.y; v[6] += b4.z; v[7] += b4.w;
         }
+        if (p.xbias) {
+          const float4 a4 = *reinterpret_cast<const float4*>(p.xbias + k0 + c * 8);
+          const float4 b4 = *reinterpret_cast<const float4*>(p.xbias + k0 + c * 8 + 4);
+          v[0] += a4.x; v[1] += a4.y; v[2] += a4.z; v[3] += a4.w;
+          v[4] += b4.x; v[5] += b4.y; v[6] += b4.z; v[7] += b4.w;
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = mlp_act(v[i], p.act);
       }
+    }
+    sxa[g] = make_float4(v[0], v[1], v[2], v[3]);
+    sxb[g] = make_float4(v[4], v[5], v[6], v[7]);
+  }
+  __syncthreads();
+
+  float acc[kMlpRowsPerWarp][NT];
+#pragma unroll
+  for (int r = 0; r < kMlpRowsPerWarp; ++r)
+#pragma unroll
+    for (int n = 0; n < NT; ++n) acc[r][n] = 0.f;
+
+  auto fma_chunk = [&](const uint4 (&w)[kMlpRowsPerWarp], int c) {
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+      const float4 xa = sxa[n * n_chunks + c];
+      const float4 xb = sxb[n * n_chunks + c];
+#pragma unroll
+      for (int r = 0; r < kMlpRowsPerWarp; ++r) {
+        float a = acc[r][n];  // a bf16 is the upper half of an fp32
+        a = fmaf(__uint_as_float(w[r].x << 16), xa.x, a);
+        a = fmaf(__uint_as_float(w[r].x & 0xffff0000u), xa.y, a);
+        a = fmaf(__uint_as_float(w[r].y << 16), xa.z, a);
+        a = fmaf(__uint_as_float(w[r].y & 0xffff0000u), xa.w, a);
+        a = fmaf(__uint_as_float(w[r].z << 16), xb.x, a);
+        a = fmaf(__uint_as_float(w[r].z & 0xffff0000u), xb.y, a);
+        a = fmaf(__uint_as_float(w[r].w << 16), xb.z, a);
+        a = fmaf(__uint_as_float(w[r].w & 0xffff0000u), xb.w, a);
+        acc[r][n] = a;
+      }
+    }
+  };
+  // two pieces per row in flight per lane: compute one while the one after next is fetched
+  for (int c = lane; c < n_chunks; c += 64) {
+    fma_chunk(wa, c);
+    if (c + 64 < n_chunks) load_w(wa, c + 64);
+    if (c + 32 < n_chunks) {
+      fma_chunk(wb, c + 32);
+      if (c + 96 < n_chunks) load_w(wb, c + 96);
     }
   }
   // reduce over the lanes; lane 0 writes
 #pragma unroll
   for (int r = 0; r < kMlpRowsPerWarp; ++r) {
 #pragma unroll
-    for (int n = 0; n < kMlpBatchTile; ++n) {
+    for (int n = 0; n < NT; ++n) {
       float a = acc[r][n];
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
