@@ -913,14 +913,15 @@ dynts_status_t dynts_evict_stats(dynts_cache_t* c, long long* rows_scanned, long
 namespace {
 
 // K-slices of a layer with `rows` outputs and K inputs: enough CTAs to fill the GPU (about 256),
-// slices that are multiples of 256 elements and fit shared memory for a tile of 8 sequences.
+// slices that are multiples of 256 elements and fit shared memory (bf16 hi and lo halves of a tile of 16
+// sequences, several CTAs per SM).
 int mlp_k_slices(int rows, int K) {
   const int units = K / 256;
   const int row_blocks = (rows + dynts::kMlpRowsPerCta - 1) / dynts::kMlpRowsPerCta;
   int best = units;  // finest split as a fallback
   for (int ks = 1; ks <= units; ++ks) {
     if (units % ks) continue;
-    if ((size_t)(K / ks) * dynts::kMlpBatchTile * 4 > 100 * 1024) continue;
+    if ((size_t)(K / ks + dynts::kMlpPad) * dynts::kMlpBatchTile * 4 > 72 * 1024) continue;
     if (row_blocks * ks >= 256) return ks;
     best = ks;
   }
@@ -952,13 +953,11 @@ dynts_status_t dynts_predictor_mlp(const void* h, const void* W1, const float* b
   if (scratch_bytes < need) return fail(DYNTS_ERR_OOM, "scratch too small: %zu < %zu bytes", scratch_bytes, need);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (!g_mlp_attr) {
-    CUDA_TRY(cudaFuncSetAttribute(dynts::mlp_layer_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
-    CUDA_TRY(cudaFuncSetAttribute(dynts::mlp_layer_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
-    CUDA_TRY(cudaFuncSetAttribute(dynts::mlp_layer_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
-    CUDA_TRY(cudaFuncSetAttribute(dynts::mlp_layer_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+    CUDA_TRY(cudaFuncSetAttribute(dynts::mlp_layer_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024));
+    CUDA_TRY(cudaFuncSetAttribute(dynts::mlp_layer_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024));
     g_mlp_attr = true;
   }
-  const int NT = batch >= 8 ? 8 : (batch >= 3 ? 4 : batch);  // sequences per batch tile
+  const int NT = batch > 8 ? 16 : 8;  // sequences per batch tile
   const int ks1 = mlp_k_slices(2 * d, d), ks2 = mlp_k_slices(d / 2, 2 * d);
   float* parts1 = static_cast<float*>(scratch);
   float* parts2 = parts1 + (size_t)ks1 * batch * (2 * d);
@@ -977,15 +976,21 @@ dynts_status_t dynts_predictor_mlp(const void* h, const void* W1, const float* b
   p.act = 0;
   p.k_slice = d / ks1;
   auto launch_layer = [&](const dynts::MlpLayerParams& q, int ks) -> cudaError_t {
-    const size_t smem = (size_t)NT * q.k_slice * sizeof(float);
+    const size_t smem = (size_t)2 * NT * (q.k_slice + dynts::kMlpPad) * 2;
     const dim3 grid(tiles, (unsigned)((q.rows + 63) / 64), (unsigned)ks);
-    switch (NT) {
-      case 1: dynts::mlp_layer_kernel<1><<<grid, dynts::kMlpThreads, smem, st>>>(q); break;
-      case 2: dynts::mlp_layer_kernel<2><<<grid, dynts::kMlpThreads, smem, st>>>(q); break;
-      case 4: dynts::mlp_layer_kernel<4><<<grid, dynts::kMlpThreads, smem, st>>>(q); break;
-      default: dynts::mlp_layer_kernel<8><<<grid, dynts::kMlpThreads, smem, st>>>(q); break;
-    }
-    return cudaGetLastError();
+    cudaLaunchConfig_t lc;
+    memset(&lc, 0, sizeof(lc));
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see griddepcontrol.wait in the kernel
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at;
+    lc.numAttrs = 1;
+    lc.stream = st;
+    lc.gridDim = grid;
+    lc.blockDim = dim3(dynts::kMlpWarps * 32, 1, 1);
+    lc.dynamicSmemBytes = smem;
+    if (NT == 8) return cudaLaunchKernelEx(&lc, dynts::mlp_layer_kernel<1>, q);
+    return cudaLaunchKernelEx(&lc, dynts::mlp_layer_kernel<2>, q);
   };
   CUDA_TRY(launch_layer(p, ks1));
 
@@ -1001,9 +1006,20 @@ dynts_status_t dynts_predictor_mlp(const void* h, const void* W1, const float* b
   p.k_slice = 2 * d / ks2;
   CUDA_TRY(launch_layer(p, ks2));
 
-  dynts::mlp_head_kernel<<<(unsigned)batch, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(W3), parts2, b2, b3, scores, d / 2,
-                                                        batch, ks2, activation);
-  CUDA_TRY(cudaGetLastError());
+  {
+    cudaLaunchConfig_t lc;
+    memset(&lc, 0, sizeof(lc));
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at;
+    lc.numAttrs = 1;
+    lc.stream = st;
+    lc.gridDim = dim3((unsigned)batch, 1, 1);
+    lc.blockDim = dim3(256, 1, 1);
+    CUDA_TRY(cudaLaunchKernelEx(&lc, dynts::mlp_head_kernel, static_cast<const __nv_bfloat16*>(W3), (const float*)parts2, b2, b3,
+                                scores, d / 2, batch, ks2, activation));
+  }
   return DYNTS_OK;
 }
 

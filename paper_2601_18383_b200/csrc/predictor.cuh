@@ -1,12 +1,11 @@
 // Importance Predictor head (Section 4.1, Eq. 7; Appendix A): a three-layer MLP d -> 2d -> d/2 -> 1
 // on the final hidden state of each sequence.  With a decode batch of a few sequences every layer
-// is a matrix-vector product bound by reading its bf16 weights once (6 d^2 bytes in all), so the
-// kernels stream weight rows with 16-byte loads and do the arithmetic as fp32 FMAs; nothing here
-// is shaped into a GEMM.
+// is bound by reading its bf16 weights once (6 d^2 bytes in all): the kernels stream weight rows
+// with 16-byte loads straight into tensor-core fragments; the activations wait in shared memory.
 //
 //   mlp_layer_kernel   y_part[ks][n][r] = sum over the K-slice ks of W[r][k] * x[n][k].
-//                      grid = (batch tiles, row blocks of 64, K slices); 8 warps x 8 rows.  The
-//                      input slice of the batch tile sits in shared memory as fp32.  The input is
+//                      grid = (batch tiles, row blocks of 64, K slices); 4 warps x 16 rows.  The
+//                      input slice of the batch tile sits in shared memory as bf16.  The input is
 //                      either the bf16 hidden state, or the previous layer's partial sums, which
 //                      are reduced (fixed order), biased and activated while they are loaded -- so
 //                      a layer split over K needs no reduction pass and no atomics.
@@ -17,10 +16,8 @@
 
 namespace dynts {
 
-constexpr int kMlpThreads = 256;
-constexpr int kMlpRowsPerWarp = 8;
-constexpr int kMlpRowsPerCta = (kMlpThreads / 32) * kMlpRowsPerWarp;  // 64
-constexpr int kMlpBatchTile = 8;
+constexpr int kMlpRowsPerCta = 64;
+constexpr int kMlpBatchTile = 16;  // at most; 8 for batches up to 8
 
 struct MlpLayerParams {
   const __nv_bfloat16* W;   // [rows][K] row-major
@@ -33,53 +30,75 @@ struct MlpLayerParams {
 
 __device__ __forceinline__ float mlp_act(float x, int act) { return act == 1 ? fmaxf(x, 0.f) : x; }
 
-// NT = sequences of the batch tile (1, 2, 4 or 8): the accumulators are [8 rows][NT] registers.
-// grid = (batch tiles, row blocks, K slices): the tiles of one weight block run side by side and
-// share its lines in L2.
-template <int NT>
-__global__ void __launch_bounds__(kMlpThreads, NT >= 4 ? 1 : 2) mlp_layer_kernel(const MlpLayerParams p) {
-  extern __shared__ __align__(16) float sx[];  // [tile sequences][k_slice]
+// NB = blocks of 8 sequences per batch tile (1 or 2).  grid = (batch tiles, row blocks of 64, K
+// slices): the tiles of one weight block run side by side and share its lines in L2.  4 warps, each
+// 16 weight rows.
+//
+// The products run on the tensor pipe (mma.sync m16n8k16, bf16 x bf16 -> fp32): A = 16 weight rows,
+// loaded from global memory straight into fragment registers as 16-byte pieces (a dot product does
+// not care in which order k is summed, so the 8 consecutive elements a thread loads are declared
+// to be its fragment's k-indices and the activations are read with the same permutation);
+// B = the activations of 8 sequences.  fp32 activations are split into two bf16 halves, x = hi + lo
+// with lo = bf16(x - hi), and multiplied in two mma, which keeps about 16 bits of x; a bf16 input
+// (the hidden state) needs one.
+constexpr int kMlpWarps = 4;
+constexpr int kMlpPad = 32;  // bf16 elements of padding per staged sequence: rows land in different banks
+
+__device__ __forceinline__ void mlp_mma(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                        uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int NB>
+__global__ void __launch_bounds__(kMlpWarps * 32) mlp_layer_kernel(const MlpLayerParams p) {
+  extern __shared__ __align__(16) __nv_bfloat16 sxh[];  // [8 NB sequences][k_slice + pad] hi, then the same for lo
+  constexpr int NT = 8 * NB;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int gid = lane >> 2, tig = lane & 3;
   const int ks = blockIdx.z;
   const int n0 = blockIdx.x * NT;
   const int nt = min(NT, p.Nb - n0);
   const int k0 = ks * p.k_slice;
-  const int r0 = blockIdx.y * kMlpRowsPerCta + warp * kMlpRowsPerWarp;
-  const int n_chunks = p.k_slice >> 3;  // 16-byte pieces of a row's K-slice; lane owns lane, lane + 32, ...
+  const int r0 = blockIdx.y * kMlpRowsPerCta + warp * 16;
+  const int n_chunks = p.k_slice >> 3;   // 16-byte pieces of a row's K-slice
+  const int stride = p.k_slice + kMlpPad;  // staged row length in elements
+  __nv_bfloat16* sxl = sxh + (size_t)NT * stride;
+  const bool split = p.xh == nullptr;    // fp32 input: hi + lo
 
-  auto load_w = [&](uint4 (&w)[kMlpRowsPerWarp], int c) {
+  const __nv_bfloat16* wrow0 = p.W + (size_t)min(r0 + gid, p.rows - 1) * p.K + k0;      // clamped rows are computed
+  const __nv_bfloat16* wrow1 = p.W + (size_t)min(r0 + gid + 8, p.rows - 1) * p.K + k0;  // and dropped
+  // Thread (gid, tig) owns the pieces tig + 4i of rows gid and gid + 8; a group of 4 i is one step.
+  auto load_w = [&](uint4 (&w)[8], int step) {
 #pragma unroll
-    for (int r = 0; r < kMlpRowsPerWarp; ++r) {
-      const int row = min(r0 + r, p.rows - 1);  // clamped: rows past the end are computed and dropped
-      w[r] = ldg_stream(p.W + (size_t)row * p.K + k0 + c * 8);
+    for (int i = 0; i < 4; ++i) {
+      const int c = 16 * step + tig + 4 * i;
+      w[2 * i] = ldg_stream(wrow0 + c * 8);
+      w[2 * i + 1] = ldg_stream(wrow1 + c * 8);
     }
   };
-  // The first weight pieces are requested before the input slice is staged: their latency overlaps it.
-  uint4 wa[kMlpRowsPerWarp], wb[kMlpRowsPerWarp];
-  if (lane < n_chunks) load_w(wa, lane);
-  if (lane + 32 < n_chunks) load_w(wb, lane + 32);
+  const int n_steps = n_chunks >> 4;  // k_slice is a multiple of 256 = 16 pieces x 2 ... host guarantees 128 | k_slice
+  uint4 wa[8], wb[8];
+  load_w(wa, 0);
+  if (n_steps > 1) load_w(wb, 1);
+  // The weights do not depend on the kernel before this one in the stream; the activations do.
+  // (launched with programmatic stream serialisation)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
-  // input slice -> shared memory (fp32), eight elements per thread and step.  Piece c of sequence n
-  // is stored as two float4: sxa[n * n_chunks + c] (elements 0-3) and sxb[...] (elements 4-7), so that
-  // the lanes of a warp, which own consecutive pieces, read consecutive 16-byte words.  Sequences
-  // past the end of the batch are zero.
-  float4* sxa = reinterpret_cast<float4*>(sx);
-  float4* sxb = sxa + (size_t)NT * n_chunks;
-#pragma unroll 2
-  for (int g = tid; g < NT * n_chunks; g += kMlpThreads) {
+  // stage the input slice: 8 elements per thread and step
+  for (int g = tid; g < NT * n_chunks; g += kMlpWarps * 32) {
     const int n = g / n_chunks, c = g - n * n_chunks;
-    float v[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = 0.f;
+    uint4 hi = make_uint4(0u, 0u, 0u, 0u), lo = hi;
     if (n < nt) {
       const size_t off = (size_t)(n0 + n) * p.K + k0 + c * 8;
-      if (p.xh) {
-        const uint4 w = *reinterpret_cast<const uint4*>(p.xh + off);
-        v[0] = __uint_as_float(w.x << 16); v[1] = __uint_as_float(w.x & 0xffff0000u);
-        v[2] = __uint_as_float(w.y << 16); v[3] = __uint_as_float(w.y & 0xffff0000u);
-        v[4] = __uint_as_float(w.z << 16); v[5] = __uint_as_float(w.z & 0xffff0000u);
-        v[6] = __uint_as_float(w.w << 16); v[7] = __uint_as_float(w.w & 0xffff0000u);
+      if (!split) {
+        hi = *reinterpret_cast<const uint4*>(p.xh + off);
       } else {
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = 0.f;
         for (int q = 0; q < p.n_parts; ++q) {
           const float4 a4 = *reinterpret_cast<const float4*>(p.xparts + (size_t)q * p.Nb * p.K + off);
           const float4 b4 = *reinterpret_cast<const float4*>(p.xparts + (size_t)q * p.Nb * p.K + off + 4);
@@ -92,59 +111,64 @@ __global__ void __launch_bounds__(kMlpThreads, NT >= 4 ? 1 : 2) mlp_layer_kernel
           v[0] += a4.x; v[1] += a4.y; v[2] += a4.z; v[3] += a4.w;
           v[4] += b4.x; v[5] += b4.y; v[6] += b4.z; v[7] += b4.w;
         }
+        uint32_t hw[4], lw[4];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = mlp_act(v[i], p.act);
+        for (int i = 0; i < 4; ++i) {
+          const float x0 = mlp_act(v[2 * i], p.act), x1 = mlp_act(v[2 * i + 1], p.act);
+          const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
+          const __nv_bfloat16 l0 = __float2bfloat16_rn(x0 - __bfloat162float(h0));
+          const __nv_bfloat16 l1 = __float2bfloat16_rn(x1 - __bfloat162float(h1));
+          hw[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+          lw[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+        }
+        hi = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+        lo = make_uint4(lw[0], lw[1], lw[2], lw[3]);
       }
     }
-    sxa[g] = make_float4(v[0], v[1], v[2], v[3]);
-    sxb[g] = make_float4(v[4], v[5], v[6], v[7]);
+    *reinterpret_cast<uint4*>(sxh + (size_t)n * stride + c * 8) = hi;
+    if (split) *reinterpret_cast<uint4*>(sxl + (size_t)n * stride + c * 8) = lo;
   }
   __syncthreads();
 
-  float acc[kMlpRowsPerWarp][NT];
+  float acc[NB][4];
 #pragma unroll
-  for (int r = 0; r < kMlpRowsPerWarp; ++r)
+  for (int b = 0; b < NB; ++b)
 #pragma unroll
-    for (int n = 0; n < NT; ++n) acc[r][n] = 0.f;
+    for (int e = 0; e < 4; ++e) acc[b][e] = 0.f;
 
-  auto fma_chunk = [&](const uint4 (&w)[kMlpRowsPerWarp], int c) {
+  auto mma_step = [&](const uint4 (&w)[8], int step) {
 #pragma unroll
-    for (int n = 0; n < NT; ++n) {
-      const float4 xa = sxa[n * n_chunks + c];
-      const float4 xb = sxb[n * n_chunks + c];
+    for (int i = 0; i < 4; ++i) {
+      const int c = 16 * step + tig + 4 * i;
 #pragma unroll
-      for (int r = 0; r < kMlpRowsPerWarp; ++r) {
-        float a = acc[r][n];  // a bf16 is the upper half of an fp32
-        a = fmaf(__uint_as_float(w[r].x << 16), xa.x, a);
-        a = fmaf(__uint_as_float(w[r].x & 0xffff0000u), xa.y, a);
-        a = fmaf(__uint_as_float(w[r].y << 16), xa.z, a);
-        a = fmaf(__uint_as_float(w[r].y & 0xffff0000u), xa.w, a);
-        a = fmaf(__uint_as_float(w[r].z << 16), xb.x, a);
-        a = fmaf(__uint_as_float(w[r].z & 0xffff0000u), xb.y, a);
-        a = fmaf(__uint_as_float(w[r].w << 16), xb.z, a);
-        a = fmaf(__uint_as_float(w[r].w & 0xffff0000u), xb.w, a);
-        acc[r][n] = a;
+      for (int b = 0; b < NB; ++b) {
+        const uint4 xh4 = *reinterpret_cast<const uint4*>(sxh + (size_t)(8 * b + gid) * stride + c * 8);
+        mlp_mma(acc[b], w[2 * i].x, w[2 * i + 1].x, w[2 * i].y, w[2 * i + 1].y, xh4.x, xh4.y);
+        mlp_mma(acc[b], w[2 * i].z, w[2 * i + 1].z, w[2 * i].w, w[2 * i + 1].w, xh4.z, xh4.w);
+        if (split) {
+          const uint4 xl4 = *reinterpret_cast<const uint4*>(sxl + (size_t)(8 * b + gid) * stride + c * 8);
+          mlp_mma(acc[b], w[2 * i].x, w[2 * i + 1].x, w[2 * i].y, w[2 * i + 1].y, xl4.x, xl4.y);
+          mlp_mma(acc[b], w[2 * i].z, w[2 * i + 1].z, w[2 * i].w, w[2 * i + 1].w, xl4.z, xl4.w);
+        }
       }
     }
   };
-  // two pieces per row in flight per lane: compute one while the one after next is fetched
-  for (int c = lane; c < n_chunks; c += 64) {
-    fma_chunk(wa, c);
-    if (c + 64 < n_chunks) load_w(wa, c + 64);
-    if (c + 32 < n_chunks) {
-      fma_chunk(wb, c + 32);
-      if (c + 96 < n_chunks) load_w(wb, c + 96);
+  // two steps (2 x 8 pieces of 16 bytes per thread) in flight
+  for (int st = 0; st < n_steps; st += 2) {
+    mma_step(wa, st);
+    if (st + 2 < n_steps) load_w(wa, st + 2);
+    if (st + 1 < n_steps) {
+      mma_step(wb, st + 1);
+      if (st + 3 < n_steps) load_w(wb, st + 3);
     }
   }
-  // reduce over the lanes; lane 0 writes
+  // accumulator: rows gid (c0, c1) and gid + 8 (c2, c3), sequences 2 tig and 2 tig + 1 of the block
 #pragma unroll
-  for (int r = 0; r < kMlpRowsPerWarp; ++r) {
+  for (int b = 0; b < NB; ++b) {
 #pragma unroll
-    for (int n = 0; n < NT; ++n) {
-      float a = acc[r][n];
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-      if (lane == 0 && n < nt && r0 + r < p.rows) p.yparts[((size_t)ks * p.Nb + n0 + n) * p.rows + r0 + r] = a;
+    for (int e = 0; e < 4; ++e) {
+      const int row = r0 + gid + (e >> 1) * 8, n = 8 * b + 2 * tig + (e & 1);
+      if (row < p.rows && n < nt) p.yparts[((size_t)ks * p.Nb + n0 + n) * p.rows + row] = acc[b][e];
     }
   }
 }
@@ -154,6 +178,7 @@ __global__ void __launch_bounds__(256) mlp_head_kernel(const __nv_bfloat16* W3, 
                                                        const float* b3, float* scores, int K, int Nb, int n_parts, int act) {
   const int n = blockIdx.x, tid = threadIdx.x;
   __shared__ float red[8];
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   float a = 0.f;
   for (int k = tid; k < K; k += 256) {
     float v = 0.f;
