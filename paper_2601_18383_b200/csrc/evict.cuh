@@ -296,9 +296,17 @@ __global__ void __launch_bounds__(kFusedThreads) evict_fused_kernel(const EvictP
         __syncthreads();
         const uint32_t prefix = s_prefix;
         const int krem = s_krem;
-        for (int j = lo + tid; j < hi; j += kFusedThreads) {
-          const uint32_t key = order_key(sel[j]);
-          if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        // Scores of one slab mostly share their top bits, so most rows fall into one bin: the lanes
+        // of a warp that hit the same bin add their count with a single atomic.
+        for (int base = lo; base < hi; base += kFusedThreads) {
+          const int j = base + tid;
+          uint32_t bin = 0x100u;  // "no vote"
+          if (j < hi) {
+            const uint32_t key = order_key(sel[j]);
+            if ((key & mask) == prefix) bin = (key >> shift) & 255u;
+          }
+          const unsigned peers = __match_any_sync(0xffffffffu, bin);
+          if (bin < 0x100u && (int)(threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[bin], (unsigned)__popc(peers));
         }
         __syncthreads();
         if (tid < 32) {
