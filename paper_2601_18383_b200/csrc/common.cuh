@@ -96,25 +96,27 @@ __device__ __forceinline__ void kahan_add(float& s, float& c, float x) {
 
 // The last CTA of the grid to finish advances the per-sequence lengths: every other CTA has
 // read them before taking its ticket, so the update cannot race with a read of this launch.
-__device__ __forceinline__ void finish_ticket(const DecodeParams& p) {
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    // (this CTA's reads of the lengths returned their values long ago; no fence is needed to
-    // order them before the ticket)
-    unsigned int t = atomicAdd(p.ticket, 1u);
-    if (t == gridDim.x - 1) {
-      *p.ticket = 0u;
-      if (p.advance) {
-        for (int b = 0; b < p.Nb; ++b) {
-          if (p.active[b]) {
-            p.len[b] += 1;
-            p.tot[b] += 1;
-          }
+__device__ __forceinline__ void take_ticket(const DecodeParams& p) {  // one thread per CTA
+  // (this CTA's reads of the lengths returned their values long ago; no fence is needed to
+  // order them before the ticket)
+  unsigned int t = atomicAdd(p.ticket, 1u);
+  if (t == gridDim.x - 1) {
+    *p.ticket = 0u;
+    if (p.advance) {
+      for (int b = 0; b < p.Nb; ++b) {
+        if (p.active[b]) {
+          p.len[b] += 1;
+          p.tot[b] += 1;
         }
       }
-      __threadfence();
     }
+    __threadfence();
   }
+}
+
+__device__ __forceinline__ void finish_ticket(const DecodeParams& p) {
+  __syncthreads();
+  if (threadIdx.x == 0) take_ticket(p);
 }
 
 }  // namespace dynts

@@ -341,6 +341,10 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
   // The launch may overlap the tail of the kernel before it in the stream (programmatic dependent
   // launch): nothing above touches global memory; everything below waits until that kernel has
   // completed and its writes are visible.
+  if (tid == 32) {  // the descriptors are kernel parameters: fetching them needs no earlier kernel
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmK)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmV)) : "memory");
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (warp == 1) {
     int carry = 0, cmin = 0x7fffffff, cmax = 0;
