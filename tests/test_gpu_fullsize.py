@@ -140,3 +140,71 @@ def test_config5_attention_shapes_layer_by_layer():
     assert gpu.len(7) == cfg.budget
     gpu.close()
     torch.cuda.empty_cache()
+
+
+def test_full_kv_length_slabs_and_two_kernel_eviction():
+    """The longest slabs the configurations name (full KV of the 16384-token decode: 16640 rows):
+    the streaming kernel spreads every slab over many CTAs, and the eviction takes the two-kernel
+    path (gather list in global memory) because such a slab does not fit the fused kernel."""
+    cfg = W.get_config("c2_llama8b").scaled(name="full_kv", layers=2, batch=2, budget=16640, window=128, evict_interval=64,
+                                             prompt=256, density=0.01)
+    gpu = _steady_state(cfg, 6100, 16640 - 2)
+    slabs = [(0, 0, 0), (1, 1, 7), (0, 1, 3)]
+    worst = _check_sampled(gpu, cfg, 6100, slabs, steps=2)
+    assert worst["out"] <= H.TOL_OUT["bf16"] and worst["delta"] <= H.TOL_DELTA, worst
+    assert gpu.len(0) == 16640
+    H.check_evict_bit_exact(gpu, cfg, 12000, slabs=slabs)
+    assert gpu.len(1) == 12000
+    worst = _check_sampled(gpu, cfg, 6101, slabs, steps=1)
+    assert worst["out"] <= H.TOL_OUT["bf16"] and worst["delta"] <= H.TOL_DELTA, worst
+    gpu.close()
+    torch.cuda.empty_cache()
+
+
+def test_an_eviction_cycle_replays_as_a_cuda_graph():
+    """E decode steps and the eviction that follows return the cache to the same lengths, so the
+    cycle can be captured once and replayed; the replayed state must equal the eagerly run one."""
+    cfg = W.get_config("c2_llama8b").scaled(layers=4, batch=2, prompt=64, budget=512, window=32, evict_interval=16)
+    E = cfg.evict_interval
+    caches = []
+    for _ in range(2):
+        g = H.make_gpu(cfg)
+        k, v = gen.torch_keys_values(cfg, 7100, cfg.budget, "cuda:0")
+        g.prefill(k, v, n_pinned=cfg.prompt)
+        caches.append(g)
+    a, b = caches
+    q, kk, vv = gen.torch_step_ring(cfg, 7100, E, "cuda:0")
+    oa = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, 128), dtype=torch.bfloat16, device="cuda:0")
+    ob = torch.empty_like(oa)
+
+    def cycle(c, o):
+        for s in range(E):
+            c.decode_attn(q[s], kk[s], vv[s], o)
+        c.evict(0)
+
+    cycle(a, oa)
+    cycle(b, ob)                      # warm-up outside the capture (first-call set-up)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        b.set_stream(side)
+        with torch.cuda.graph(graph, stream=side):
+            cycle(b, ob)
+    b.set_stream(torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    # the capture ran nothing: b is one cycle behind a; replay twice, run a twice more eagerly
+    cycle(a, oa)
+    cycle(a, oa)
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    a.poll_error(); b.poll_error()
+    assert a.len(0) == b.len(0) == cfg.budget
+    assert torch.equal(oa.view(torch.int16), ob.view(torch.int16))
+    for l, bb, h in [(0, 0, 0), (3, 1, 7), (2, 0, 5)]:
+        Ka, Va, pa, sa = a.export_slab(l, bb, h)
+        Kb, Vb, pb, sb = b.export_slab(l, bb, h)
+        assert torch.equal(pa, pb) and torch.equal(H.bits(sa), H.bits(sb)) and torch.equal(H.bits(Ka), H.bits(Kb))
+    a.close(); b.close()
