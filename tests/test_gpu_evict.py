@@ -43,7 +43,7 @@ PATTERNS = {
 
 
 @pytest.mark.parametrize("pattern", sorted(PATTERNS))
-@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("fp32", 64)])
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("fp32", 64), ("fp32", 96), ("bf16", 256), ("fp32", 256)])
 def test_patterns_bit_exact(pattern, dtype, d):
     cfg = W.get_config("c2_llama8b").scaled(layers=2, batch=2, kv_heads=2, q_heads=8, head_dim=d, dtype=dtype,
                                              prompt=24, budget=700, window=32, evict_interval=600)
