@@ -23,7 +23,9 @@
 // and takes a ticket on the slab's arrival counter.  Whoever arrives last combines the partials,
 // writes the output and then walks the slab's logits once to do the single read-modify-write of
 // every score row.  Nobody ever waits for another CTA: there is no inter-CTA spin, no float
-// atomic, one writer per score row and per output element.
+// atomic, one writer per score row and per output element.  While a CTA still has chunks to
+// stream, that pass is handed to a sixth warp (the scorer) through a two-slot task queue in shared
+// memory, so the consumer warps go straight on to the next slab.
 #pragma once
 
 #include <cuda.h>
@@ -39,7 +41,7 @@ constexpr int kStStages = 6;                     // even: chunk i of a CTA goes 
                                                  // so every stage is always consumed by the same two warps
 constexpr int kStConsumerWarps = 4;
 constexpr int kStConsumers = kStConsumerWarps * 32;
-constexpr int kStThreads = kStConsumers + 32;    // + one producer warp
+constexpr int kStThreads = kStConsumers + 64;    // + one producer warp + one scorer warp
 constexpr int kStBoxBytes = kStRows * 128;       // one TMA box: 32 rows x 64 bf16
 constexpr int kStStageBytes = 4 * kStBoxBytes;   // K low/high half of head_dim, V low/high
 constexpr int kStCombFloats = kStConsumerWarps * 4 * 128;
@@ -50,7 +52,7 @@ constexpr uint32_t kStSpinLimit = 1u << 22;      // bounded mbarrier polling
 
 __host__ __device__ inline size_t stream_smem_bytes(int Nb) {
   return 1024 /* alignment slack */ + (size_t)kStStages * kStStageBytes + sizeof(float) * kStCombFloats +
-         sizeof(float) * (2 * kStConsumerWarps * 8 + kStConsumerWarps * 8 + 4 * 8) + 16 * kStStages + 64 +
+         sizeof(float) * (2 * kStConsumerWarps * 8 + kStConsumerWarps * 8 + 4 * 8) + 16 * kStStages + 64 + 256 +
          sizeof(int) * (2 * (size_t)Nb + 2);
 }
 
@@ -160,7 +162,7 @@ __device__ __forceinline__ void cursor_next_slab(StCursor& c, const int* s_cnt, 
 template <int GG, int VB>
 __device__ __forceinline__ void score_pass_vec(bool accumulate, float* __restrict__ score, float* __restrict__ comp, float* __restrict__ dout,
                                                const float* __restrict__ lg, int cap, int n, int n_old,
-                                               const float* s_finM, const float* s_finf, int tid) {
+                                               const float* s_finM, const float* s_finf, int tid, int nthr) {
   float M[GG], f[GG];
 #pragma unroll
   for (int g = 0; g < GG; ++g) {
@@ -168,11 +170,11 @@ __device__ __forceinline__ void score_pass_vec(bool accumulate, float* __restric
     f[g] = s_finf[g];
   }
   const bool drop_lines = (cap & 31) == 0;  // then every head's row range starts on a 128-byte line
-  for (int v0 = tid; 4 * v0 < n; v0 += VB * kStConsumers) {
+  for (int v0 = tid; 4 * v0 < n; v0 += VB * nthr) {
     float4 sc[VB], cc[VB], e[VB][GG];
 #pragma unroll
     for (int i = 0; i < VB; ++i) {
-      const int j = min(4 * (v0 + i * kStConsumers), cap - 4);  // clamped: always a valid address
+      const int j = min(4 * (v0 + i * nthr), cap - 4);  // clamped: always a valid address
       sc[i] = *reinterpret_cast<const float4*>(score + j);
       cc[i] = *reinterpret_cast<const float4*>(comp + j);
 #pragma unroll
@@ -180,7 +182,7 @@ __device__ __forceinline__ void score_pass_vec(bool accumulate, float* __restric
     }
 #pragma unroll
     for (int i = 0; i < VB; ++i) {
-      const int j = 4 * (v0 + i * kStConsumers);
+      const int j = 4 * (v0 + i * nthr);
       if (j >= n) continue;
       float4 dl = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
@@ -192,7 +194,7 @@ __device__ __forceinline__ void score_pass_vec(bool accumulate, float* __restric
       }
       // The logits of these rows are dead now: drop their L2 lines instead of letting them be
       // written back to DRAM (each 128-byte line was read by eight lanes of this warp in one load).
-      if (drop_lines && (threadIdx.x & 7) == 0) {
+      if (drop_lines && (tid & 7) == 0) {
 #pragma unroll
         for (int g = 0; g < GG; ++g)
           asm volatile("discard.global.L2 [%0], 128;" ::"l"(lg + (size_t)g * cap + j) : "memory");
@@ -231,11 +233,11 @@ __device__ __forceinline__ void score_pass_vec(bool accumulate, float* __restric
 
 template <int GG>
 __device__ __forceinline__ void score_pass(bool accumulate, float* score, float* comp, float* dout, const float* lg, int cap,
-                                           int n, int n_old, const float* s_finM, const float* s_finf, int tid) {
+                                           int n, int n_old, const float* s_finM, const float* s_finf, int tid, int nthr) {
   if ((cap & 3) == 0 && cap >= 4) {
-    score_pass_vec<GG, (GG <= 4 ? 5 : 2)>(accumulate, score, comp, dout, lg, cap, n, n_old, s_finM, s_finf, tid);
+    score_pass_vec<GG, (GG <= 4 ? 5 : 2)>(accumulate, score, comp, dout, lg, cap, n, n_old, s_finM, s_finf, tid, nthr);
   } else {
-    for (int j = tid; j < n; j += kStConsumers) {
+    for (int j = tid; j < n; j += nthr) {
       float dl = 0.f;
 #pragma unroll
       for (int g = 0; g < GG; ++g) dl += fast_exp2(__ldcg(lg + (size_t)g * cap + j) - s_finM[g]) * s_finf[g];
@@ -290,6 +292,13 @@ __device__ __forceinline__ void combine_partials(const float* const (&pp)[4], in
   }
 }
 
+// A score pass handed from the consumer warps to the scorer warp.
+struct StScoreTask {
+  long long slab;  // < 0: no more tasks
+  int n, n_old;
+  float M[8], f[8];
+};
+
 #define DYNTS_DISPATCH_GROUP(G, CALL) \
   switch (G) {                        \
     case 1: { constexpr int GG = 1; CALL; } break; \
@@ -321,18 +330,26 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
   float* s_finM = s_cl + 8;                                          // [8] slab max
   float* s_finf = s_finM + 8;                                        // [8] 1 / slab sum
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_finf + 8);         // full[stages], empty[stages]
-  int* s_flags = reinterpret_cast<int*>(s_bar + 2 * kStStages);      // [0] abort, [1] last arriver, [2+s] armed phase
+  int* s_flags = reinterpret_cast<int*>(s_bar + 2 * kStStages);      // [0] abort, [1] last arriver, [2+s] armed phase, [8] uniform chunk count, [10] pass handed off
   int* s_cnt = s_flags + 16;                                         // [Nb]
   int* s_off = s_cnt + Nb;                                           // [Nb + 1]
+  // hand-off of score passes to the scorer warp: two task slots and their full/empty barriers
+  uint64_t* s_tbar = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(s_off + Nb + 1) + 15) & ~(uintptr_t)15);
+  StScoreTask* s_task = reinterpret_cast<StScoreTask*>(s_tbar + 4);
   volatile int* s_abort = s_flags;
 
   const uint32_t bar_full = smem_u32(s_bar), bar_empty = smem_u32(s_bar + kStStages);
+  const uint32_t tbar_full = smem_u32(s_tbar), tbar_empty = smem_u32(s_tbar + 2);
 
   // ---- per-CTA set-up: barriers and the chunk prefix of the sequences -------------------------
   if (tid == 0) {
     for (int s = 0; s < kStStages; ++s) {
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, 2);  // the two warps that consume the stage
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(tbar_full + 8 * s, 1);
+      mbar_init(tbar_empty + 8 * s, 1);
     }
     for (int i = 0; i < 8; ++i) s_flags[i] = 0;  // (s_flags[8] belongs to the prefix warp below)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -425,7 +442,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         if (++c.chunk == c.cb) cursor_next_slab(c, s_cnt, Nb, Hkv);
       }
     }
-  } else if (cnt > 0) {
+  } else if (cnt > 0 && warp < kStConsumerWarps) {
     // ================================== consumers ============================================
     const int gid = lane >> 2, tig = lane & 3;
     const int pair = warp >> 1, u16 = (warp & 1) * 16;  // pair: parity of the chunks (items) this warp takes
@@ -435,6 +452,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
     StCursor c;
     cursor_seek(c, g_begin, s_off, s_cnt, Nb);
     int it = 0;
+    int n_posted = 0;  // score passes handed to the scorer warp (thread 0's copy counts)
     while (it < cnt) {
       // ---- one segment: chunks [c.chunk, c.chunk + seg) of one slab -----------------------------
       const int seg = min(c.cb - c.chunk, cnt - it);
@@ -698,12 +716,63 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
       if (finish && need_pass) {
         // a5: final weights of every row of the slab, summed over the group's heads (Eq. 6)
         consumer_sync();  // s_finM / s_finf, and this CTA's own logits
-        float* dout = p.delta_out ? p.delta_out + slab * (size_t)p.cap : nullptr;
-        DYNTS_DISPATCH_GROUP(G, score_pass<GG>(p.accumulate != 0, score, p.comp + slab * (size_t)p.cap, dout, lg, p.cap, n, n_old, s_finM, s_finf, tid));
+        bool handed = false;
+        if (it + seg < cnt) {
+          // More chunks follow: leave the pass to the scorer warp (if it has a free task slot) and
+          // go on streaming.  After the last chunk the four consumer warps do the pass themselves.
+          if (tid == 0) {
+            const int slot = n_posted & 1;
+            int ok = 0;
+            if (mbar_try_wait(tbar_empty + 8 * slot, (((uint32_t)n_posted >> 1) & 1u) ^ 1u)) {
+              StScoreTask& tk = s_task[slot];
+              tk.slab = (long long)slab;
+              tk.n = n;
+              tk.n_old = n_old;
+#pragma unroll
+              for (int g = 0; g < 8; ++g) {
+                tk.M[g] = s_finM[g];
+                tk.f[g] = s_finf[g];
+              }
+              mbar_arrive(tbar_full + 8 * slot);  // release: the task and, through the barrier above, the logits
+              ++n_posted;
+              ok = 1;
+            }
+            s_flags[10] = ok;
+          }
+          consumer_sync();
+          handed = s_flags[10] != 0;
+        }
+        if (!handed) {
+          float* dout = p.delta_out ? p.delta_out + slab * (size_t)p.cap : nullptr;
+          DYNTS_DISPATCH_GROUP(G, score_pass<GG>(p.accumulate != 0, score, p.comp + slab * (size_t)p.cap, dout, lg, p.cap, n,
+                                                 n_old, s_finM, s_finf, tid, kStConsumers));
+        }
       }
       consumer_sync();  // shared scratch is reused by the next segment
       it += seg;
       if (it < cnt) cursor_next_slab(c, s_cnt, Nb, Hkv);
+    }
+    if (tid == 0 && it >= cnt) {  // tell the scorer warp that nothing more will come
+      const int slot = n_posted & 1;
+      mbar_wait(tbar_empty + 8 * slot, (((uint32_t)n_posted >> 1) & 1u) ^ 1u, s_abort, p.err);
+      s_task[slot].slab = -1;
+      mbar_arrive(tbar_full + 8 * slot);
+    }
+  } else if (cnt > 0) {
+    // ================= scorer: score passes of finished slabs, beside the streaming =================
+    for (int t = 0;; ++t) {
+      const int slot = t & 1;
+      mbar_wait(tbar_full + 8 * slot, (uint32_t)(t >> 1) & 1u, s_abort, p.err);
+      __syncwarp();
+      if (*s_abort) break;
+      const StScoreTask& tk = s_task[slot];
+      if (tk.slab < 0) break;
+      const size_t slab = (size_t)tk.slab;
+      float* dout = p.delta_out ? p.delta_out + slab * (size_t)p.cap : nullptr;
+      DYNTS_DISPATCH_GROUP(G, score_pass<GG>(p.accumulate != 0, p.score + slab * (size_t)p.cap, p.comp + slab * (size_t)p.cap, dout,
+                                             p.logit + slab * (size_t)G * p.cap, p.cap, tk.n, tk.n_old, tk.M, tk.f, lane, 32));
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tbar_empty + 8 * slot);
     }
   }
 
