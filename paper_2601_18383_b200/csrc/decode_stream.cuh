@@ -252,42 +252,66 @@ __device__ __forceinline__ void score_pass(bool accumulate, float* score, float*
   }
 }
 
-// The slab's last arriver combines the partials of the k <= 4 CTAs that worked on it; thread tid
-// produces output column tid of every head.  pp[i] = partial of contributor i (clamped copies
-// beyond k).  All loads are issued before the first use.
+// The slab's last arriver combines the partials of the k CTAs p_first..p_first+k-1 that worked on
+// it; thread tid produces output column tid of every head.  The partials are taken four at a time:
+// all loads of a group are issued before the first use, and a running (max, sum, output) is
+// rescaled between groups, so the cost is one memory round trip per four contributors.
 template <int GG>
-__device__ __forceinline__ void combine_partials(const float* const (&pp)[4], int k, __nv_bfloat16* out,
-                                                 float* s_finM, float* s_finf, int tid) {
+__device__ __forceinline__ void combine_partials(const float* part, int p_first, int k, long long g0, long long per_cta,
+                                                 __nv_bfloat16* out, float* s_finM, float* s_finf, int tid) {
   constexpr int d = 128;
-  float pm[4][GG], pl[4][GG], po[4][GG];
+  float M[GG], L[GG], acc[GG];
 #pragma unroll
-  for (int qi = 0; qi < 4; ++qi) {
+  for (int g = 0; g < GG; ++g) {
+    M[g] = -CUDART_INF_F;
+    L[g] = 0.f;
+    acc[g] = 0.f;
+  }
+  for (int q0 = 0; q0 < k; q0 += 4) {
+    const float* pp[4];
+#pragma unroll
+    for (int qi = 0; qi < 4; ++qi) {
+      const int q = p_first + min(q0 + qi, k - 1);  // clamped copies beyond k are loaded and ignored
+      const int slot = (g0 <= per_cta * q) ? 0 : 1;  // 0: the slab is the first of CTA q's piece
+      pp[qi] = part + ((size_t)q * 2 + slot) * kStPartStride;
+    }
+    float pm[4][GG], pl[4][GG], po[4][GG];
+#pragma unroll
+    for (int qi = 0; qi < 4; ++qi) {
+#pragma unroll
+      for (int g = 0; g < GG; ++g) {
+        pm[qi][g] = __ldcg(pp[qi] + 8 * d + g);
+        pl[qi][g] = __ldcg(pp[qi] + 8 * d + 8 + g);
+        po[qi][g] = __ldcg(pp[qi] + (size_t)g * d + tid);
+      }
+    }
 #pragma unroll
     for (int g = 0; g < GG; ++g) {
-      pm[qi][g] = __ldcg(pp[qi] + 8 * d + g);
-      pl[qi][g] = __ldcg(pp[qi] + 8 * d + 8 + g);
-      po[qi][g] = __ldcg(pp[qi] + (size_t)g * d + tid);
+      float Mn = M[g];
+#pragma unroll
+      for (int qi = 0; qi < 4; ++qi)
+        if (q0 + qi < k) Mn = fmaxf(Mn, pm[qi][g]);
+      const float r = fast_exp2(M[g] - Mn);  // 0 for the first group (M = -inf; every partial max is finite)
+      float Ln = L[g] * r, an = acc[g] * r;
+#pragma unroll
+      for (int qi = 0; qi < 4; ++qi) {
+        if (q0 + qi < k) {
+          const float w = fast_exp2(pm[qi][g] - Mn);
+          Ln += pl[qi][g] * w;
+          an += po[qi][g] * w;
+        }
+      }
+      M[g] = Mn;
+      L[g] = Ln;
+      acc[g] = an;
     }
   }
 #pragma unroll
   for (int g = 0; g < GG; ++g) {
-    float M = -CUDART_INF_F;
-#pragma unroll
-    for (int qi = 0; qi < 4; ++qi)
-      if (qi < k) M = fmaxf(M, pm[qi][g]);
-    float L = 0.f, acc = 0.f;
-#pragma unroll
-    for (int qi = 0; qi < 4; ++qi) {
-      if (qi < k) {
-        const float w = fast_exp2(pm[qi][g] - M);
-        L += pl[qi][g] * w;
-        acc += po[qi][g] * w;
-      }
-    }
-    out[(size_t)g * d + tid] = __float2bfloat16_rn(acc / L);
+    out[(size_t)g * d + tid] = __float2bfloat16_rn(acc[g] / L[g]);
     if (tid == 0) {
-      s_finM[g] = M;
-      s_finf[g] = 1.0f / L;
+      s_finM[g] = M[g];
+      s_finf[g] = 1.0f / L[g];
     }
   }
 }
@@ -677,40 +701,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         if (finish) {
           // Last arriver: combine the partials of CTAs p_first..p_last; thread tid does column tid.
           const int k = p_last - p_first + 1;
-          if (k <= 4) {
-            const float* pp[4];
-#pragma unroll
-            for (int qi = 0; qi < 4; ++qi) {
-              const int q = min(p_first + qi, p_last);
-              const int slot = (g0 <= per_cta * q) ? 0 : 1;
-              pp[qi] = p.part + ((size_t)q * 2 + slot) * kStPartStride;
-            }
-            DYNTS_DISPATCH_GROUP(G, combine_partials<GG>(pp, k, out, s_finM, s_finf, tid));
-          } else {
-#pragma unroll
-            for (int g = 0; g < kMaxGroup; ++g) {
-              if (g < G) {
-                float M = -CUDART_INF_F;
-                for (int q = p_first; q <= p_last; ++q) {
-                  const int slot = (g0 <= per_cta * q) ? 0 : 1;
-                  M = fmaxf(M, __ldcg(p.part + ((size_t)q * 2 + slot) * kStPartStride + 8 * d + g));
-                }
-                float L = 0.f, acc = 0.f;
-                for (int q = p_first; q <= p_last; ++q) {
-                  const int slot = (g0 <= per_cta * q) ? 0 : 1;
-                  const float* pq = p.part + ((size_t)q * 2 + slot) * kStPartStride;
-                  const float f = fast_exp2(__ldcg(pq + 8 * d + g) - M);
-                  L += __ldcg(pq + 8 * d + 8 + g) * f;
-                  acc += __ldcg(pq + (size_t)g * d + tid) * f;
-                }
-                out[(size_t)g * d + tid] = __float2bfloat16_rn(acc / L);
-                if (tid == 0) {
-                  s_finM[g] = M;
-                  s_finf[g] = 1.0f / L;
-                }
-              }
-            }
-          }
+          DYNTS_DISPATCH_GROUP(G, combine_partials<GG>(p.part, p_first, k, g0, per_cta, out, s_finM, s_finf, tid));
         }
       }
       if (finish && need_pass) {
