@@ -5,7 +5,9 @@
 // rows; the chunks of all slabs of the launch form one list, ordered slab by slab, and the
 // persistent grid (two CTAs per SM) cuts that list into equal contiguous pieces, one per CTA
 // ("stream-K": a CTA usually starts in the middle of one slab, covers some slabs completely and
-// stops in the middle of another).  Inside a CTA one producer thread walks the piece and issues
+// stops in the middle of another; when all slabs are equally long and there are at least about as
+// many as CTAs, a piece is a whole number of slabs instead and no slab is shared).  Inside a CTA
+// one producer thread walks the piece and issues
 // TMA tile loads (cp.async.bulk.tensor, 128-byte swizzle, no multicast) of the K and V rows of
 // each chunk into a 6-stage shared-memory ring guarded by mbarriers, running ahead of the four
 // consumer warps across chunk and slab boundaries, so the HBM stream never pauses for an
