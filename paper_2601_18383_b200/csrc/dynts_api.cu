@@ -928,7 +928,7 @@ int mlp_k_slices(int rows, int K) {
   return best;
 }
 
-bool g_mlp_attr = false;
+bool g_mlp_attr[64] = {false};  // per device: function attributes are set once per device
 
 }  // namespace
 
@@ -952,10 +952,13 @@ dynts_status_t dynts_predictor_mlp(const void* h, const void* W1, const float* b
   const size_t need = dynts_predictor_mlp_scratch_bytes(d, batch);
   if (scratch_bytes < need) return fail(DYNTS_ERR_OOM, "scratch too small: %zu < %zu bytes", scratch_bytes, need);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (!g_mlp_attr) {
+  int dev = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(DYNTS_ERR_INVALID_ARG, "device index %d not supported", dev);
+  if (!g_mlp_attr[dev]) {
     CUDA_TRY(cudaFuncSetAttribute(dynts::mlp_layer_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024));
     CUDA_TRY(cudaFuncSetAttribute(dynts::mlp_layer_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024));
-    g_mlp_attr = true;
+    g_mlp_attr[dev] = true;
   }
   const int NT = batch > 8 ? 16 : 8;  // sequences per batch tile
   const int ks1 = mlp_k_slices(2 * d, d), ks2 = mlp_k_slices(d / 2, 2 * d);
