@@ -294,10 +294,10 @@ def run_ours(args, cfg, rank, world, device):
     result = {
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": warm,
         "ms_per_step": round(ms / K, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 inputs, fp32 accumulate" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+        "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": cfg.name, "layers": cfg.layers, "batch": cfg.batch, "q_heads": cfg.q_heads,
                    "kv_heads": cfg.kv_heads, "head_dim": cfg.head_dim, "budget": cfg.budget, "window": cfg.window,
-                   "evict_interval": E, "prompt_pinned": cfg.prompt, "dist": cfg.dist, "score_source": args.score_source, "selection": args.selection,
+                   "evict_interval": E, "prompt_pinned": cfg.prompt, "dist": cfg.dist, "score_source": args.score_source, "selection": args.selection, "accumulate": "fp32 (softmax, output, scores)",
                    "cache_bytes": cache.nbytes, "l2_policy": "inputs larger than L2 (KV cache %.0f MB vs 126 MB L2)" % (cache.nbytes / 1e6),
                    "replicas": world},
         "hbm_gbs_decode": round(dec_gbs, 1), "roofline": roofline, "evict": evict, "e2e": e2e,
