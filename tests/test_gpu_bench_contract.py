@@ -1,0 +1,42 @@
+"""The benchmark's JSON line on a GPU: the keys and invariants its consumers rely on (a short run
+on the tiny workload and on a shortened default workload)."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+pytestmark = pytest.mark.gpu
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _run(*extra):
+    cmd = [sys.executable, "bench.py", "--steps", "128", "--warmup", "64", "--cpu-seconds", "1"] + list(extra)
+    res = subprocess.run(cmd, cwd=ROOT, capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0, res.stderr[-3000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    return json.loads(lines[0])
+
+
+@pytest.mark.parametrize("extra", [(), ("--score-source", "external"), ("--workload", "c1_tiny_fp32")])
+def test_bench_line_contract(extra):
+    d = _run(*extra)
+    assert d["metric"] == "decode tokens/s at budget B" and d["unit"] == "tokens/s" and d["higher_is_better"] is True
+    assert d["n_gpus"] == 1 and d["steps"] == 128 and d["warmup"] >= 64 and d["scaling"] == "weak"
+    assert d["vs_baseline"] is None and d["data"] == "synthetic" and d["dtype"] in ("bf16", "f32")
+    assert d["value"] > 0 and abs(d["value"] - d["config"]["batch"] / (d["ms_per_step"] * 1e-3)) <= 0.01 * d["value"]
+    assert "workload" in d["config"] and "model" not in d["config"]
+    r = d["roofline"]
+    assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["peak"] > 0 and r["achieved"] > 0
+    assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-3 and "traffic" in r
+    e = d["e2e"]
+    assert e["value"] > 0 and e["unit"] == "tokens/s" and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0
+    assert e["value"] < d["value"] * 1.05                      # the end-to-end arm includes the copies
+    c = d["cpu_baseline"]
+    assert c["kind"] == "oracle" and c["cores"] >= 1 and c["value"] > 0 and c["sample"]
+    assert d["gpu_launches"] >= 128
+    assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
+    if d["evict"] is not None:
+        assert d["evict"]["bound"] == "hbm" and d["evict"]["achieved"] >= 0
