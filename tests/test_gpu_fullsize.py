@@ -208,3 +208,45 @@ def test_an_eviction_cycle_replays_as_a_cuda_graph():
         Kb, Vb, pb, sb = b.export_slab(l, bb, h)
         assert torch.equal(pa, pb) and torch.equal(H.bits(sa), H.bits(sb)) and torch.equal(H.bits(Ka), H.bits(Kb))
     a.close(); b.close()
+
+
+def test_two_caches_on_two_streams_do_not_interfere():
+    """Two caches of different shapes driven alternately on their own streams (their kernels may
+    overlap on the GPU) give bit-identical results to the same caches driven one after the other."""
+    cfgs = [W.get_config("c2_llama8b").scaled(layers=6, batch=3, prompt=64, budget=448, window=32, evict_interval=16),
+            W.get_config("c3_qwen7b").scaled(layers=4, batch=2, kv_heads=2, q_heads=14, prompt=48, budget=320, window=16,
+                                            evict_interval=16)]
+    results = []
+    for mode in ("interleaved", "sequential"):
+        caches, rings, outs, streams = [], [], [], []
+        for i, cfg in enumerate(cfgs):
+            g = H.make_gpu(cfg)
+            k, v = gen.torch_keys_values(cfg, 8100 + i, cfg.budget, "cuda:0")
+            g.prefill(k, v, n_pinned=cfg.prompt)
+            caches.append(g)
+            rings.append(gen.torch_step_ring(cfg, 8100 + i, 16, "cuda:0"))
+            outs.append(torch.zeros((cfg.layers, cfg.batch, cfg.q_heads, 128), dtype=torch.bfloat16, device="cuda:0"))
+            streams.append(torch.cuda.Stream())
+        torch.cuda.synchronize()
+        if mode == "interleaved":
+            for i, g in enumerate(caches):
+                g.set_stream(streams[i])
+        order = [(s, i) for s in range(48) for i in range(2)] if mode == "interleaved" else \
+                [(s, i) for i in range(2) for s in range(48)]
+        for s, i in order:
+            q, kk, vv = rings[i]
+            caches[i].decode_attn(q[s % 16], kk[s % 16], vv[s % 16], outs[i])
+            if (s + 1) % 16 == 0:
+                caches[i].evict(0)
+        torch.cuda.synchronize()
+        snap = []
+        for i, g in enumerate(caches):
+            g.poll_error()
+            cfg = cfgs[i]
+            K, V, pos, score = g.export_slab(cfg.layers - 1, cfg.batch - 1, cfg.kv_heads - 1)
+            snap.append((outs[i].clone(), K, pos, score))
+            g.close()
+        results.append(snap)
+    for a, b in zip(*results):
+        assert torch.equal(a[0].view(torch.int16), b[0].view(torch.int16))
+        assert torch.equal(H.bits(a[1]), H.bits(b[1])) and torch.equal(a[2], b[2]) and torch.equal(H.bits(a[3]), H.bits(b[3]))
