@@ -12,6 +12,8 @@ What each function follows in the paper:
 * ``decode_step`` (delta/score part) -- Eq. 6: a token's importance is the attention it receives
   summed over query rows.  Here the rows are the decode queries seen so far, summed over the
   query heads that share the KV head (Appendix B.1 aggregates heads; sum is this build's reading).
+* ``prefill_attention`` -- the same Eq. 4-5 for every prompt position (the prefill phase that fills
+  the question window of Section 4.2).
 * ``select_keep`` / ``evict`` -- Section 4.2: the question window (the first M rows) and the local
   window (the last W rows) are always retained, the top-k of the selection window by score are
   retained, the rest are evicted.  Ties go to the lower index; retained rows keep their order.
@@ -171,6 +173,33 @@ def decode_step(cache: OracleCache, q: np.ndarray, k_new: np.ndarray, v_new: np.
         if active is None or active[b]:
             cache.next_pos[b] += 1
     return out, delta
+
+
+# ----------------------------------------------------------------------------------------------
+# Eq. 4-5 over the prompt: the prefill phase that fills the question window (Section 4.2)
+# ----------------------------------------------------------------------------------------------
+
+def prefill_attention(q: np.ndarray, k: np.ndarray, v: np.ndarray) -> np.ndarray:
+    """Token-level attention of every prompt position over the positions up to and including
+    itself (Eq. 4-5 with t = 1..M), for all layers, sequences and heads.
+
+    q [L, Nb, Hq, T, d]; k, v [L, Nb, Hkv, T, d] -> out [L, Nb, Hq, T, d] float64.  Query head g
+    of KV head h is head h * G + g (the grouping of decode_step)."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    L, Nb, Hq, T, d = q.shape
+    Hkv = k.shape[2]
+    G = Hq // Hkv
+    out = np.zeros_like(q)
+    for l in range(L):
+        for b in range(Nb):
+            for hq in range(Hq):
+                h = hq // G
+                for t in range(T):
+                    alpha = attention_weights(q[l, b, hq, t][None, :], k[l, b, h, :t + 1])   # Eq. 4 over j <= t
+                    out[l, b, hq, t] = attention_output(alpha, v[l, b, h, :t + 1])[0]       # Eq. 5
+    return out
 
 
 # ----------------------------------------------------------------------------------------------

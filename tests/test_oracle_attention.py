@@ -211,3 +211,33 @@ def test_pinned_rows_stay_infinite_and_new_row_starts_at_self_mass():
     assert np.isinf(s.score[:3]).all()
     assert s.score[3] == delta[0][0][0][3]
     assert list(s.pos[:4]) == [0, 1, 2, 3]
+
+
+def test_prefill_attention_against_masked_softmax_and_decode_consistency():
+    """Prefill attention row t must equal (a) the textbook masked softmax(QK^T/sqrt(d))V computed
+    with a lower-triangular mask, and (b) what a decode step gives for the same token when the
+    first t rows are already cached."""
+    r = np.random.default_rng(12)
+    L, Nb, Hq, Hkv, T, d = 2, 2, 4, 2, 9, 8
+    q = r.standard_normal((L, Nb, Hq, T, d))
+    k = r.standard_normal((L, Nb, Hkv, T, d))
+    v = r.standard_normal((L, Nb, Hkv, T, d))
+    out = O.prefill_attention(q, k, v)
+    G = Hq // Hkv
+    mask = np.tril(np.ones((T, T), dtype=bool))
+    for l in range(L):
+        for b in range(Nb):
+            for hq in range(Hq):
+                e = q[l, b, hq] @ k[l, b, hq // G].T / np.sqrt(d)
+                e = np.where(mask, e, -np.inf)
+                p = np.exp(e - e.max(axis=1, keepdims=True))
+                ref = (p / p.sum(axis=1, keepdims=True)) @ v[l, b, hq // G]
+                np.testing.assert_allclose(out[l, b, hq], ref, rtol=1e-12, atol=1e-12)
+    # first position attends to itself only
+    for hq in range(Hq):
+        np.testing.assert_allclose(out[0, 0, hq, 0], v[0, 0, hq // G, 0], rtol=1e-13)
+    # decode consistency: cache the first T-1 rows, decode the last token
+    cache = O.OracleCache(L, Nb, Hq, Hkv, d, 2, T + 2)
+    O.prefill(cache, k[..., :T - 1, :], v[..., :T - 1, :])
+    o_dec, _ = O.decode_step(cache, q[..., T - 1, :], k[..., T - 1, :], v[..., T - 1, :])
+    np.testing.assert_allclose(o_dec, out[..., T - 1, :], rtol=1e-12, atol=1e-12)
