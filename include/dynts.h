@@ -93,6 +93,16 @@ dynts_status_t dynts_cache_set_stream(dynts_cache_t* c, void* stream);
  * Positions are 0..n_tokens-1.  Replaces the sequences' previous content. */
 dynts_status_t dynts_prefill(dynts_cache_t* c, const void* k, const void* v, int n_tokens, int n_pinned);
 
+/* dynts_prefill plus the attention of the prompt itself (Eq. 4-5 for t = 1..n_tokens: position t
+ * attends to positions 1..t), for a model that runs its prefill through this library.
+ *   q, out: device [L, Nb, Hq, n_tokens, d];  k, v: device [L, Nb, Hkv, n_tokens, d]; bf16, d = 128.
+ * The rows are stored exactly as dynts_prefill stores them (the first n_pinned pinned with score
+ * +inf); prompt attention adds nothing to the scores (the paper pins the question instead of
+ * scoring it).  A dense contraction: runs on the tensor pipe.  Other dtypes and head sizes:
+ * DYNTS_ERR_INVALID_ARG. */
+dynts_status_t dynts_prefill_attn(dynts_cache_t* c, const void* q, const void* k, const void* v, void* out, int n_tokens,
+                                  int n_pinned);
+
 /* The same for one sequence of a ragged batch; k, v: device [L, Hkv, n_tokens, d].  Marks the
  * sequence active. */
 dynts_status_t dynts_prefill_seq(dynts_cache_t* c, int seq, const void* k, const void* v, int n_tokens, int n_pinned);

@@ -20,6 +20,7 @@
 #include "decode_stream.cuh"
 #include "evict.cuh"
 #include "predictor.cuh"
+#include "prefill_attn.cuh"
 
 namespace {
 
@@ -129,7 +130,7 @@ struct dynts_cache {
   char* stage_dev = nullptr;
   size_t stage_bytes = 0;
   bool attr_generic_f32 = false, attr_generic_bf16 = false, attr_mma = false, attr_select = false;
-  bool attr_stream = false, attr_fused = false;
+  bool attr_stream = false, attr_fused = false, attr_prefill = false;
   bool have_maps = false;    // tensor maps of the K and V slabs for the streaming kernel
   CUtensorMap map_K, map_V;
   int sm_count = 0;
@@ -638,6 +639,37 @@ dynts_status_t dynts_cache_set_stream(dynts_cache_t* c, void* stream) {
 
 dynts_status_t dynts_prefill(dynts_cache_t* c, const void* k, const void* v, int n_tokens, int n_pinned) {
   return do_prefill(c, -1, k, v, n_tokens, n_pinned);
+}
+
+dynts_status_t dynts_prefill_attn(dynts_cache_t* c, const void* q, const void* k, const void* v, void* out, int n_tokens,
+                                  int n_pinned) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (!q || !out || !aligned16(q) || !aligned16(out))
+    return fail(DYNTS_ERR_INVALID_ARG, "q and out must be non-NULL and 16-byte aligned");
+  if (c->cfg.dtype != DYNTS_BF16 || c->cfg.head_dim != 128)
+    return fail(DYNTS_ERR_INVALID_ARG, "prefill attention needs bf16 and head_dim 128");
+  if (n_tokens < 1) return fail(DYNTS_ERR_INVALID_ARG, "n_tokens must be positive");
+  dynts_status_t st = do_prefill(c, -1, k, v, n_tokens, n_pinned);  // rows, positions, pins
+  if (st != DYNTS_OK) return st;
+  if (!c->attr_prefill) {
+    CUDA_TRY(cudaFuncSetAttribute(dynts::prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dynts::kPfSmemBytes));
+    c->attr_prefill = true;
+  }
+  dynts::PrefillAttnParams p;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.k = static_cast<const __nv_bfloat16*>(k);
+  p.v = static_cast<const __nv_bfloat16*>(v);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.T = n_tokens;
+  p.Hq = c->cfg.q_heads;
+  p.Hkv = c->cfg.kv_heads;
+  p.scale_log2 = (float)(1.4426950408889634 / std::sqrt(128.0));
+  const dim3 grid((unsigned)((n_tokens + dynts::kPfRows - 1) / dynts::kPfRows), (unsigned)c->cfg.q_heads,
+                  (unsigned)(c->cfg.layers * c->cfg.batch));
+  dynts::prefill_attn_kernel<<<grid, dynts::kPfThreads, dynts::kPfSmemBytes, c->stream>>>(p);
+  CUDA_TRY(cudaGetLastError());
+  c->launches += 1;
+  return DYNTS_OK;
 }
 
 dynts_status_t dynts_prefill_seq(dynts_cache_t* c, int seq, const void* k, const void* v, int n_tokens, int n_pinned) {

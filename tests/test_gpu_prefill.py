@@ -1,0 +1,75 @@
+"""GPU parity of the prefill path: attention of every prompt position over the positions up to
+itself (Eq. 4-5 for t = 1..M) against the float64 oracle, and the cache state it leaves behind."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from oracle import dynts_oracle as O
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _qkv(cfg, T, seed):
+    r = np.random.default_rng(seed)
+    bf = lambda x: W.to_cache_dtype(x, "bf16")
+    q = bf(r.standard_normal((cfg.layers, cfg.batch, cfg.q_heads, T, cfg.head_dim)))
+    k, v = W.prompt_kv(cfg, seed, n_tokens=T)
+    return q, k, v
+
+
+@pytest.mark.parametrize("T", [1, 17, 64, 65, 200, 512])
+@pytest.mark.parametrize("G", [4, 7])
+def test_prefill_attention_matches_oracle(T, G):
+    cfg = W.get_config("c2_llama8b").scaled(layers=2, batch=2, kv_heads=2, q_heads=2 * G, prompt=T, budget=max(T, 64),
+                                             window=min(8, T), evict_interval=16)
+    q, k, v = _qkv(cfg, T, 40 + T + G)
+    gpu = H.make_gpu(cfg)
+    out = torch.full((cfg.layers, cfg.batch, cfg.q_heads, T, 128), float("nan"), dtype=torch.bfloat16, device="cuda:0")
+    gpu.prefill_attn(H.dev(q, cfg), H.dev(k, cfg), H.dev(v, cfg), out)
+    gpu.synchronize()
+    gpu.poll_error()
+    ref = O.prefill_attention(q, k, v)
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert H.rel_err_vectors(got, ref) <= H.TOL_OUT["bf16"]
+    # the cache holds the prompt exactly as dynts_prefill would have stored it
+    assert gpu.len(0) == T
+    for (l, b, h) in [(0, 0, 0), (1, 1, 1)]:
+        Kd, Vd, pos, score = gpu.export_slab(l, b, h)
+        assert np.array_equal(Kd.float().numpy(), k[l, b, h]) and np.array_equal(Vd.float().numpy(), v[l, b, h])
+        assert np.array_equal(pos.numpy(), np.arange(T)) and np.isinf(score.numpy()).all()
+    gpu.close()
+
+
+def test_decode_after_prefill_attention_continues_the_sequence():
+    """The last prefill row and the first decode step are the same operation on consecutive
+    tokens: run prefill over T tokens, then decode token T + 1, and compare both with a prefill
+    over T + 1 tokens."""
+    cfg = W.get_config("c2_llama8b").scaled(layers=1, batch=1, kv_heads=2, q_heads=8, prompt=90, budget=128, window=8,
+                                             evict_interval=16)
+    T = 90
+    q, k, v = _qkv(cfg, T + 1, 77)
+    ref = O.prefill_attention(q, k, v)
+    gpu = H.make_gpu(cfg)
+    out = torch.empty((1, 1, 8, T, 128), dtype=torch.bfloat16, device="cuda:0")
+    gpu.prefill_attn(H.dev(q[..., :T, :], cfg), H.dev(k[..., :T, :], cfg), H.dev(v[..., :T, :], cfg), out)
+    o1 = torch.empty((1, 1, 8, 128), dtype=torch.bfloat16, device="cuda:0")
+    gpu.decode_attn(H.dev(q[..., T, :], cfg), H.dev(k[..., T, :], cfg), H.dev(v[..., T, :], cfg), o1)
+    gpu.synchronize()
+    assert H.rel_err_vectors(out.float().cpu().numpy(), ref[..., :T, :]) <= H.TOL_OUT["bf16"]
+    assert H.rel_err_vectors(o1.float().cpu().numpy(), ref[..., T, :]) <= H.TOL_OUT["bf16"]
+    gpu.close()
+
+
+def test_prefill_attention_rejects_other_shapes():
+    import paper_2601_18383_b200 as D
+    cfg = W.get_config("c1_tiny_fp32").scaled(prompt=8)
+    gpu = H.make_gpu(cfg)
+    x = torch.zeros((1, 1, 4, 8, 64), device="cuda:0")
+    kv = torch.zeros((1, 1, 1, 8, 64), device="cuda:0")
+    with pytest.raises(D.DyntsError) as e:
+        gpu.prefill_attn(x, kv, kv, x)
+    assert e.value.status == D.DYNTS_ERR_INVALID_ARG and gpu.len(0) == 0
+    gpu.close()
