@@ -286,6 +286,11 @@ def run_ours(args, cfg, rank, world, device):
     if rank == 0 and world == 1:
         predictor = time_predictor(cfg.batch, device, peak)
 
+    # ---- prefill attention of the prompt (dense: tensor-bound) ------------------------------------
+    prefill = None
+    if rank == 0 and world == 1 and cfg.dtype == "bf16" and cfg.head_dim == 128:
+        prefill = time_prefill(cfg, device)
+
     # ---- CPU baseline: the oracle, as it stands, on this machine's host cores (rank 0, N = 1) ------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -301,7 +306,7 @@ def run_ours(args, cfg, rank, world, device):
                    "cache_bytes": cache.nbytes, "l2_policy": "inputs larger than L2 (KV cache %.0f MB vs 126 MB L2)" % (cache.nbytes / 1e6),
                    "replicas": world},
         "hbm_gbs_decode": round(dec_gbs, 1), "roofline": roofline, "evict": evict, "e2e": e2e,
-        "predictor_mlp": predictor, "cpu_baseline": cpu, "clocks": clocks, "gpu_launches": int(launches),
+        "predictor_mlp": predictor, "prefill_attn": prefill, "cpu_baseline": cpu, "clocks": clocks, "gpu_launches": int(launches),
     }
     cache.close()
     return result
@@ -338,6 +343,42 @@ def time_predictor(batch, device, peak, d=4096, iters=40):
     gbs = wbytes / (us * 1e-6) / 1e9
     return {"d": d, "batch": batch, "us_per_call": round(us, 2), "weight_bytes": wbytes, "bound": "hbm",
             "achieved": round(gbs, 1), "peak": peak, "unit": "GB/s", "frac": round(gbs / peak, 4)}
+
+
+def time_prefill(cfg, device, iters=10):
+    """Times dynts_prefill_attn on the workload's prompt (all layers, batch, heads); flops = 4 d per
+    (query, key) pair of the causal triangle; peak = the measured dense bf16 GEMM rate."""
+    import torch
+    import paper_2601_18383_b200 as D
+    sub = cfg.scaled(layers=min(cfg.layers, 8), seq_budgets=None, budget=max(cfg.budget, cfg.prompt))
+    T = sub.prompt
+    cache = D.Cache(sub.layers, sub.batch, sub.q_heads, sub.kv_heads, sub.head_dim, sub.budget, sub.window, sub.evict_interval,
+                    dtype="bf16", device=device)
+    g = torch.Generator(device=device).manual_seed(7)
+    q = torch.randn((sub.layers, sub.batch, sub.q_heads, T, 128), generator=g, device=device).to(torch.bfloat16)
+    k, v = gen.torch_keys_values(sub, 9, T, device)
+    out = torch.empty_like(q)
+    st = torch.cuda.current_stream(device)
+    for _ in range(3):
+        cache.prefill_attn(q, k, v, out)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(st)
+    for _ in range(iters):
+        cache.prefill_attn(q, k, v, out)
+    b.record(st)
+    torch.cuda.synchronize(device)
+    us = a.elapsed_time(b) * 1e3 / iters
+    cache.close()
+    flops = 4 * 128 * (T * (T + 1) // 2) * sub.layers * sub.batch * sub.q_heads
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak_tf, kind = float(json.load(f)["bf16_tflops"]), "measured"
+    except Exception:
+        peak_tf, kind = 1590.0, "fallback"
+    tf = flops / (us * 1e-6) / 1e12
+    return {"prompt_tokens": T, "layers_timed": sub.layers, "us_per_call": round(us, 1), "flops": flops, "bound": "tensor",
+            "achieved": round(tf, 1), "peak": peak_tf, "peak_kind": kind, "unit": "TFLOP/s", "frac": round(tf / peak_tf, 4),
+            "note": "includes the copy of the prompt K/V rows into the slabs"}
 
 
 def oracle_baseline(cfg, cache, q_ring, k_ring, v_ring, budget_s=20.0, slabs=None):
