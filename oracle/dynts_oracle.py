@@ -22,6 +22,11 @@ What each function follows in the paper:
 * ``set_new_scores`` / ``predictor_mlp`` / ``paper_target`` / ``run_paper_schedule`` -- Section 4.1
   (Eq. 7: one predictor score per token) and Section 4.2 as written (select when the count reaches
   the budget B, keep a ratio of the selection window).
+* ``fp8_e4m3_*`` / ``OracleCache(kv_format="e4m3")`` -- no passage of the paper: K/V rows stored as
+  8-bit floats (the OCP 8-bit floating point format E4M3: 1 sign, 4 exponent bits with bias 7,
+  3 mantissa bits, no infinities, largest finite value 448) with one scale per tensor.  A row is
+  stored as the nearest representable value of x / scale (ties to the even code, saturating) and
+  read back as value * scale; everything downstream is unchanged.
 * ``eviction_count`` / ``effective_length`` -- Section 5, the closed form for the cache length.
 * ``attn_flops`` / ``predictor_flops`` / ``break_even_volume`` -- Appendix A and Eq. 9-10.
 
@@ -62,6 +67,49 @@ def attention_output(alpha: np.ndarray, V: np.ndarray) -> np.ndarray:
 
 
 # ----------------------------------------------------------------------------------------------
+# 8-bit K/V storage (E4M3): the format written out from its definition
+# ----------------------------------------------------------------------------------------------
+
+def fp8_e4m3_values() -> np.ndarray:
+    """The 127 non-negative finite E4M3 values by code 0..126 (ascending): exponent field 0 holds
+    the subnormals m/8 * 2^-6, fields 1..15 hold (1 + m/8) * 2^(e - 7); code 127 (all ones) is NaN."""
+    vals = []
+    for code in range(127):
+        e, m = code >> 3, code & 7
+        vals.append(m / 8.0 * 2.0 ** -6 if e == 0 else (1.0 + m / 8.0) * 2.0 ** (e - 7))
+    return np.array(vals, dtype=np.float64)
+
+
+def fp8_e4m3_encode(x: np.ndarray) -> np.ndarray:
+    """Codes (uint8, sign in bit 7) of the E4M3 values nearest to x: round to nearest, ties to the
+    code with an even mantissa bit, magnitudes beyond 448 saturate to 448.  x is taken as float32
+    (the precision the device converts from)."""
+    x = np.asarray(x, dtype=np.float32).astype(np.float64)
+    table = fp8_e4m3_values()
+    a = np.abs(x)
+    hi = np.clip(np.searchsorted(table, a, side="left"), 0, 126)      # first value >= a (or the last)
+    lo = np.clip(hi - 1, 0, 126)
+    d_lo, d_hi = a - table[lo], table[hi] - a
+    pick_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))
+    code = np.where(pick_hi, hi, lo)
+    code = np.where(a >= table[126], 126, code)
+    return (code | np.where(np.signbit(x), 128, 0)).astype(np.uint8)
+
+
+def fp8_e4m3_decode(code: np.ndarray) -> np.ndarray:
+    code = np.asarray(code, dtype=np.uint8)
+    mag = fp8_e4m3_values()[np.minimum(code & 127, 126)]
+    return np.where(code & 128, -mag, mag)
+
+
+def fp8_e4m3_store(x: np.ndarray, scale: float) -> np.ndarray:
+    """What a cache with E4M3 rows holds for x: decode(encode(x / scale)) * scale, the division in
+    float32 (the precision in which the device takes this integer decision)."""
+    x32 = np.asarray(x, dtype=np.float32) / np.float32(scale)
+    return fp8_e4m3_decode(fp8_e4m3_encode(x32)) * float(np.float32(scale))
+
+
+# ----------------------------------------------------------------------------------------------
 # Cache state
 # ----------------------------------------------------------------------------------------------
 
@@ -80,8 +128,11 @@ class Slab:
 
 class OracleCache:
     def __init__(self, layers: int, batch: int, q_heads: int, kv_heads: int, head_dim: int,
-                 window: int, capacity: int):
+                 window: int, capacity: int, kv_format: Optional[str] = None, k_scale: float = 1.0,
+                 v_scale: float = 1.0):
         assert q_heads % kv_heads == 0
+        assert kv_format in (None, "e4m3")
+        self.kv_format, self.k_scale, self.v_scale = kv_format, k_scale, v_scale
         self.layers, self.batch = layers, batch
         self.q_heads, self.kv_heads, self.head_dim = q_heads, kv_heads, head_dim
         self.group = q_heads // kv_heads
@@ -97,6 +148,13 @@ class OracleCache:
         if s is None:
             s = self._slabs[key] = Slab(self.capacity, self.head_dim)
         return s
+
+    def stored_k(self, k: np.ndarray) -> np.ndarray:
+        """The value the cache holds for a key row (the row itself unless rows are 8-bit)."""
+        return fp8_e4m3_store(k, self.k_scale) if self.kv_format == "e4m3" else k
+
+    def stored_v(self, v: np.ndarray) -> np.ndarray:
+        return fp8_e4m3_store(v, self.v_scale) if self.kv_format == "e4m3" else v
 
     def length(self, seq: int) -> int:
         return self.slab(0, seq, 0).n
@@ -125,8 +183,8 @@ def prefill(cache: OracleCache, k: np.ndarray, v: np.ndarray, n_pinned: Optional
                 s = cache.slab(l, b, h)
                 src_k = k[l, b, h] if seq is None else k[l, h]
                 src_v = v[l, b, h] if seq is None else v[l, h]
-                s.K[:T] = src_k
-                s.V[:T] = src_v
+                s.K[:T] = cache.stored_k(src_k)
+                s.V[:T] = cache.stored_v(src_v)
                 s.pos[:T] = np.arange(T)
                 s.score[:T] = 0.0
                 s.score[:m] = np.inf
@@ -156,8 +214,8 @@ def decode_step(cache: OracleCache, q: np.ndarray, k_new: np.ndarray, v_new: np.
         if active is not None and not active[b]:
             continue
         assert s.n < cache.capacity, "append past capacity: an eviction was skipped"
-        s.K[s.n] = k_new[l, b, h]
-        s.V[s.n] = v_new[l, b, h]
+        s.K[s.n] = cache.stored_k(k_new[l, b, h])
+        s.V[s.n] = cache.stored_v(v_new[l, b, h])
         s.pos[s.n] = cache.next_pos[b]
         s.score[s.n] = 0.0
         s.n += 1
