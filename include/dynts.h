@@ -42,7 +42,12 @@ typedef enum dynts_status {
   DYNTS_ERR_DEVICE = 7       /* a kernel found an inconsistent length or bound and skipped work */
 } dynts_status_t;
 
-typedef enum dynts_dtype { DYNTS_BF16 = 0, DYNTS_FP32 = 1 } dynts_dtype_t;
+/* DYNTS_BF16_KV8: q, k, v, out are bf16; the slabs hold each K/V element as an 8-bit float (E4M3:
+ * 1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest finite value 448)
+ * with one scale per tensor: a row element x is stored as the code nearest to x / scale (ties to
+ * the even code, magnitudes beyond 448 saturate) and read as value(code) * scale.  The paper does
+ * not describe this storage; it halves the bytes a decode step reads.  Needs head_dim % 16 == 0. */
+typedef enum dynts_dtype { DYNTS_BF16 = 0, DYNTS_FP32 = 1, DYNTS_BF16_KV8 = 2 } dynts_dtype_t;
 
 typedef enum dynts_score_source { DYNTS_SCORE_ATTENTION = 0, DYNTS_SCORE_EXTERNAL = 1 } dynts_score_source_t;
 
@@ -52,7 +57,7 @@ typedef struct dynts_config {
   int window;         /* W_l: most recent rows, always kept */
   int evict_interval; /* E: decode steps between evictions; slab capacity = max budget + E */
   int capacity;       /* rows per slab; 0 => max budget + evict_interval */
-  int dtype;          /* dynts_dtype_t of q, k, v, out and the slabs */
+  int dtype;          /* dynts_dtype_t of q, k, v, out and of the slab rows */
   const int* seq_budgets; /* host [batch] per-sequence targets, or NULL => budget for all */
   void* storage;          /* device memory for the whole cache, 256-byte aligned, or NULL:
                              the library then allocates with cudaMalloc and frees in destroy */
@@ -181,6 +186,11 @@ dynts_status_t dynts_evict_ex(dynts_cache_t* c, const int* seq_targets);
  *    current); make that first call before any stream capture begins. */
 dynts_status_t dynts_evict_noalloc(void* K, void* V, int* pos, float* score, int n_slabs, int head_dim, int dtype,
                                    int capacity, int n_rows, int n_pinned, int window, int target, void* stream);
+
+/* Scales of a DYNTS_BF16_KV8 cache (default 1, 1).  Host floats; k_scale, v_scale > 0 and finite.
+ * Allowed only while no sequence holds rows (DYNTS_ERR_STATE otherwise): stored codes are not
+ * re-encoded.  Choose scale ~ max|x| / 448 of the tensor to use the format's range. */
+dynts_status_t dynts_cache_set_kv_scale(dynts_cache_t* c, float k_scale, float v_scale);
 
 /* ---- predictor scores and the paper's own trigger ------------------------------------------ */
 

@@ -24,6 +24,7 @@ DYNTS_ERR_CUDA = 6
 DYNTS_ERR_DEVICE = 7
 DYNTS_BF16 = 0
 DYNTS_FP32 = 1
+DYNTS_BF16_KV8 = 2
 DYNTS_SCORE_ATTENTION = 0
 DYNTS_SCORE_EXTERNAL = 1
 
@@ -85,6 +86,7 @@ _sigs = {
     "dynts_cache_set_launch": (C.c_int, [_P, C.c_int, C.c_int]),
     "dynts_cache_launch_count": (C.c_longlong, [_P]),
     "dynts_cache_set_score_source": (C.c_int, [_P, C.c_int]),
+    "dynts_cache_set_kv_scale": (C.c_int, [_P, C.c_float, C.c_float]),
     "dynts_append_scores": (C.c_int, [_P, _P]),
     "dynts_evict_at_budget": (C.c_int, [_P, C.c_int, C.c_double]),
     "dynts_predictor_mlp_scratch_bytes": (C.c_size_t, [C.c_int, C.c_int]),
@@ -255,6 +257,10 @@ def dynts_cache_set_score_source(c, source):
     return _check(lib.dynts_cache_set_score_source(c, source))
 
 
+def dynts_cache_set_kv_scale(c, k_scale, v_scale):
+    return _check(lib.dynts_cache_set_kv_scale(c, float(k_scale), float(v_scale)))
+
+
 def dynts_append_scores(c, s_new):
     return _check(lib.dynts_append_scores(c, _ptr(s_new)))
 
@@ -294,10 +300,11 @@ class Cache:
         self.torch = torch
         self.device = torch.device(device)
         self.dtype_name = dtype
-        self.torch_dtype = {"bf16": torch.bfloat16, "fp32": torch.float32}[dtype]
+        self.torch_dtype = {"bf16": torch.bfloat16, "fp32": torch.float32, "bf16_kv8": torch.bfloat16}[dtype]   # q, k, v, out
+        self.slab_dtype = torch.uint8 if dtype == "bf16_kv8" else self.torch_dtype   # rows as exported (E4M3 codes)
         self.layers, self.batch, self.q_heads, self.kv_heads, self.head_dim = layers, batch, q_heads, kv_heads, head_dim
         cfg = make_config(layers, batch, q_heads, kv_heads, head_dim, budget, window, evict_interval,
-                          DYNTS_BF16 if dtype == "bf16" else DYNTS_FP32, capacity, seq_budgets)
+                          {"bf16": DYNTS_BF16, "fp32": DYNTS_FP32, "bf16_kv8": DYNTS_BF16_KV8}[dtype], capacity, seq_budgets)
         nbytes = dynts_cache_bytes(cfg)
         if nbytes == 0:
             raise DyntsError(DYNTS_ERR_INVALID_ARG, "invalid cache configuration")
@@ -374,6 +381,9 @@ class Cache:
     def set_score_source(self, source):
         return dynts_cache_set_score_source(self.handle, source)
 
+    def set_kv_scale(self, k_scale, v_scale):
+        return dynts_cache_set_kv_scale(self.handle, k_scale, v_scale)
+
     def append_scores(self, s_new):
         return dynts_append_scores(self.handle, s_new)
 
@@ -399,8 +409,8 @@ class Cache:
         """Host copies (K, V, pos, score) of one slab's n rows."""
         torch = self.torch
         n = self.len(seq)
-        K = torch.empty((n, self.head_dim), dtype=self.torch_dtype)
-        V = torch.empty((n, self.head_dim), dtype=self.torch_dtype)
+        K = torch.empty((n, self.head_dim), dtype=self.slab_dtype)
+        V = torch.empty((n, self.head_dim), dtype=self.slab_dtype)
         pos = torch.empty((n,), dtype=torch.int32)
         score = torch.empty((n,), dtype=torch.float32)
         m = dynts_cache_export(self.handle, layer, seq, head, K, V, pos, score)

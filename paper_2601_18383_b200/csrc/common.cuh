@@ -3,6 +3,7 @@
 
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 
 namespace dynts {
@@ -40,7 +41,9 @@ struct DecodeParams {
   int tile_tokens;    // rows of logits a CTA can hold in shared memory
   int slabs_per_cta;  // streaming kernel: > 0 => every CTA takes this many whole slabs
   int accumulate;     // 1: add each row's attention mass to its score (Eq. 6); 0: scores come from the caller
-  float scale_log2;   // log2(e) / sqrt(d)
+  float scale_log2;   // log2(e) / sqrt(d); times k_scale when the slabs hold 8-bit rows
+  float k_scale, v_scale;  // 8-bit slabs: a row is stored as e4m3(x / scale) and read as code value x scale
+  float out_scale;    // factor of the output (v_scale for 8-bit slabs, else 1)
 };
 
 struct EvictParams {
@@ -69,6 +72,27 @@ __device__ __forceinline__ float to_float(float x) { return x; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
 __device__ __forceinline__ void from_float(float* p, float x) { *p = x; }
 __device__ __forceinline__ void from_float(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+
+// 8-bit floats (E4M3: 1 sign, 4 exponent bits with bias 7, 3 mantissa bits, largest finite 448).
+// Two codes in a 16-bit word -> two halves (exact); low byte -> low half.
+__device__ __forceinline__ uint32_t e4m3x2_to_half2(unsigned short v) {
+  uint32_t h;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h) : "h"(v));
+  return h;
+}
+__device__ __forceinline__ float e4m3_to_float(uint8_t v) {
+  const uint32_t h = e4m3x2_to_half2((unsigned short)v);
+  return __half2float(__ushort_as_half((unsigned short)(h & 0xffffu)));
+}
+// Codes of lo and hi (round to nearest even, magnitudes beyond 448 saturate): lo in the low byte.
+__device__ __forceinline__ unsigned short float2_to_e4m3x2(float lo, float hi) {
+  unsigned short r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ uint8_t float_to_e4m3(float x) { return (uint8_t)(float2_to_e4m3x2(x, 0.f) & 0xffu); }
+// The code stored for a row element x of a slab with scale s (the division is IEEE fp32).
+__device__ __forceinline__ uint8_t store_e4m3(float x, float s) { return float_to_e4m3(__fdiv_rn(x, s)); }
 
 // Streaming 16-byte load that bypasses L1 allocation (each K/V byte is read once per step).
 __device__ __forceinline__ uint4 ldg_stream(const void* p) {

@@ -22,6 +22,8 @@
 #include <cooperative_groups.h>
 #include <math_constants.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace dynts {
@@ -106,7 +108,7 @@ __device__ __forceinline__ void cluster_epilogue(const DecodeParams& p, float* p
         const float orr = *cluster.map_shared_rank(part_O + e, r);
         acc += orr * fast_exp2(mr - M);
       }
-      from_float(out + e, acc * fin_f[g]);
+      from_float(out + e, acc * fin_f[g] * p.out_scale);
     }
   }
 
@@ -154,8 +156,11 @@ __device__ __forceinline__ void cluster_epilogue(const DecodeParams& p, float* p
 // ---------------------------------------------------------------------------------------------
 constexpr int kGenericThreads = 256;
 
-template <typename T>
+// KV8: the slabs hold E4M3 codes (q, k_new, v_new, out stay of type T); the new row is encoded before
+// anything reads it, so this step already sees the value later steps will see.
+template <typename T, bool KV8 = false>
 __global__ void __launch_bounds__(kGenericThreads) decode_attn_generic_kernel(const DecodeParams p) {
+  using TS = typename std::conditional<KV8, uint8_t, T>::type;  // slab element
   cg::cluster_group cluster = cg::this_cluster();
   const unsigned S = cluster.num_blocks();
   const unsigned rank = cluster.block_rank();
@@ -191,15 +196,24 @@ __global__ void __launch_bounds__(kGenericThreads) decode_attn_generic_kernel(co
   const T* q = reinterpret_cast<const T*>(p.q) + u.qoff;
   const T* knew = reinterpret_cast<const T*>(p.k_new) + u.kvoff;
   const T* vnew = reinterpret_cast<const T*>(p.v_new) + u.kvoff;
-  T* Ks = reinterpret_cast<T*>(p.K) + u.slab * (size_t)p.cap * d;
-  T* Vs = reinterpret_cast<T*>(p.V) + u.slab * (size_t)p.cap * d;
+  TS* Ks = reinterpret_cast<TS*>(p.K) + u.slab * (size_t)p.cap * d;
+  TS* Vs = reinterpret_cast<TS*>(p.V) + u.slab * (size_t)p.cap * d;
+  auto slab_val = [](TS x) -> float {
+    if constexpr (KV8) return e4m3_to_float(x);
+    else return to_float(x);
+  };
 
   for (int e = tid; e < G * d; e += kGenericThreads) sQ[e] = to_float(q[e]);
   // a1: append the new row (its score is written by the epilogue)
   if (n_old >= t_begin && n_old < t_end) {
     for (int c = tid; c < d; c += kGenericThreads) {
-      Ks[(size_t)n_old * d + c] = knew[c];
-      Vs[(size_t)n_old * d + c] = vnew[c];
+      if constexpr (KV8) {
+        Ks[(size_t)n_old * d + c] = store_e4m3(to_float(knew[c]), p.k_scale);
+        Vs[(size_t)n_old * d + c] = store_e4m3(to_float(vnew[c]), p.v_scale);
+      } else {
+        Ks[(size_t)n_old * d + c] = knew[c];
+        Vs[(size_t)n_old * d + c] = vnew[c];
+      }
     }
     if (tid == 0) p.pos[u.slab * (size_t)p.cap + n_old] = p.tot[u.b];
   }
@@ -207,12 +221,13 @@ __global__ void __launch_bounds__(kGenericThreads) decode_attn_generic_kernel(co
 
   // a2: logits, one warp per row
   for (int j = t_begin + warp; j < t_end; j += kGenericThreads / 32) {
-    const T* kr = (j == n_old) ? knew : Ks + (size_t)j * d;
     float acc[kMaxGroup];
 #pragma unroll
     for (int g = 0; g < kMaxGroup; ++g) acc[g] = 0.f;
     for (int c = lane; c < d; c += 32) {
-      const float kv = to_float(kr[c]);
+      float kv;
+      if constexpr (KV8) kv = slab_val(Ks[(size_t)j * d + c]);  // the appended row was written by this CTA above
+      else kv = (j == n_old) ? to_float(knew[c]) : slab_val(Ks[(size_t)j * d + c]);
 #pragma unroll
       for (int g = 0; g < kMaxGroup; ++g)
         if (g < G) acc[g] = fmaf(kv, sQ[g * d + c], acc[g]);
@@ -258,8 +273,9 @@ __global__ void __launch_bounds__(kGenericThreads) decode_attn_generic_kernel(co
     for (int g = 0; g < kMaxGroup; ++g) acc[g] = 0.f;
     if (tg < ngroups) {
       for (int j = t_begin + tg; j < t_end; j += ngroups) {
-        const T* vr = (j == n_old) ? vnew : Vs + (size_t)j * d;
-        const float vv = to_float(vr[c]);
+        float vv;
+        if constexpr (KV8) vv = slab_val(Vs[(size_t)j * d + c]);
+        else vv = (j == n_old) ? to_float(vnew[c]) : slab_val(Vs[(size_t)j * d + c]);
         const float* t = tile + (size_t)(j - t_begin) * G;
 #pragma unroll
         for (int g = 0; g < kMaxGroup; ++g)

@@ -51,7 +51,8 @@ bool stream_capable(const dynts_config_t* c) {
   return c->dtype == DYNTS_BF16 && c->head_dim == 128 && c->batch <= dynts::kStMaxBatch;
 }
 
-int elt_bytes_of(int dtype) { return dtype == DYNTS_FP32 ? 4 : 2; }
+int elt_bytes_of(int dtype) { return dtype == DYNTS_FP32 ? 4 : 2; }        // q, k, v, out
+int kv_elt_bytes_of(int dtype) { return dtype == DYNTS_BF16_KV8 ? 1 : elt_bytes_of(dtype); }  // slab rows
 
 bool config_ok(const dynts_config_t* c, int* cap_out) {
   if (!c) return false;
@@ -59,7 +60,8 @@ bool config_ok(const dynts_config_t* c, int* cap_out) {
   if (c->q_heads % c->kv_heads) return false;
   if (c->q_heads / c->kv_heads > dynts::kMaxGroup) return false;
   if (c->head_dim % 8 || c->head_dim > 256) return false;
-  if (c->dtype != DYNTS_BF16 && c->dtype != DYNTS_FP32) return false;
+  if (c->dtype != DYNTS_BF16 && c->dtype != DYNTS_FP32 && c->dtype != DYNTS_BF16_KV8) return false;
+  if (c->dtype == DYNTS_BF16_KV8 && c->head_dim % 16) return false;  // rows move in 16-byte pieces
   if (c->budget < 1 || c->window < 0 || c->window > c->budget || c->evict_interval < 1) return false;
   int maxb = c->budget;
   if (c->seq_budgets)
@@ -76,7 +78,7 @@ bool config_ok(const dynts_config_t* c, int* cap_out) {
 Layout make_layout(const dynts_config_t* c, int cap) {
   Layout L;
   const size_t slabs = (size_t)c->layers * c->batch * c->kv_heads;
-  const size_t kv = slabs * cap * c->head_dim * elt_bytes_of(c->dtype);
+  const size_t kv = slabs * cap * c->head_dim * kv_elt_bytes_of(c->dtype);
   size_t off = 0;
   auto take = [&](size_t bytes) {
     size_t o = off;
@@ -113,7 +115,9 @@ struct dynts_cache {
   dynts_config_t cfg;
   int cap = 0;
   int G = 1;
-  int elt = 2;
+  int elt = 2;               // bytes per element of q, k, v, out
+  int kv_elt = 2;            // bytes per element of the slab rows
+  float k_scale = 1.f, v_scale = 1.f;  // 8-bit slabs: stored code = e4m3(x / scale)
   bool ready = false;        // storage exists
   bool owns_storage = false;
   char* base = nullptr;
@@ -129,7 +133,7 @@ struct dynts_cache {
   // staging for the host-buffer entry point
   char* stage_dev = nullptr;
   size_t stage_bytes = 0;
-  bool attr_generic_f32 = false, attr_generic_bf16 = false, attr_mma = false, attr_select = false;
+  bool attr_generic_f32 = false, attr_generic_bf16 = false, attr_generic_kv8 = false, attr_mma = false, attr_select = false;
   bool attr_stream = false, attr_fused = false, attr_prefill = false;
   bool have_maps = false;    // tensor maps of the K and V slabs for the streaming kernel
   CUtensorMap map_K, map_V;
@@ -199,6 +203,7 @@ dynts_status_t materialise(dynts_cache* c) {
   c->cap = cap;
   c->G = c->cfg.q_heads / c->cfg.kv_heads;
   c->elt = elt_bytes_of(c->cfg.dtype);
+  c->kv_elt = kv_elt_bytes_of(c->cfg.dtype);
   c->lay = make_layout(&c->cfg, cap);
   if (c->cfg.storage) {
     if ((reinterpret_cast<uintptr_t>(c->cfg.storage) & 255u) != 0)
@@ -313,6 +318,14 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
   p.slabs_per_cta = 0;
   p.accumulate = c->score_source == 0 ? 1 : 0;
   p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)f.head_dim));
+  p.k_scale = c->k_scale;
+  p.v_scale = c->v_scale;
+  p.out_scale = 1.f;
+  const bool kv8 = f.dtype == DYNTS_BF16_KV8;
+  if (kv8) {
+    p.scale_log2 *= c->k_scale;
+    p.out_scale = c->v_scale;
+  }
 
   const bool mma_ok = f.dtype == DYNTS_BF16 && f.head_dim == 128 && c->G <= 8;
   const bool stream_ok = mma_ok && c->have_maps;
@@ -391,6 +404,14 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
     lc.blockDim = dim3(dynts::kMmaThreads, 1, 1);
     lc.dynamicSmemBytes = smem;
     e = cudaLaunchKernelEx(&lc, dynts::decode_attn_mma_kernel, p);
+  } else if (kv8) {
+    const size_t smem = dynts::generic_smem_bytes(c->G, f.head_dim, tile_tokens);
+    dynts_status_t st =
+        ensure_smem_attr(dynts::decode_attn_generic_kernel<__nv_bfloat16, true>, smem, &c->attr_generic_kv8, true);
+    if (st != DYNTS_OK) return st;
+    lc.blockDim = dim3(dynts::kGenericThreads, 1, 1);
+    lc.dynamicSmemBytes = smem;
+    e = cudaLaunchKernelEx(&lc, dynts::decode_attn_generic_kernel<__nv_bfloat16, true>, p);
   } else if (f.dtype == DYNTS_FP32) {
     const size_t smem = dynts::generic_smem_bytes(c->G, f.head_dim, tile_tokens);
     dynts_status_t st = ensure_smem_attr(dynts::decode_attn_generic_kernel<float>, smem, &c->attr_generic_f32, true);
@@ -451,12 +472,15 @@ dynts_status_t do_prefill(dynts_cache* c, int seq, const void* k, const void* v,
   p.Hkv = c->cfg.kv_heads;
   p.d = c->cfg.head_dim;
   p.cap = c->cap;
-  p.elt_bytes = c->elt;
+  p.elt_bytes = c->kv_elt;
+  p.kv8 = c->cfg.dtype == DYNTS_BF16_KV8 ? 1 : 0;
+  p.k_scale = c->k_scale;
+  p.v_scale = c->v_scale;
   p.T = T;
   p.n_pinned = n_pinned;
   p.seq = seq;
   const unsigned ny = (unsigned)(seq < 0 ? c->slabs() : (size_t)c->cfg.layers * c->cfg.kv_heads);
-  const size_t pieces = (size_t)T * c->cfg.head_dim * c->elt / 16;
+  const size_t pieces = (size_t)T * c->cfg.head_dim * c->elt / 16;  // 16-byte pieces of the source
   const unsigned nx = (unsigned)std::max<size_t>(1, std::min<size_t>(64, (pieces + 255) / 256));
   dynts::prefill_kernel<<<dim3(nx, ny, 1), 256, 0, c->stream>>>(p);
   CUDA_TRY(cudaGetLastError());
@@ -507,7 +531,7 @@ dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validat
   p.d = c->cfg.head_dim;
   p.cap = c->cap;
   p.window = c->cfg.window;
-  p.elt_bytes = c->elt;
+  p.elt_bytes = c->kv_elt;
   if (global) {
     // one score per token: sum the slab scores of each sequence, every slab then ranks by the sum
     if (c->cap > 10000) return fail(DYNTS_ERR_CAPACITY, "sequence-wide selection supports up to 10000 rows per slab");
@@ -541,7 +565,7 @@ dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validat
     if (st != DYNTS_OK) return st;
     dynts::evict_select_kernel<<<(unsigned)c->slabs(), dynts::kSelectThreads, smem, c->stream>>>(p);
     CUDA_TRY(cudaGetLastError());
-    const int pieces = c->cfg.head_dim * c->elt / 16;
+    const int pieces = c->cfg.head_dim * c->kv_elt / 16;
     const unsigned groups = (unsigned)((pieces + 3) / 4);
     dynts::evict_compact_kernel<<<dim3(2 * groups, (unsigned)c->slabs(), 1), dynts::kCompactThreads, 0, c->stream>>>(p);
     CUDA_TRY(cudaGetLastError());
@@ -646,8 +670,8 @@ dynts_status_t dynts_prefill_attn(dynts_cache_t* c, const void* q, const void* k
   if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
   if (!q || !out || !aligned16(q) || !aligned16(out))
     return fail(DYNTS_ERR_INVALID_ARG, "q and out must be non-NULL and 16-byte aligned");
-  if (c->cfg.dtype != DYNTS_BF16 || c->cfg.head_dim != 128)
-    return fail(DYNTS_ERR_INVALID_ARG, "prefill attention needs bf16 and head_dim 128");
+  if ((c->cfg.dtype != DYNTS_BF16 && c->cfg.dtype != DYNTS_BF16_KV8) || c->cfg.head_dim != 128)
+    return fail(DYNTS_ERR_INVALID_ARG, "prefill attention needs bf16 q/k/v and head_dim 128");
   if (n_tokens < 1) return fail(DYNTS_ERR_INVALID_ARG, "n_tokens must be positive");
   dynts_status_t st = do_prefill(c, -1, k, v, n_tokens, n_pinned);  // rows, positions, pins
   if (st != DYNTS_OK) return st;
@@ -805,7 +829,7 @@ dynts_status_t dynts_cache_export(dynts_cache_t* c, int layer, int seq, int head
   CUDA_TRY(cudaStreamSynchronize(c->stream));
   const size_t slab = ((size_t)layer * c->cfg.batch + seq) * c->cfg.kv_heads + head;
   const int rows = c->len_h[seq];
-  const size_t row_bytes = (size_t)c->cfg.head_dim * c->elt;
+  const size_t row_bytes = (size_t)c->cfg.head_dim * c->kv_elt;
   if (K) CUDA_TRY(cudaMemcpy(K, static_cast<char*>(c->K()) + slab * c->cap * row_bytes, rows * row_bytes, cudaMemcpyDeviceToHost));
   if (V) CUDA_TRY(cudaMemcpy(V, static_cast<char*>(c->V()) + slab * c->cap * row_bytes, rows * row_bytes, cudaMemcpyDeviceToHost));
   if (pos) CUDA_TRY(cudaMemcpy(pos, c->pos() + slab * c->cap, rows * sizeof(int), cudaMemcpyDeviceToHost));
@@ -827,7 +851,7 @@ dynts_status_t dynts_cache_import(dynts_cache_t* c, int layer, int seq, int head
   if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "import in the middle of a layer-by-layer step");
   CUDA_TRY(cudaStreamSynchronize(c->stream));
   const size_t slab = ((size_t)layer * c->cfg.batch + seq) * c->cfg.kv_heads + head;
-  const size_t row_bytes = (size_t)c->cfg.head_dim * c->elt;
+  const size_t row_bytes = (size_t)c->cfg.head_dim * c->kv_elt;
   CUDA_TRY(cudaMemcpy(static_cast<char*>(c->K()) + slab * c->cap * row_bytes, K, n * row_bytes, cudaMemcpyHostToDevice));
   CUDA_TRY(cudaMemcpy(static_cast<char*>(c->V()) + slab * c->cap * row_bytes, V, n * row_bytes, cudaMemcpyHostToDevice));
   CUDA_TRY(cudaMemcpy(c->pos() + slab * c->cap, pos, n * sizeof(int), cudaMemcpyHostToDevice));
@@ -885,6 +909,19 @@ dynts_status_t dynts_cache_set_score_source(dynts_cache_t* c, int source) {
     return fail(DYNTS_ERR_INVALID_ARG, "score source must be DYNTS_SCORE_ATTENTION or DYNTS_SCORE_EXTERNAL");
   if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "a layer-by-layer step is in progress");
   c->score_source = source;
+  return DYNTS_OK;
+}
+
+dynts_status_t dynts_cache_set_kv_scale(dynts_cache_t* c, float k_scale, float v_scale) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (c->cfg.dtype != DYNTS_BF16_KV8) return fail(DYNTS_ERR_INVALID_ARG, "the cache does not hold 8-bit rows");
+  if (!(k_scale > 0.f) || !(v_scale > 0.f) || std::isinf(k_scale) || std::isinf(v_scale))
+    return fail(DYNTS_ERR_INVALID_ARG, "scales must be positive and finite (%g, %g)", (double)k_scale, (double)v_scale);
+  if (c->ready)
+    for (int b = 0; b < c->cfg.batch; ++b)
+      if (c->len_h[b] > 0) return fail(DYNTS_ERR_STATE, "rows are already stored with the current scales");
+  c->k_scale = k_scale;
+  c->v_scale = v_scale;
   return DYNTS_OK;
 }
 
@@ -1090,8 +1127,10 @@ dynts_status_t dynts_evict_noalloc(void* K, void* V, int* pos, float* score, int
                                    int capacity, int n_rows, int n_pinned, int window, int target, void* stream) {
   if (!K || !V || !pos || !score) return fail(DYNTS_ERR_INVALID_ARG, "NULL tensor pointer");
   if (!aligned16(K) || !aligned16(V)) return fail(DYNTS_ERR_INVALID_ARG, "K and V must be 16-byte aligned");
-  if (dtype != DYNTS_BF16 && dtype != DYNTS_FP32) return fail(DYNTS_ERR_INVALID_ARG, "unknown dtype %d", dtype);
-  if (n_slabs < 1 || head_dim < 8 || head_dim % 8 || head_dim > 256 || capacity < 1)
+  if (dtype != DYNTS_BF16 && dtype != DYNTS_FP32 && dtype != DYNTS_BF16_KV8)
+    return fail(DYNTS_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+  if (n_slabs < 1 || head_dim < 8 || head_dim % 8 || head_dim > 256 || capacity < 1 ||
+      (dtype == DYNTS_BF16_KV8 && head_dim % 16))
     return fail(DYNTS_ERR_INVALID_ARG, "bad shape: n_slabs %d head_dim %d capacity %d", n_slabs, head_dim, capacity);
   if (n_rows < 0 || n_rows > capacity || n_pinned < 0 || n_pinned > n_rows || window < 0 || target < 1)
     return fail(DYNTS_ERR_INVALID_ARG, "bad lengths: n_rows %d n_pinned %d window %d target %d", n_rows, n_pinned,
@@ -1142,7 +1181,7 @@ dynts_status_t dynts_evict_noalloc(void* K, void* V, int* pos, float* score, int
   p.d = head_dim;
   p.cap = capacity;
   p.window = window;
-  p.elt_bytes = elt_bytes_of(dtype);
+  p.elt_bytes = kv_elt_bytes_of(dtype);
   noalloc_setup_kernel<<<1, 1, 0, st>>>(base, n_rows, n_pinned, target);
   CUDA_TRY(cudaGetLastError());
   dynts::evict_select_kernel<<<(unsigned)n_slabs, dynts::kSelectThreads, (size_t)capacity * 8, st>>>(p);

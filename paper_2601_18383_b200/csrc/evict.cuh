@@ -480,6 +480,8 @@ struct PrefillParams {
   int* pinned;
   int* active;
   int L, Nb, Hkv, d, cap, elt_bytes, T, n_pinned, seq;
+  int kv8;                 // 1: k, v are bf16 and the slabs take their E4M3 codes (elt_bytes = 1)
+  float k_scale, v_scale;
 };
 
 __global__ void __launch_bounds__(256) prefill_kernel(const PrefillParams p) {
@@ -496,15 +498,35 @@ __global__ void __launch_bounds__(256) prefill_kernel(const PrefillParams p) {
   }
   const size_t slab = ((size_t)l * p.Nb + b) * p.Hkv + h;
   const size_t row_bytes = (size_t)p.d * p.elt_bytes;
-  const int pieces = (int)(row_bytes >> 4);
-  const char* ks = reinterpret_cast<const char*>(p.k) + (size_t)sl * p.T * row_bytes;
-  const char* vs = reinterpret_cast<const char*>(p.v) + (size_t)sl * p.T * row_bytes;
   char* Kd = reinterpret_cast<char*>(p.K) + slab * p.cap * row_bytes;
   char* Vd = reinterpret_cast<char*>(p.V) + slab * p.cap * row_bytes;
-  const size_t total = (size_t)p.T * pieces;
-  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
-    reinterpret_cast<uint4*>(Kd)[e] = reinterpret_cast<const uint4*>(ks)[e];
-    reinterpret_cast<uint4*>(Vd)[e] = reinterpret_cast<const uint4*>(vs)[e];
+  if (p.kv8) {
+    // 8 bf16 elements (16 bytes) in, 8 codes out per thread and step; rows are contiguous on both sides
+    const __nv_bfloat16* ks = reinterpret_cast<const __nv_bfloat16*>(p.k) + (size_t)sl * p.T * p.d;
+    const __nv_bfloat16* vs = reinterpret_cast<const __nv_bfloat16*>(p.v) + (size_t)sl * p.T * p.d;
+    const size_t total = (size_t)p.T * p.d / 8;
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+      const uint4 kin = reinterpret_cast<const uint4*>(ks)[e], vin = reinterpret_cast<const uint4*>(vs)[e];
+      const __nv_bfloat16* kb = reinterpret_cast<const __nv_bfloat16*>(&kin);
+      const __nv_bfloat16* vb = reinterpret_cast<const __nv_bfloat16*>(&vin);
+      uint32_t ko[2] = {0u, 0u}, vo[2] = {0u, 0u};
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        ko[i >> 2] |= (uint32_t)store_e4m3(__bfloat162float(kb[i]), p.k_scale) << (8 * (i & 3));
+        vo[i >> 2] |= (uint32_t)store_e4m3(__bfloat162float(vb[i]), p.v_scale) << (8 * (i & 3));
+      }
+      reinterpret_cast<uint2*>(Kd)[e] = make_uint2(ko[0], ko[1]);
+      reinterpret_cast<uint2*>(Vd)[e] = make_uint2(vo[0], vo[1]);
+    }
+  } else {
+    const int pieces = (int)(row_bytes >> 4);
+    const char* ks = reinterpret_cast<const char*>(p.k) + (size_t)sl * p.T * row_bytes;
+    const char* vs = reinterpret_cast<const char*>(p.v) + (size_t)sl * p.T * row_bytes;
+    const size_t total = (size_t)p.T * pieces;
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+      reinterpret_cast<uint4*>(Kd)[e] = reinterpret_cast<const uint4*>(ks)[e];
+      reinterpret_cast<uint4*>(Vd)[e] = reinterpret_cast<const uint4*>(vs)[e];
+    }
   }
   for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < p.T; t += gridDim.x * blockDim.x) {
     p.pos[slab * p.cap + t] = t;
