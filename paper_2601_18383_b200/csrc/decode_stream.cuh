@@ -1,5 +1,5 @@
 // Persistent streaming variant of the fused decode attention + importance accumulation
-// (Eq. 4-6) for sm_100a: bf16 slabs, head_dim 128, G <= 8.
+// (Eq. 4-6) for sm_100a: bf16 or 8-bit (E4M3) slabs, head_dim 128, G <= 8.
 //
 // Work decomposition.  Every slab (layer, sequence, KV head) of n rows is cut into chunks of 32
 // rows; the chunks of all slabs of the launch form one list, ordered slab by slab, and the
@@ -28,6 +28,16 @@
 // atomic, one writer per score row and per output element.  While a CTA still has chunks to
 // stream, that pass is handed to a sixth warp (the scorer) through a two-slot task queue in shared
 // memory, so the consumer warps go straight on to the next slab.
+//
+// 8-bit slabs (KV8 = true): a stage holds one 32 x 128-byte box of K codes and one of V codes.
+// ldmatrix moves bytes, so the same 8 x 16-byte matrices are fetched; a thread's 32-bit register
+// then holds four codes, which cvt.rn.f16x2.e4m3x2 turns (exactly) into two f16 pairs, and the
+// products run as f16 mma with fp32 accumulation.  For Q K^T the four codes of a register are four
+// consecutive head_dim indices of one token; a dot product does not care in which order head_dim
+// is summed, so the query fragment is simply loaded with the same permutation.  For P V the
+// transposed ldmatrix pairs two tokens of two adjacent columns in a register; a byte permute
+// regroups them into (token, token+1) pairs per column, and the accumulator rows are declared to be
+// columns 16mb + 2gid and 16mb + 2gid + 1.  q is converted to f16 (|q| must stay below 65504).
 #pragma once
 
 #include <cuda.h>
@@ -116,6 +126,27 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, u
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
                : "r"(addr));
+}
+__device__ __forceinline__ void mma_f16_m16n8k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                 uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// Four E4M3 codes in a register -> f16 pairs of bytes (0, 1) and (2, 3).
+__device__ __forceinline__ void e4m3x4_to_half2x2(uint32_t r, uint32_t& lo, uint32_t& hi) {
+  asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tcvt.rn.f16x2.e4m3x2 %0, l;\n\tcvt.rn.f16x2.e4m3x2 %1, h;\n\t}"
+      : "=r"(lo), "=r"(hi)
+      : "r"(r));
+}
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+  __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+// Two bf16 in a word -> the same two values as f16.
+__device__ __forceinline__ uint32_t bf16x2_to_half2(uint32_t w) {
+  return pack_half2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kStConsumers) : "memory"); }
 
@@ -260,7 +291,7 @@ __device__ __forceinline__ void score_pass(bool accumulate, float* score, float*
 // rescaled between groups, so the cost is one memory round trip per four contributors.
 template <int GG>
 __device__ __forceinline__ void combine_partials(const float* part, int p_first, int k, long long g0, long long per_cta,
-                                                 __nv_bfloat16* out, float* s_finM, float* s_finf, int tid) {
+                                                 __nv_bfloat16* out, float out_scale, float* s_finM, float* s_finf, int tid) {
   constexpr int d = 128;
   float M[GG], L[GG], acc[GG];
 #pragma unroll
@@ -310,7 +341,7 @@ __device__ __forceinline__ void combine_partials(const float* part, int p_first,
   }
 #pragma unroll
   for (int g = 0; g < GG; ++g) {
-    out[(size_t)g * d + tid] = __float2bfloat16_rn(acc[g] / L[g]);
+    out[(size_t)g * d + tid] = __float2bfloat16_rn(acc[g] / L[g] * out_scale);
     if (tid == 0) {
       s_finM[g] = M[g];
       s_finf[g] = 1.0f / L[g];
@@ -337,10 +368,13 @@ struct StScoreTask {
     default: { constexpr int GG = 8; CALL; } break; \
   }
 
+template <bool KV8>
 __global__ void __launch_bounds__(kStThreads, 2)
 decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmK,
                           const __grid_constant__ CUtensorMap tmV) {
   constexpr int d = 128;
+  constexpr int kTxBytes = KV8 ? 2 * kStBoxBytes : 4 * kStBoxBytes;  // bytes a stage receives
+  constexpr int kVBox = KV8 ? 1 : 2;                                   // index of the first V box of a stage
   const int G = p.G, Nb = p.Nb, Hkv = p.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -458,13 +492,18 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         }
         const uint32_t full = bar_full + 8 * stage;
         const uint32_t dst = smem_u32(s_stage + (size_t)stage * kStStageBytes);
-        mbar_arrive_expect_tx(full, kStStageBytes);
+        mbar_arrive_expect_tx(full, kTxBytes);
         s_flags[2 + stage] = 1 + (int)ph;  // phase of the loads now in flight, for the drain below
         const int row = (int)(slab * (size_t)p.cap) + c.chunk * kStRows;
-        tma_load_2d(dst, &tmK, 0, row, full, pol);
-        tma_load_2d(dst + kStBoxBytes, &tmK, 64, row, full, pol);
-        tma_load_2d(dst + 2 * kStBoxBytes, &tmV, 0, row, full, pol);
-        tma_load_2d(dst + 3 * kStBoxBytes, &tmV, 64, row, full, pol);
+        if constexpr (KV8) {
+          tma_load_2d(dst, &tmK, 0, row, full, pol);
+          tma_load_2d(dst + kStBoxBytes, &tmV, 0, row, full, pol);
+        } else {
+          tma_load_2d(dst, &tmK, 0, row, full, pol);
+          tma_load_2d(dst + kStBoxBytes, &tmK, 64, row, full, pol);
+          tma_load_2d(dst + 2 * kStBoxBytes, &tmV, 0, row, full, pol);
+          tma_load_2d(dst + 3 * kStBoxBytes, &tmV, 64, row, full, pol);
+        }
         if (++c.chunk == c.cb) cursor_next_slab(c, s_cnt, Nb, Hkv);
       }
     }
@@ -500,13 +539,21 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
 
       // Query fragments of the group, straight from global memory (2 KB at most, L2-resident):
       // a0 = Q[head gid][16kk + 2tig, +1], a2 = Q[head gid][16kk + 8 + 2tig, +1].
+      // (8-bit slabs: k-step kk covers head_dim 16kk..16kk+15 and this thread's four k-indices are
+      // 16kk + 4tig + {0, 1 | 2, 3}, the order in which its register of codes holds them; f16.)
       uint32_t qa[8][2];
       {
         const uint32_t* hq = reinterpret_cast<const uint32_t*>(reinterpret_cast<const __nv_bfloat16*>(p.q) + unit * (size_t)G * d);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
-          qa[kk][0] = gid < G ? __ldg(hq + gid * 64 + 8 * kk + tig) : 0u;
-          qa[kk][1] = gid < G ? __ldg(hq + gid * 64 + 8 * kk + 4 + tig) : 0u;
+          if constexpr (KV8) {
+            const uint2 w = gid < G ? __ldg(reinterpret_cast<const uint2*>(hq + gid * 64 + 8 * kk + 2 * tig)) : make_uint2(0u, 0u);
+            qa[kk][0] = bf16x2_to_half2(w.x);
+            qa[kk][1] = bf16x2_to_half2(w.y);
+          } else {
+            qa[kk][0] = gid < G ? __ldg(hq + gid * 64 + 8 * kk + tig) : 0u;
+            qa[kk][1] = gid < G ? __ldg(hq + gid * 64 + 8 * kk + 4 + tig) : 0u;
+          }
         }
       }
 
@@ -529,13 +576,38 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           if (n_old >= t0 && n_old < t0 + 16) {
             // a1: the appended row.  The tile holds whatever the slab had at row n_old; overwrite
             // it in shared memory with k_new / v_new and store the row to the slab.
-            const int r = n_old - row0, ch = lane & 15, isv = lane >> 4;
-            const __nv_bfloat16* nrow = reinterpret_cast<const __nv_bfloat16*>(isv ? p.v_new : p.k_new) + unit * d;
-            const uint4 val = __ldg(reinterpret_cast<const uint4*>(nrow) + ch);
-            uint8_t* box = st + (2 * isv + (ch >> 3)) * kStBoxBytes;
-            *reinterpret_cast<uint4*>(box + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = val;
-            __nv_bfloat16* grow = reinterpret_cast<__nv_bfloat16*>(isv ? p.V : p.K) + (slab * (size_t)p.cap + n_old) * d;
-            reinterpret_cast<uint4*>(grow)[ch] = val;
+            const int r = n_old - row0;
+            if constexpr (KV8) {
+              // lanes 0-15: 16-byte piece ch of the K (lanes 0-7) or V (8-15) row = 16 elements, encoded here
+              if (lane < 16) {
+                const int ch = lane & 7, isv = lane >> 3;
+                const __nv_bfloat16* nrow = reinterpret_cast<const __nv_bfloat16*>(isv ? p.v_new : p.k_new) + unit * d + 16 * ch;
+                const uint4 a = __ldg(reinterpret_cast<const uint4*>(nrow)), b = __ldg(reinterpret_cast<const uint4*>(nrow) + 1);
+                const float sc = isv ? p.v_scale : p.k_scale;
+                const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+                uint32_t o4[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const float f0 = __fdiv_rn(__uint_as_float(w[2 * i] << 16), sc);
+                  const float f1 = __fdiv_rn(__uint_as_float(w[2 * i] & 0xffff0000u), sc);
+                  const float f2 = __fdiv_rn(__uint_as_float(w[2 * i + 1] << 16), sc);
+                  const float f3 = __fdiv_rn(__uint_as_float(w[2 * i + 1] & 0xffff0000u), sc);
+                  o4[i] = (uint32_t)float2_to_e4m3x2(f0, f1) | ((uint32_t)float2_to_e4m3x2(f2, f3) << 16);
+                }
+                const uint4 val = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+                *reinterpret_cast<uint4*>(st + isv * kStBoxBytes + r * 128 + ((ch ^ (r & 7)) << 4)) = val;
+                uint8_t* grow = reinterpret_cast<uint8_t*>(isv ? p.V : p.K) + (slab * (size_t)p.cap + n_old) * d;
+                reinterpret_cast<uint4*>(grow)[ch] = val;
+              }
+            } else {
+              const int ch = lane & 15, isv = lane >> 4;
+              const __nv_bfloat16* nrow = reinterpret_cast<const __nv_bfloat16*>(isv ? p.v_new : p.k_new) + unit * d;
+              const uint4 val = __ldg(reinterpret_cast<const uint4*>(nrow) + ch);
+              uint8_t* box = st + (2 * isv + (ch >> 3)) * kStBoxBytes;
+              *reinterpret_cast<uint4*>(box + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = val;
+              __nv_bfloat16* grow = reinterpret_cast<__nv_bfloat16*>(isv ? p.V : p.K) + (slab * (size_t)p.cap + n_old) * d;
+              reinterpret_cast<uint4*>(grow)[ch] = val;
+            }
             if (lane == 0) {
               p.pos[slab * (size_t)p.cap + n_old] = p.tot[c.b];
               if (!p.accumulate) {  // external scores: the new row starts at 0 until the caller sets it
@@ -551,22 +623,53 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           // latency overlaps; the V fragments are fetched before the softmax arithmetic)
           float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
           const uint32_t kbase = smem_u32(st) + lrow * 128;
-          const uint32_t vbase = kbase + 2 * kStBoxBytes;
+          const uint32_t vbase = kbase + kVBox * kStBoxBytes;
           uint32_t fr[8][4];
+          if constexpr (KV8) {
+            // matrices of one ldmatrix: tokens 0-7 x piece 2j, tokens 0-7 x piece 2j+1, tokens 8-15 x the same
+            uint32_t kr[4][4];
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const int chk = ((2 * kk) & 7) + lchk;
-            ldmatrix_x4(kbase + (kk >> 2) * kStBoxBytes + ((chk ^ (lrow & 7)) << 4), fr[kk][0], fr[kk][1], fr[kk][2], fr[kk][3]);
-          }
+            for (int j = 0; j < 4; ++j)
+              ldmatrix_x4(kbase + (((2 * j + lchk) ^ (lrow & 7)) << 4), kr[j][0], kr[j][1], kr[j][2], kr[j][3]);
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            mma_bf16_m16n8k16(s0, qa[kk][0], 0u, qa[kk][1], 0u, fr[kk][0], fr[kk][1]);
-            mma_bf16_m16n8k16(s1, qa[kk][0], 0u, qa[kk][1], 0u, fr[kk][2], fr[kk][3]);
-          }
+            for (int j = 0; j < 4; ++j) {
 #pragma unroll
-          for (int mb = 0; mb < 8; ++mb) {
-            const int chk = ((2 * mb) & 7) + lchk;
-            ldmatrix_x4_trans(vbase + (mb >> 2) * kStBoxBytes + ((chk ^ (lrow & 7)) << 4), fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3]);
+              for (int h = 0; h < 2; ++h) {  // piece 2j + h = k-step kk
+                const int kk = 2 * j + h;
+                uint32_t b0, b1;
+                e4m3x4_to_half2x2(kr[j][h], b0, b1);
+                mma_f16_m16n8k16(s0, qa[kk][0], 0u, qa[kk][1], 0u, b0, b1);
+                e4m3x4_to_half2x2(kr[j][2 + h], b0, b1);
+                mma_f16_m16n8k16(s1, qa[kk][0], 0u, qa[kk][1], 0u, b0, b1);
+              }
+            }
+            // V: the transposed load gives (token 2tig, columns 2gid, 2gid+1 | token 2tig+1, the same columns)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint32_t v0, v1, v2, v3;  // tokens 0-7 x pieces 2j, 2j+1; tokens 8-15 x pieces 2j, 2j+1
+              ldmatrix_x4_trans(vbase + (((2 * j + lchk) ^ (lrow & 7)) << 4), v0, v1, v2, v3);
+              // -> (token, token+1) pairs of column 2gid (low half) and 2gid+1 (high half)
+              e4m3x4_to_half2x2(__byte_perm(v0, 0u, 0x3120), fr[2 * j][0], fr[2 * j][1]);
+              e4m3x4_to_half2x2(__byte_perm(v2, 0u, 0x3120), fr[2 * j][2], fr[2 * j][3]);
+              e4m3x4_to_half2x2(__byte_perm(v1, 0u, 0x3120), fr[2 * j + 1][0], fr[2 * j + 1][1]);
+              e4m3x4_to_half2x2(__byte_perm(v3, 0u, 0x3120), fr[2 * j + 1][2], fr[2 * j + 1][3]);
+            }
+          } else {
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+              const int chk = ((2 * kk) & 7) + lchk;
+              ldmatrix_x4(kbase + (kk >> 2) * kStBoxBytes + ((chk ^ (lrow & 7)) << 4), fr[kk][0], fr[kk][1], fr[kk][2], fr[kk][3]);
+            }
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+              mma_bf16_m16n8k16(s0, qa[kk][0], 0u, qa[kk][1], 0u, fr[kk][0], fr[kk][1]);
+              mma_bf16_m16n8k16(s1, qa[kk][0], 0u, qa[kk][1], 0u, fr[kk][2], fr[kk][3]);
+            }
+#pragma unroll
+            for (int mb = 0; mb < 8; ++mb) {
+              const int chk = ((2 * mb) & 7) + lchk;
+              ldmatrix_x4_trans(vbase + (mb >> 2) * kStBoxBytes + ((chk ^ (lrow & 7)) << 4), fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3]);
+            }
           }
           // a3: online softmax of head gid over the unit's 16 tokens
           const int tk = t0 + 2 * tig;
@@ -597,18 +700,20 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           const float p2 = fast_exp2(x[2] - m_safe), p3 = fast_exp2(x[3] - m_safe);
           l_part = l_part * corr + ((p0 + p1) + (p2 + p3));
           m_run = m_new;
-          const uint32_t pb0 = pack_bf16x2(p0, p1);  // B fragment: tokens 2tig, 2tig+1 of head gid
-          const uint32_t pb1 = pack_bf16x2(p2, p3);  // tokens 2tig+8, 2tig+9
+          const uint32_t pb0 = KV8 ? pack_half2(p0, p1) : pack_bf16x2(p0, p1);  // B fragment: tokens 2tig, 2tig+1 of head gid
+          const uint32_t pb1 = KV8 ? pack_half2(p2, p3) : pack_bf16x2(p2, p3);  // tokens 2tig+8, 2tig+9
           const float c_even = __shfl_sync(0xffffffffu, corr, 8 * tig);      // head 2tig
           const float c_odd = __shfl_sync(0xffffffffu, corr, 8 * tig + 4);   // head 2tig+1
           // a4: O^T[d][head] += V^T P; accumulator mb covers d = 16mb + gid (+8), heads 2tig, 2tig+1
+          // (8-bit slabs: d = 16mb + 2gid (+1); operand order a0..a3 = rows gid | gid+8, tokens 0-7 | 8-15)
 #pragma unroll
           for (int mb = 0; mb < 8; ++mb) {
             o[mb][0] *= c_even;
             o[mb][1] *= c_odd;
             o[mb][2] *= c_even;
             o[mb][3] *= c_odd;
-            mma_bf16_m16n8k16(o[mb], fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3], pb0, pb1);
+            if constexpr (KV8) mma_f16_m16n8k16(o[mb], fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3], pb0, pb1);
+            else mma_bf16_m16n8k16(o[mb], fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3], pb0, pb1);
           }
         }
         __syncwarp();
@@ -645,10 +750,12 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           float* c0 = s_comb + ((size_t)warp * 4 + 2 * (tig & 1)) * d;
 #pragma unroll
           for (int mb = 0; mb < 8; ++mb) {
-            c0[16 * mb + gid] = o[mb][0];
-            c0[d + 16 * mb + gid] = o[mb][1];
-            c0[16 * mb + 8 + gid] = o[mb][2];
-            c0[d + 16 * mb + 8 + gid] = o[mb][3];
+            const int ca = KV8 ? 16 * mb + 2 * gid : 16 * mb + gid;      // column of accumulator rows gid
+            const int cb2 = KV8 ? ca + 1 : ca + 8;                       // and gid + 8
+            c0[ca] = o[mb][0];
+            c0[d + ca] = o[mb][1];
+            c0[cb2] = o[mb][2];
+            c0[d + cb2] = o[mb][3];
           }
         }
         consumer_sync();  // also orders s_wm / s_wl
@@ -668,7 +775,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
               l += s_wl[w * 8 + g] * f;
             }
             if (exclusive) {
-              out[(size_t)g * d + tid] = __float2bfloat16_rn(acc / l);
+              out[(size_t)g * d + tid] = __float2bfloat16_rn(acc / l * p.out_scale);
               if (tid == 0) {
                 s_finM[g] = mc;
                 s_finf[g] = 1.0f / l;
@@ -703,7 +810,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         if (finish) {
           // Last arriver: combine the partials of CTAs p_first..p_last; thread tid does column tid.
           const int k = p_last - p_first + 1;
-          DYNTS_DISPATCH_GROUP(G, combine_partials<GG>(p.part, p_first, k, g0, per_cta, out, s_finM, s_finf, tid));
+          DYNTS_DISPATCH_GROUP(G, combine_partials<GG>(p.part, p_first, k, g0, per_cta, out, p.out_scale, s_finM, s_finf, tid));
         }
       }
       if (finish && need_pass) {

@@ -46,9 +46,9 @@ struct Layout {
   size_t K, V, pos, score, comp, agg, src, hdr, len, tot, pinned, target, active, ticket, logit, part, arrive, total;
 };
 
-// The streaming decode kernel covers bf16 slabs with head_dim 128.
+// The streaming decode kernel covers bf16 and 8-bit slabs with head_dim 128.
 bool stream_capable(const dynts_config_t* c) {
-  return c->dtype == DYNTS_BF16 && c->head_dim == 128 && c->batch <= dynts::kStMaxBatch;
+  return (c->dtype == DYNTS_BF16 || c->dtype == DYNTS_BF16_KV8) && c->head_dim == 128 && c->batch <= dynts::kStMaxBatch;
 }
 
 int elt_bytes_of(int dtype) { return dtype == DYNTS_FP32 ? 4 : 2; }        // q, k, v, out
@@ -177,14 +177,17 @@ dynts_status_t make_slab_maps(dynts_cache* c) {
   tensor_map_encode_fn encode = reinterpret_cast<tensor_map_encode_fn>(fn);
   const cuuint64_t rows = (cuuint64_t)c->slabs() * c->cap;
   if (rows >= ((cuuint64_t)1 << 31)) return DYNTS_OK;  // row coordinates are 32-bit: keep the cluster kernels
+  // bf16 rows: 256 bytes read as two boxes of 64 elements; 8-bit rows: 128 bytes, one box of 128 codes
+  const bool kv8 = c->cfg.dtype == DYNTS_BF16_KV8;
   const cuuint64_t dims[2] = {128, rows};
-  const cuuint64_t strides[1] = {256};
-  const cuuint32_t box[2] = {64, (cuuint32_t)dynts::kStRows};
+  const cuuint64_t strides[1] = {kv8 ? 128u : 256u};
+  const cuuint32_t box[2] = {kv8 ? 128u : 64u, (cuuint32_t)dynts::kStRows};
   const cuuint32_t estr[2] = {1, 1};
-  CUresult r1 = encode(&c->map_K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c->K(), dims, strides, box, estr,
+  const CUtensorMapDataType mtype = kv8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  CUresult r1 = encode(&c->map_K, mtype, 2, c->K(), dims, strides, box, estr,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  CUresult r2 = encode(&c->map_V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c->V(), dims, strides, box, estr,
+  CUresult r2 = encode(&c->map_V, mtype, 2, c->V(), dims, strides, box, estr,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r1 != CUDA_SUCCESS || r2 != CUDA_SUCCESS)
@@ -328,17 +331,20 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
   }
 
   const bool mma_ok = f.dtype == DYNTS_BF16 && f.head_dim == 128 && c->G <= 8;
-  const bool stream_ok = mma_ok && c->have_maps;
+  const bool stream_ok = (mma_ok || (kv8 && f.head_dim == 128 && c->G <= 8)) && c->have_maps;
   int variant = c->variant;
   if (variant == 0) variant = stream_ok ? 3 : (mma_ok ? 2 : 1);
+  if (variant == 2 && kv8) variant = 1;  // the cluster tensor-core kernel reads bf16 rows only
   if (variant == 2 && !mma_ok) return fail(DYNTS_ERR_INVALID_ARG, "tensor-core variant needs bf16, head_dim 128, G <= 8");
   if (variant == 3 && !stream_ok)
-    return fail(DYNTS_ERR_INVALID_ARG, "streaming variant needs bf16, head_dim 128, G <= 8, batch <= %d", dynts::kStMaxBatch);
+    return fail(DYNTS_ERR_INVALID_ARG, "streaming variant needs bf16 or 8-bit slabs, head_dim 128, G <= 8, batch <= %d",
+                dynts::kStMaxBatch);
 
   if (variant == 3) {
     const size_t smem = dynts::stream_smem_bytes(Nb);
+    auto* stream_kernel = kv8 ? dynts::decode_attn_stream_kernel<true> : dynts::decode_attn_stream_kernel<false>;
     if (!c->attr_stream) {
-      CUDA_TRY(cudaFuncSetAttribute(dynts::decode_attn_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      CUDA_TRY(cudaFuncSetAttribute(stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)dynts::stream_smem_bytes(dynts::kStMaxBatch)));
       c->attr_stream = true;
     }
@@ -375,7 +381,7 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
     sc.gridDim = dim3((unsigned)ctas, 1, 1);
     sc.blockDim = dim3(dynts::kStThreads, 1, 1);
     sc.dynamicSmemBytes = smem;
-    cudaError_t e = cudaLaunchKernelEx(&sc, dynts::decode_attn_stream_kernel, p, c->map_K, c->map_V);
+    cudaError_t e = cudaLaunchKernelEx(&sc, stream_kernel, p, c->map_K, c->map_V);
     if (e != cudaSuccess) return fail(DYNTS_ERR_CUDA, "decode launch (streaming, %d CTAs): %s", ctas, cudaGetErrorString(e));
     c->launches += 1;
     if (advance)

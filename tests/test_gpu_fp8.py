@@ -139,3 +139,62 @@ def test_scale_rules():
     plain.close()
     with pytest.raises(D.DyntsError):
         D.Cache(1, 1, 4, 1, 72, 64, 8, 8, dtype="bf16_kv8")          # rows of 72 bytes do not split into 16-byte pieces
+
+
+def _sampled_full_size(name, seed, rows, ks, vs, n_slabs, steps):
+    """Full-size cache in the launch configuration the benchmark times (streaming kernel): sampled
+    slabs are exported as codes before each step and the oracle recomputes them one by one."""
+    import paper_2601_18383_b200 as D
+    from workloads import gen
+    cfg = W.get_config(name)
+    gpu = D.Cache(cfg.layers, cfg.batch, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.budget, cfg.window,
+                  cfg.evict_interval, dtype="bf16_kv8", seq_budgets=cfg.seq_budgets)
+    gpu.set_kv_scale(ks, vs)
+    k, v = gen.torch_keys_values(cfg, seed, rows, "cuda:0")
+    gpu.prefill(k, v, n_pinned=cfg.prompt)
+    del k, v
+    r = np.random.default_rng(seed)
+    all_ = [(l, b, h) for l in range(cfg.layers) for b in range(cfg.batch) for h in range(cfg.kv_heads)]
+    slabs = [all_[i] for i in r.choice(len(all_), size=n_slabs, replace=False)] + [all_[0], all_[-1]]
+    ring = gen.torch_step_ring(cfg, seed, steps, "cuda:0")
+    out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda:0")
+    delta = torch.zeros((cfg.layers, cfg.batch, cfg.kv_heads, gpu.capacity), dtype=torch.float32, device="cuda:0")
+    G = cfg.group
+    worst = dict(out=0.0, delta=0.0)
+    for s in range(steps):
+        pre = {sl: gpu.export_slab(*sl) for sl in slabs}
+        q, k, v = ring[0][s], ring[1][s], ring[2][s]
+        gpu.decode_attn(q, k, v, out, delta)
+        gpu.synchronize()
+        gpu.poll_error()
+        qh, kh, vh = q.double().cpu().numpy(), k.float().cpu().numpy(), v.float().cpu().numpy()
+        og, dh = out.float().cpu().numpy(), delta.cpu().numpy()
+        for (l, b, h) in slabs:
+            Kc, Vc, _, _ = pre[(l, b, h)]
+            Kr = np.concatenate([O.fp8_e4m3_decode(Kc.numpy()) * float(np.float32(ks)), O.fp8_e4m3_store(kh[l, b, h], ks)[None]])
+            Vr = np.concatenate([O.fp8_e4m3_decode(Vc.numpy()) * float(np.float32(vs)), O.fp8_e4m3_store(vh[l, b, h], vs)[None]])
+            alpha = O.attention_weights(qh[l, b, h * G:(h + 1) * G], Kr)
+            o_ref = O.attention_output(alpha, Vr)
+            worst["out"] = max(worst["out"], H.rel_err_vectors(og[l, b, h * G:(h + 1) * G], o_ref))
+            worst["delta"] = max(worst["delta"], float(np.abs(dh[l, b, h, :Kr.shape[0]] - alpha.sum(axis=0)).max()))
+            Kn, Vn, _, _ = gpu.export_slab(l, b, h)                      # the appended row's codes
+            assert np.array_equal(Kn.numpy()[-1], O.fp8_e4m3_encode(kh[l, b, h] / np.float32(ks)))
+            assert np.array_equal(Vn.numpy()[-1], O.fp8_e4m3_encode(vh[l, b, h] / np.float32(vs)))
+            assert np.array_equal(Kn.numpy()[:-1], Kc.numpy())
+    return gpu, cfg, slabs, worst
+
+
+def test_config2_full_size_8_bit():
+    gpu, cfg, slabs, worst = _sampled_full_size("c2_llama8b", 5100, W.get_config("c2_llama8b").capacity - 3, 0.02, 0.05, 8, 3)
+    assert worst["out"] <= H.TOL_OUT["bf16"] and worst["delta"] <= H.TOL_DELTA, worst
+    assert gpu.len(0) == cfg.capacity
+    H.check_evict_bit_exact(gpu, cfg, 0, slabs=slabs)
+    assert gpu.len(0) == cfg.budget
+    gpu.close()
+
+
+def test_config3_full_size_8_bit():
+    gpu, cfg, slabs, worst = _sampled_full_size("c3_qwen7b", 5200, W.get_config("c3_qwen7b").budget + 7, 0.03125, 0.0625, 6, 3)
+    assert worst["out"] <= H.TOL_OUT["bf16"] and worst["delta"] <= H.TOL_DELTA, worst
+    gpu.close()
+    torch.cuda.empty_cache()
