@@ -106,12 +106,14 @@ def physical_gpu_index(local_index: int) -> int:
     return local_index
 
 
-def setup_cache(cfg, seed, device):
+def setup_cache(cfg, seed, device, kv8=False):
     """A cache in steady state: every sequence holds `budget` rows (the prompt rows pinned)."""
     import torch
     import paper_2601_18383_b200 as D
     cache = D.Cache(cfg.layers, cfg.batch, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.budget, cfg.window,
-                    cfg.evict_interval, dtype=cfg.dtype, seq_budgets=cfg.seq_budgets, device=device)
+                    cfg.evict_interval, dtype="bf16_kv8" if kv8 else cfg.dtype, seq_budgets=cfg.seq_budgets, device=device)
+    if kv8:
+        cache.set_kv_scale(1.0 / 32, 1.0 / 32)     # synthetic rows are O(1): well inside the format's range
     if cfg.seq_budgets:
         one = cfg.scaled(batch=1)
         for b in range(cfg.batch):
@@ -135,12 +137,17 @@ def run_ours(args, cfg, rank, world, device):
 
     E = cfg.evict_interval
     ring_n = 64
-    cache = setup_cache(cfg, 1000 * int(cfg.name[1]) + rank, device)
+    kv8 = args.kv_dtype == "fp8"
+    if kv8 and (cfg.dtype != "bf16" or cfg.head_dim % 16):
+        raise SystemExit("--kv-dtype fp8 needs a bf16 workload")
+    cache = setup_cache(cfg, 1000 * int(cfg.name[1]) + rank, device, kv8)
     q_ring, k_ring, v_ring = gen.torch_step_ring(cfg, 77 + rank, ring_n, device)
     out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=q_ring.dtype, device=device)
     stream = torch.cuda.current_stream(device)
     external = args.score_source == "external"
     bytes_per_slot = BYTES_PER_SLOT - 8 if external else BYTES_PER_SLOT   # no score read-modify-write
+    if kv8:
+        bytes_per_slot -= 2 * cfg.head_dim                                # K and V rows of head_dim bytes each
     if external:
         import paper_2601_18383_b200 as D
         cache.set_score_source(D.DYNTS_SCORE_EXTERNAL)
@@ -200,7 +207,7 @@ def run_ours(args, cfg, rank, world, device):
 
     # ---- per-kernel durations (separate pass: event pairs around every launch) -----------------
     Kp = min(K, 8 * E)
-    elt = 2 if cfg.dtype == "bf16" else 4
+    elt = 1 if kv8 else (2 if cfg.dtype == "bf16" else 4)
     row_move_bytes = 2 * (2 * cfg.head_dim * elt + 8)      # K row + V row + pos + score, read and written
     # One event pair per run of back-to-back decode launches (the E launches between two evictions)
     # and one per eviction: the average launch duration includes the gaps between launches, as in
@@ -235,7 +242,7 @@ def run_ours(args, cfg, rank, world, device):
                                                                  else " + importance accumulation)"),
         "bound": "hbm", "achieved": round(dec_gbs, 1), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
         "frac": round(dec_gbs / peak, 4),
-        "traffic": None if (NCU_TRAFFIC_RATIO is None or external or cfg.name != "c2_llama8b") else int(NCU_TRAFFIC_RATIO * algo_bytes),
+        "traffic": None if (NCU_TRAFFIC_RATIO is None or external or kv8 or cfg.name != "c2_llama8b") else int(NCU_TRAFFIC_RATIO * algo_bytes),
         "algorithmic_bytes_per_launch": int(algo_bytes), "avg_launch_us": round(dec_avg_ms * 1e3, 2),
         "launches_timed": dec_launches,
     }
@@ -293,7 +300,7 @@ def run_ours(args, cfg, rank, world, device):
 
     # ---- CPU baseline: the oracle, as it stands, on this machine's host cores (rank 0, N = 1) ------
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not kv8:
         cpu = oracle_baseline(cfg, cache, q_ring, k_ring, v_ring, budget_s=args.cpu_seconds)
 
     result = {
@@ -302,7 +309,7 @@ def run_ours(args, cfg, rank, world, device):
         "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": cfg.name, "layers": cfg.layers, "batch": cfg.batch, "q_heads": cfg.q_heads,
                    "kv_heads": cfg.kv_heads, "head_dim": cfg.head_dim, "budget": cfg.budget, "window": cfg.window,
-                   "evict_interval": E, "prompt_pinned": cfg.prompt, "dist": cfg.dist, "score_source": args.score_source, "selection": args.selection, "accumulate": "fp32 (softmax, output, scores)",
+                   "evict_interval": E, "prompt_pinned": cfg.prompt, "dist": cfg.dist, "score_source": args.score_source, "selection": args.selection, "kv_dtype": "e4m3 codes, scale 1/32" if kv8 else cfg.dtype, "accumulate": "fp32 (softmax, output, scores)",
                    "cache_bytes": cache.nbytes, "l2_policy": "inputs larger than L2 (KV cache %.0f MB vs 126 MB L2)" % (cache.nbytes / 1e6),
                    "replicas": world},
         "hbm_gbs_decode": round(dec_gbs, 1), "roofline": roofline, "evict": evict, "e2e": e2e,
@@ -502,6 +509,8 @@ def main():
                     help="attention: Eq. 6 mass accumulated online (default); external: one predictor score per token (Eq. 7)")
     ap.add_argument("--selection", default="slab", choices=["slab", "global"],
                     help="slab: every (layer, KV head) selects on its own scores; global: one selection per sequence")
+    ap.add_argument("--kv-dtype", default="bf16", choices=["bf16", "fp8"],
+                    help="fp8: the slabs hold E4M3 codes (q, k, v, out stay bf16); bf16 workloads only")
     ap.add_argument("--cluster", type=int, default=0)
     ap.add_argument("--variant", type=int, default=0)
     args = ap.parse_args()

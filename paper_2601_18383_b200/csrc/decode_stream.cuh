@@ -14,9 +14,10 @@
 // epilogue.  Chunk i of a CTA goes to stage i mod 6 and to the warp pair i mod 2; with an even
 // stage count every stage is always consumed by the same two warps, which is what makes the
 // parity wait on its barrier unambiguous (a waiter is never two phases away from the barrier).
-// The consumer warps take 16 rows each: QK^T and PV run on the tensor pipe
-// (mma.sync m16n8k16, bf16 in, fp32 accumulate) with operands fetched by ldmatrix from the
-// swizzled tiles, online softmax in registers.
+// The consumer warps take 16 rows each: K Q^T (the unit's 16 tokens on M, the heads on N) and
+// V^T P (head_dim on M, the heads on N) run on the tensor pipe (mma.sync m16n8k16, fp32
+// accumulate: 16 mma per unit, which is what bounds the consumers) with operands fetched by
+// ldmatrix from the swizzled tiles; online softmax in registers, P transposed by movmatrix.
 //
 // The final softmax normaliser of a slab is known only when all its chunks are done, and the
 // importance score needs the normalised weights (Eq. 6).  So every row's scaled logits go to a
@@ -139,6 +140,13 @@ __device__ __forceinline__ void e4m3x4_to_half2x2(uint32_t r, uint32_t& lo, uint
   asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tcvt.rn.f16x2.e4m3x2 %0, l;\n\tcvt.rn.f16x2.e4m3x2 %1, h;\n\t}"
       : "=r"(lo), "=r"(hi)
       : "r"(r));
+}
+// Transposes the 8x8 matrix of 16-bit elements a warp holds as one register per thread (row gid,
+// columns 2tig, 2tig+1): afterwards the thread holds elements [2tig][gid] and [2tig+1][gid].
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d_;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d_) : "r"(a));
+  return d_;
 }
 __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
   __half2 v = __floats2half2_rn(lo, hi);
@@ -562,7 +570,8 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
       for (int mb = 0; mb < 8; ++mb)
 #pragma unroll
         for (int e = 0; e < 4; ++e) o[mb][e] = 0.f;
-      float m_run = -CUDART_INF_F, l_part = 0.f;
+      // running max and sum of heads 2tig (A) and 2tig+1 (B); the sums cover this thread's tokens only
+      float mA_run = -CUDART_INF_F, mB_run = -CUDART_INF_F, lA = 0.f, lB = 0.f;
 
       for (int k = (pair ^ it) & 1; k < seg; k += 2) {
         const int item = it + k;  // item & 1 == pair
@@ -618,7 +627,8 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
           }
-          // a2: S^T[head][token] = Q K^T for two blocks of 8 tokens
+          // a2: S[token][head] = K Q^T: the unit's 16 tokens on M, the group's heads on N, one mma per
+          // 16 head_dim indices (two accumulators, summed, so that the chain of dependent mma is half as long)
           // (all fragment loads of a phase are issued before its mma chain, so their shared-memory
           // latency overlaps; the V fragments are fetched before the softmax arithmetic)
           float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
@@ -633,15 +643,13 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
               ldmatrix_x4(kbase + (((2 * j + lchk) ^ (lrow & 7)) << 4), kr[j][0], kr[j][1], kr[j][2], kr[j][3]);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-#pragma unroll
-              for (int h = 0; h < 2; ++h) {  // piece 2j + h = k-step kk
-                const int kk = 2 * j + h;
-                uint32_t b0, b1;
-                e4m3x4_to_half2x2(kr[j][h], b0, b1);
-                mma_f16_m16n8k16(s0, qa[kk][0], 0u, qa[kk][1], 0u, b0, b1);
-                e4m3x4_to_half2x2(kr[j][2 + h], b0, b1);
-                mma_f16_m16n8k16(s1, qa[kk][0], 0u, qa[kk][1], 0u, b0, b1);
-              }
+              uint32_t a0, a1, a2, a3;  // piece 2j = k-step 2j: (tokens 0-7 | 8-15) x (codes 0, 1 | 2, 3 of the register)
+              e4m3x4_to_half2x2(kr[j][0], a0, a2);
+              e4m3x4_to_half2x2(kr[j][2], a1, a3);
+              mma_f16_m16n8k16(s0, a0, a1, a2, a3, qa[2 * j][0], qa[2 * j][1]);
+              e4m3x4_to_half2x2(kr[j][1], a0, a2);
+              e4m3x4_to_half2x2(kr[j][3], a1, a3);
+              mma_f16_m16n8k16(s1, a0, a1, a2, a3, qa[2 * j + 1][0], qa[2 * j + 1][1]);
             }
             // V: the transposed load gives (token 2tig, columns 2gid, 2gid+1 | token 2tig+1, the same columns)
 #pragma unroll
@@ -655,15 +663,16 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
               e4m3x4_to_half2x2(__byte_perm(v3, 0u, 0x3120), fr[2 * j + 1][2], fr[2 * j + 1][3]);
             }
           } else {
+            // registers of one ldmatrix: tokens 0-7 x k 0-7, tokens 0-7 x k 8-15, tokens 8-15 x the same
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk) {
               const int chk = ((2 * kk) & 7) + lchk;
               ldmatrix_x4(kbase + (kk >> 2) * kStBoxBytes + ((chk ^ (lrow & 7)) << 4), fr[kk][0], fr[kk][1], fr[kk][2], fr[kk][3]);
             }
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-              mma_bf16_m16n8k16(s0, qa[kk][0], 0u, qa[kk][1], 0u, fr[kk][0], fr[kk][1]);
-              mma_bf16_m16n8k16(s1, qa[kk][0], 0u, qa[kk][1], 0u, fr[kk][2], fr[kk][3]);
+            for (int kk = 0; kk < 8; kk += 2) {
+              mma_bf16_m16n8k16(s0, fr[kk][0], fr[kk][2], fr[kk][1], fr[kk][3], qa[kk][0], qa[kk][1]);
+              mma_bf16_m16n8k16(s1, fr[kk + 1][0], fr[kk + 1][2], fr[kk + 1][1], fr[kk + 1][3], qa[kk + 1][0], qa[kk + 1][1]);
             }
 #pragma unroll
             for (int mb = 0; mb < 8; ++mb) {
@@ -671,39 +680,41 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
               ldmatrix_x4_trans(vbase + (mb >> 2) * kStBoxBytes + ((chk ^ (lrow & 7)) << 4), fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3]);
             }
           }
-          // a3: online softmax of head gid over the unit's 16 tokens
-          const int tk = t0 + 2 * tig;
+          // a3: online softmax.  This thread holds tokens gid and gid+8 of heads 2tig and 2tig+1.
+          const int tkA = t0 + gid, tkB = tkA + 8;
+          const bool hA = 2 * tig < G, hB = 2 * tig + 1 < G;
           float x[4];
-          x[0] = (gid < G && tk < n) ? s0[0] * p.scale_log2 : -CUDART_INF_F;
-          x[1] = (gid < G && tk + 1 < n) ? s0[1] * p.scale_log2 : -CUDART_INF_F;
-          x[2] = (gid < G && tk + 8 < n) ? s1[0] * p.scale_log2 : -CUDART_INF_F;
-          x[3] = (gid < G && tk + 9 < n) ? s1[1] * p.scale_log2 : -CUDART_INF_F;
-          if (gid < G && need_pass) {
-            float* t = lg + (size_t)gid * p.cap + tk;  // tk is even: 8-byte stores when the row base allows
-            if ((p.cap & 1) == 0 && tk + 9 < n) {
-              *reinterpret_cast<float2*>(t) = make_float2(x[0], x[1]);
-              *reinterpret_cast<float2*>(t + 8) = make_float2(x[2], x[3]);
-            } else {
-              if (tk < n) t[0] = x[0];
-              if (tk + 1 < n) t[1] = x[1];
-              if (tk + 8 < n) t[8] = x[2];
-              if (tk + 9 < n) t[9] = x[3];
-            }
+          x[0] = (hA && tkA < n) ? (s0[0] + s1[0]) * p.scale_log2 : -CUDART_INF_F;
+          x[1] = (hB && tkA < n) ? (s0[1] + s1[1]) * p.scale_log2 : -CUDART_INF_F;
+          x[2] = (hA && tkB < n) ? (s0[2] + s1[2]) * p.scale_log2 : -CUDART_INF_F;
+          x[3] = (hB && tkB < n) ? (s0[3] + s1[3]) * p.scale_log2 : -CUDART_INF_F;
+          if (need_pass) {
+            float* ta = lg + (size_t)(2 * tig) * p.cap;  // a warp's store covers 8 consecutive rows of 4 heads
+            float* tb = ta + p.cap;
+            if (hA && tkA < n) ta[tkA] = x[0];
+            if (hB && tkA < n) tb[tkA] = x[1];
+            if (hA && tkB < n) ta[tkB] = x[2];
+            if (hB && tkB < n) tb[tkB] = x[3];
           }
-          float um = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
-          um = fmaxf(um, __shfl_xor_sync(0xffffffffu, um, 1));
-          um = fmaxf(um, __shfl_xor_sync(0xffffffffu, um, 2));
-          const float m_new = fmaxf(m_run, um);
-          const float m_safe = (m_new == -CUDART_INF_F) ? 0.f : m_new;
-          const float corr = fast_exp2(m_run - m_safe);
-          const float p0 = fast_exp2(x[0] - m_safe), p1 = fast_exp2(x[1] - m_safe);
-          const float p2 = fast_exp2(x[2] - m_safe), p3 = fast_exp2(x[3] - m_safe);
-          l_part = l_part * corr + ((p0 + p1) + (p2 + p3));
-          m_run = m_new;
-          const uint32_t pb0 = KV8 ? pack_half2(p0, p1) : pack_bf16x2(p0, p1);  // B fragment: tokens 2tig, 2tig+1 of head gid
-          const uint32_t pb1 = KV8 ? pack_half2(p2, p3) : pack_bf16x2(p2, p3);  // tokens 2tig+8, 2tig+9
-          const float c_even = __shfl_sync(0xffffffffu, corr, 8 * tig);      // head 2tig
-          const float c_odd = __shfl_sync(0xffffffffu, corr, 8 * tig + 4);   // head 2tig+1
+          float umA = fmaxf(x[0], x[2]), umB = fmaxf(x[1], x[3]);
+#pragma unroll
+          for (int o_ = 4; o_ < 32; o_ <<= 1) {  // over the unit's tokens: lanes of equal tig
+            umA = fmaxf(umA, __shfl_xor_sync(0xffffffffu, umA, o_));
+            umB = fmaxf(umB, __shfl_xor_sync(0xffffffffu, umB, o_));
+          }
+          const float mA_new = fmaxf(mA_run, umA), mB_new = fmaxf(mB_run, umB);
+          const float mA_safe = (mA_new == -CUDART_INF_F) ? 0.f : mA_new;
+          const float mB_safe = (mB_new == -CUDART_INF_F) ? 0.f : mB_new;
+          const float c_even = fast_exp2(mA_run - mA_safe), c_odd = fast_exp2(mB_run - mB_safe);
+          const float p0 = fast_exp2(x[0] - mA_safe), p1 = fast_exp2(x[1] - mB_safe);
+          const float p2 = fast_exp2(x[2] - mA_safe), p3 = fast_exp2(x[3] - mB_safe);
+          lA = lA * c_even + (p0 + p2);
+          lB = lB * c_odd + (p1 + p3);
+          mA_run = mA_new;
+          mB_run = mB_new;
+          // P[token][head] -> the B fragment of P V (tokens 2tig, 2tig+1 | +8 of head gid): an 8x8 transpose per half
+          const uint32_t pb0 = movmatrix_trans(KV8 ? pack_half2(p0, p1) : pack_bf16x2(p0, p1));
+          const uint32_t pb1 = movmatrix_trans(KV8 ? pack_half2(p2, p3) : pack_bf16x2(p2, p3));
           // a4: O^T[d][head] += V^T P; accumulator mb covers d = 16mb + gid (+8), heads 2tig, 2tig+1
           // (8-bit slabs: d = 16mb + 2gid (+1); operand order a0..a3 = rows gid | gid+8, tokens 0-7 | 8-15)
 #pragma unroll
@@ -721,11 +732,16 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
       }
 
       // ---- segment end: warp partials -> CTA partial ---------------------------------------------
-      l_part += __shfl_xor_sync(0xffffffffu, l_part, 1);
-      l_part += __shfl_xor_sync(0xffffffffu, l_part, 2);
-      if (tig == 0) {
-        s_wm[warp * 8 + gid] = m_run;
-        s_wl[warp * 8 + gid] = l_part;
+#pragma unroll
+      for (int o_ = 4; o_ < 32; o_ <<= 1) {  // sums over the tokens held by the lanes of equal tig
+        lA += __shfl_xor_sync(0xffffffffu, lA, o_);
+        lB += __shfl_xor_sync(0xffffffffu, lB, o_);
+      }
+      if (gid == 0) {
+        s_wm[warp * 8 + 2 * tig] = mA_run;
+        s_wm[warp * 8 + 2 * tig + 1] = mB_run;
+        s_wl[warp * 8 + 2 * tig] = lA;
+        s_wl[warp * 8 + 2 * tig + 1] = lB;
       }
       // Who else works on this slab?  Chunk g0 is its first one.
       const long long g0 = g_begin + it - c.chunk;
