@@ -51,6 +51,7 @@ namespace dynts {
 
 constexpr int kStRows = 32;                      // rows per chunk = per ring stage
 constexpr int kStStages = 6;                     // even: chunk i of a CTA goes to stage i % 6 and to the warp pair i % 2,
+constexpr int kStStages8 = 12;                   // 8-bit slabs: stages of half the bytes, twice as many (the same bytes in flight)
                                                  // so every stage is always consumed by the same two warps
 constexpr int kStConsumerWarps = 4;
 constexpr int kStConsumers = kStConsumerWarps * 32;
@@ -65,7 +66,7 @@ constexpr uint32_t kStSpinLimit = 1u << 22;      // bounded mbarrier polling
 
 __host__ __device__ inline size_t stream_smem_bytes(int Nb) {
   return 1024 /* alignment slack */ + (size_t)kStStages * kStStageBytes + sizeof(float) * kStCombFloats +
-         sizeof(float) * (2 * kStConsumerWarps * 8 + kStConsumerWarps * 8 + 4 * 8) + 16 * kStStages + 64 + 256 +
+         sizeof(float) * (2 * kStConsumerWarps * 8 + kStConsumerWarps * 8 + 4 * 8) + 16 * kStStages8 + 128 + 256 +
          sizeof(int) * (2 * (size_t)Nb + 2);
 }
 
@@ -381,7 +382,8 @@ __global__ void __launch_bounds__(kStThreads, 2)
 decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmK,
                           const __grid_constant__ CUtensorMap tmV) {
   constexpr int d = 128;
-  constexpr int kTxBytes = KV8 ? 2 * kStBoxBytes : 4 * kStBoxBytes;  // bytes a stage receives
+  constexpr int kTxBytes = KV8 ? 2 * kStBoxBytes : 4 * kStBoxBytes;  // bytes a stage holds and receives
+  constexpr int NS = KV8 ? kStStages8 : kStStages;                    // ring stages (NS * kTxBytes = 96 KB either way)
   constexpr int kVBox = KV8 ? 1 : 2;                                   // index of the first V box of a stage
   const int G = p.G, Nb = p.Nb, Hkv = p.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -389,7 +391,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
   extern __shared__ uint8_t st_smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(st_smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* s_stage = sm;                                             // [stages][4 boxes]
-  float* s_comb = reinterpret_cast<float*>(s_stage + kStStages * kStStageBytes);  // [warps][4 heads][128]
+  float* s_comb = reinterpret_cast<float*>(s_stage + NS * kTxBytes);  // [warps][4 heads][128]
   float* s_wm = s_comb + kStCombFloats;                              // [warps][8]
   float* s_wl = s_wm + kStConsumerWarps * 8;
   float* s_sc = s_wl + kStConsumerWarps * 8;                         // [warps][8] rescale of each warp's partial
@@ -398,20 +400,20 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
   float* s_finM = s_cl + 8;                                          // [8] slab max
   float* s_finf = s_finM + 8;                                        // [8] 1 / slab sum
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_finf + 8);         // full[stages], empty[stages]
-  int* s_flags = reinterpret_cast<int*>(s_bar + 2 * kStStages);      // [0] abort, [1] last arriver, [2+s] armed phase, [8] uniform chunk count, [10] pass handed off
-  int* s_cnt = s_flags + 16;                                         // [Nb]
+  int* s_flags = reinterpret_cast<int*>(s_bar + 2 * NS);      // [0] abort, [1] last arriver, [8] uniform chunk count, [10] pass handed off, [16+s] armed phase of stage s
+  int* s_cnt = s_flags + 32;                                         // [Nb]
   int* s_off = s_cnt + Nb;                                           // [Nb + 1]
   // hand-off of score passes to the scorer warp: two task slots and their full/empty barriers
   uint64_t* s_tbar = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(s_off + Nb + 1) + 15) & ~(uintptr_t)15);
   StScoreTask* s_task = reinterpret_cast<StScoreTask*>(s_tbar + 4);
   volatile int* s_abort = s_flags;
 
-  const uint32_t bar_full = smem_u32(s_bar), bar_empty = smem_u32(s_bar + kStStages);
+  const uint32_t bar_full = smem_u32(s_bar), bar_empty = smem_u32(s_bar + NS);
   const uint32_t tbar_full = smem_u32(s_tbar), tbar_empty = smem_u32(s_tbar + 2);
 
   // ---- per-CTA set-up: barriers and the chunk prefix of the sequences -------------------------
   if (tid == 0) {
-    for (int s = 0; s < kStStages; ++s) {
+    for (int s = 0; s < NS; ++s) {
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, 2);  // the two warps that consume the stage
     }
@@ -420,6 +422,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
       mbar_init(tbar_empty + 8 * s, 1);
     }
     for (int i = 0; i < 8; ++i) s_flags[i] = 0;  // (s_flags[8] belongs to the prefix warp below)
+    for (int i = 16; i < 32; ++i) s_flags[i] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -482,15 +485,15 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
       StCursor c;
       cursor_seek(c, g_begin, s_off, s_cnt, Nb);
       const uint64_t pol = l2_evict_first_policy();
+      int n_old = p.len[c.b];  // re-read only when the cursor moves to another sequence's slab
       for (int it = 0; it < cnt; ++it) {
-        const int stage = it % kStStages;
-        const uint32_t ph = (uint32_t)(it / kStStages) & 1u;
+        const int stage = it % NS;
+        const uint32_t ph = (uint32_t)(it / NS) & 1u;
         mbar_wait(bar_empty + 8 * stage, ph ^ 1u, s_abort, p.err);
         if (*s_abort) break;
         const size_t slab = ((size_t)(p.layer0 + c.lrel) * Nb + c.b) * Hkv + c.h;
-        const int n_old = p.len[c.b];
         if (c.lrel >= p.n_layers || c.b >= Nb || c.h >= Hkv || n_old + 1 > p.cap || (c.chunk + 1) * kStRows > p.cap + kStRows ||
-            (smem_u32(s_stage + (size_t)stage * kStStageBytes) & 1023u) != 0u) {
+            (smem_u32(s_stage + (size_t)stage * kTxBytes) & 1023u) != 0u) {
           // the chunk list and the slab bounds disagree: record, stop feeding, let the waits expire
           atomicOr(p.err, kErrStreamBounds);
           p.dbg[0] = c.lrel; p.dbg[1] = c.b; p.dbg[2] = c.h; p.dbg[3] = c.chunk; p.dbg[4] = n_old; p.dbg[5] = it;
@@ -499,9 +502,9 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           break;
         }
         const uint32_t full = bar_full + 8 * stage;
-        const uint32_t dst = smem_u32(s_stage + (size_t)stage * kStStageBytes);
+        const uint32_t dst = smem_u32(s_stage + (size_t)stage * kTxBytes);
         mbar_arrive_expect_tx(full, kTxBytes);
-        s_flags[2 + stage] = 1 + (int)ph;  // phase of the loads now in flight, for the drain below
+        s_flags[16 + stage] = 1 + (int)ph;  // phase of the loads now in flight, for the drain below
         const int row = (int)(slab * (size_t)p.cap) + c.chunk * kStRows;
         if constexpr (KV8) {
           tma_load_2d(dst, &tmK, 0, row, full, pol);
@@ -512,7 +515,10 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           tma_load_2d(dst + 2 * kStBoxBytes, &tmV, 0, row, full, pol);
           tma_load_2d(dst + 3 * kStBoxBytes, &tmV, 64, row, full, pol);
         }
-        if (++c.chunk == c.cb) cursor_next_slab(c, s_cnt, Nb, Hkv);
+        if (++c.chunk == c.cb && it + 1 < cnt) {
+          cursor_next_slab(c, s_cnt, Nb, Hkv);
+          n_old = p.len[c.b];
+        }
       }
     }
   } else if (cnt > 0 && warp < kStConsumerWarps) {
@@ -575,11 +581,11 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
 
       for (int k = (pair ^ it) & 1; k < seg; k += 2) {
         const int item = it + k;  // item & 1 == pair
-        const int stage = item % kStStages;
+        const int stage = item % NS;
         const int row0 = (c.chunk + k) * kStRows;
-        mbar_wait(bar_full + 8 * stage, (uint32_t)(item / kStStages) & 1u, s_abort, p.err);
+        mbar_wait(bar_full + 8 * stage, (uint32_t)(item / NS) & 1u, s_abort, p.err);
         __syncwarp();
-        uint8_t* st = s_stage + (size_t)stage * kStStageBytes;
+        uint8_t* st = s_stage + (size_t)stage * kTxBytes;
         const int t0 = row0 + u16;  // first row of this warp's unit
         if (t0 < n) {
           if (n_old >= t0 && n_old < t0 + 16) {
@@ -717,12 +723,19 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           const uint32_t pb1 = movmatrix_trans(KV8 ? pack_half2(p2, p3) : pack_bf16x2(p2, p3));
           // a4: O^T[d][head] += V^T P; accumulator mb covers d = 16mb + gid (+8), heads 2tig, 2tig+1
           // (8-bit slabs: d = 16mb + 2gid (+1); operand order a0..a3 = rows gid | gid+8, tokens 0-7 | 8-15)
+          // (once the running maxima have settled, which is after the first few units of a slab, the
+          // rescale factors are exactly 1 and the 32 multiplications are skipped)
+          if (!__all_sync(0xffffffffu, (c_even == 1.0f || !hA) && (c_odd == 1.0f || !hB))) {  // (padding heads hold zeros)
+#pragma unroll
+            for (int mb = 0; mb < 8; ++mb) {
+              o[mb][0] *= c_even;
+              o[mb][1] *= c_odd;
+              o[mb][2] *= c_even;
+              o[mb][3] *= c_odd;
+            }
+          }
 #pragma unroll
           for (int mb = 0; mb < 8; ++mb) {
-            o[mb][0] *= c_even;
-            o[mb][1] *= c_odd;
-            o[mb][2] *= c_even;
-            o[mb][3] *= c_odd;
             if constexpr (KV8) mma_f16_m16n8k16(o[mb], fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3], pb0, pb1);
             else mma_bf16_m16n8k16(o[mb], fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3], pb0, pb1);
           }
@@ -896,8 +909,8 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
   // then give the loads in flight a bounded time to land before the shared memory is released.
   __syncthreads();
   if (*s_abort && tid == 0) {
-    for (int s = 0; s < kStStages; ++s) {
-      const int armed = s_flags[2 + s];
+    for (int s = 0; s < NS; ++s) {
+      const int armed = s_flags[16 + s];
       if (armed == 0) continue;
       for (uint32_t i = 0; i < kStSpinLimit; ++i)
         if (mbar_try_wait(bar_full + 8 * s, (uint32_t)(armed - 1))) break;
