@@ -365,7 +365,11 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
       const long long slabs = (long long)n_layers * n_active * f.kv_heads;
       const long long per = (slabs + ctas - 1) / ctas;
       const long long used = (slabs + per - 1) / per;
-      if (uniform && used * 5 >= (long long)ctas * 4) {
+      // (bf16 slabs: the launch is HBM-bound, so 80 % of the CTA slots are enough and the combine is
+      // what one saves; 8-bit slabs: a CTA's own pipeline bounds it, so idle slots cost throughput
+      // unless the launch is so short -- a slab or two per CTA -- that the combine would cost more)
+      const bool mostly = used * 5 >= (long long)ctas * 4, nearly_all = used * 20 >= (long long)ctas * 19;
+      if (uniform && (kv8 ? (nearly_all || (mostly && per <= 2)) : mostly)) {
         p.slabs_per_cta = (int)per;
         ctas = (int)used;
       }
