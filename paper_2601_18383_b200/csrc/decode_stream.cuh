@@ -118,6 +118,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar), "l"(policy)
       : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar,
+                                            uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(policy)
+      : "memory");
+}
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
@@ -379,12 +387,15 @@ struct StScoreTask {
 
 template <bool KV8>
 __global__ void __launch_bounds__(kStThreads, 2)
-decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmK,
-                          const __grid_constant__ CUtensorMap tmV) {
+decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmKV) {
   constexpr int d = 128;
   constexpr int kTxBytes = KV8 ? 2 * kStBoxBytes : 4 * kStBoxBytes;  // bytes a stage holds and receives
   constexpr int NS = KV8 ? kStStages8 : kStStages;                    // ring stages (NS * kTxBytes = 96 KB either way)
-  constexpr int kVBox = KV8 ? 1 : 2;                                   // index of the first V box of a stage
+  // A stage holds the boxes [K, V] (8-bit rows) or [K low half, V low half, K high half, V high half]
+  // of head_dim (bf16 rows): one tile load brings the K box and the V box of the same columns.
+  constexpr int kHalf = 2 * kStBoxBytes;                               // bf16: offset of the high-half boxes
+  // Stages are released to the producer in groups: one wait of the producer thread per group.
+  constexpr int kGS = KV8 ? 4 : 2, kNG = NS / kGS;
   const int G = p.G, Nb = p.Nb, Hkv = p.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -415,7 +426,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
       mbar_init(bar_full + 8 * s, 1);
-      mbar_init(bar_empty + 8 * s, 2);  // the two warps that consume the stage
+      mbar_init(bar_empty + 8 * s, 2 * kGS);  // (used for s < kNG) the two warps that consume each stage of group s
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(tbar_full + 8 * s, 1);
@@ -430,8 +441,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
   // launch): nothing above touches global memory; everything below waits until that kernel has
   // completed and its writes are visible.
   if (tid == 32) {  // the descriptors are kernel parameters: fetching them needs no earlier kernel
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmK)) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmV)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmKV)) : "memory");
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (warp == 1) {
@@ -481,43 +491,56 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
 
   if (cnt > 0 && warp == kStConsumerWarps) {
     // =========================== producer: one thread feeds the ring ===========================
+    // Every barrier operation and tile-load issue costs this one thread a few hundred cycles of
+    // latency, and its rate bounds the CTA.  So per chunk it does only: arm the stage's barrier,
+    // issue one load (two for bf16 rows) that brings the K and the V box together, bump counters.
+    // It waits for free stages once per group of kGS stages, and everything that depends on the
+    // slab is recomputed only when the cursor moves to the next slab.
     if (lane == 0) {
       StCursor c;
       cursor_seek(c, g_begin, s_off, s_cnt, Nb);
       const uint64_t pol = l2_evict_first_policy();
-      int n_old = p.len[c.b];  // re-read only when the cursor moves to another sequence's slab
+      const uint32_t sbase = smem_u32(s_stage);
+      int stage = 0, grp = 0, in_grp = 0;
+      uint32_t ph = 0;  // parity of the round (it / NS)
+      int n_old = p.len[c.b];
+      int row = (int)((((size_t)(p.layer0 + c.lrel) * Nb + c.b) * Hkv + c.h) * (size_t)p.cap) + c.chunk * kStRows;
+      bool ok = c.lrel < p.n_layers && c.b < Nb && c.h < Hkv && n_old + 1 <= p.cap && c.cb * kStRows <= p.cap + kStRows &&
+                (sbase & 1023u) == 0u;
       for (int it = 0; it < cnt; ++it) {
-        const int stage = it % NS;
-        const uint32_t ph = (uint32_t)(it / NS) & 1u;
-        mbar_wait(bar_empty + 8 * stage, ph ^ 1u, s_abort, p.err);
-        if (*s_abort) break;
-        const size_t slab = ((size_t)(p.layer0 + c.lrel) * Nb + c.b) * Hkv + c.h;
-        if (c.lrel >= p.n_layers || c.b >= Nb || c.h >= Hkv || n_old + 1 > p.cap || (c.chunk + 1) * kStRows > p.cap + kStRows ||
-            (smem_u32(s_stage + (size_t)stage * kTxBytes) & 1023u) != 0u) {
+        if (in_grp == 0) {  // the group's stages of the previous round have all been consumed
+          mbar_wait(bar_empty + 8 * grp, ph ^ 1u, s_abort, p.err);
+          if (*s_abort) break;
+        }
+        if (!ok) {
           // the chunk list and the slab bounds disagree: record, stop feeding, let the waits expire
           atomicOr(p.err, kErrStreamBounds);
           p.dbg[0] = c.lrel; p.dbg[1] = c.b; p.dbg[2] = c.h; p.dbg[3] = c.chunk; p.dbg[4] = n_old; p.dbg[5] = it;
-          p.dbg[6] = (int)blockIdx.x; p.dbg[7] = (int)smem_u32(s_stage);
+          p.dbg[6] = (int)blockIdx.x; p.dbg[7] = (int)sbase;
           *s_abort = 1;
           break;
         }
         const uint32_t full = bar_full + 8 * stage;
-        const uint32_t dst = smem_u32(s_stage + (size_t)stage * kTxBytes);
+        const uint32_t dst = sbase + (uint32_t)stage * kTxBytes;
         mbar_arrive_expect_tx(full, kTxBytes);
         s_flags[16 + stage] = 1 + (int)ph;  // phase of the loads now in flight, for the drain below
-        const int row = (int)(slab * (size_t)p.cap) + c.chunk * kStRows;
-        if constexpr (KV8) {
-          tma_load_2d(dst, &tmK, 0, row, full, pol);
-          tma_load_2d(dst + kStBoxBytes, &tmV, 0, row, full, pol);
-        } else {
-          tma_load_2d(dst, &tmK, 0, row, full, pol);
-          tma_load_2d(dst + kStBoxBytes, &tmK, 64, row, full, pol);
-          tma_load_2d(dst + 2 * kStBoxBytes, &tmV, 0, row, full, pol);
-          tma_load_2d(dst + 3 * kStBoxBytes, &tmV, 64, row, full, pol);
+        tma_load_3d(dst, &tmKV, 0, row, 0, full, pol);
+        if constexpr (!KV8) tma_load_3d(dst + kHalf, &tmKV, 64, row, 0, full, pol);
+        row += kStRows;
+        ++stage;
+        if (++in_grp == kGS) {
+          in_grp = 0;
+          if (++grp == kNG) {
+            grp = 0;
+            stage = 0;
+            ph ^= 1u;
+          }
         }
         if (++c.chunk == c.cb && it + 1 < cnt) {
           cursor_next_slab(c, s_cnt, Nb, Hkv);
           n_old = p.len[c.b];
+          row = (int)((((size_t)(p.layer0 + c.lrel) * Nb + c.b) * Hkv + c.h) * (size_t)p.cap);
+          ok = c.lrel < p.n_layers && c.b < Nb && c.h < Hkv && n_old + 1 <= p.cap && c.cb * kStRows <= p.cap + kStRows;
         }
       }
     }
@@ -618,7 +641,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
               const int ch = lane & 15, isv = lane >> 4;
               const __nv_bfloat16* nrow = reinterpret_cast<const __nv_bfloat16*>(isv ? p.v_new : p.k_new) + unit * d;
               const uint4 val = __ldg(reinterpret_cast<const uint4*>(nrow) + ch);
-              uint8_t* box = st + (2 * isv + (ch >> 3)) * kStBoxBytes;
+              uint8_t* box = st + (isv + 2 * (ch >> 3)) * kStBoxBytes;
               *reinterpret_cast<uint4*>(box + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = val;
               __nv_bfloat16* grow = reinterpret_cast<__nv_bfloat16*>(isv ? p.V : p.K) + (slab * (size_t)p.cap + n_old) * d;
               reinterpret_cast<uint4*>(grow)[ch] = val;
@@ -639,7 +662,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           // latency overlaps; the V fragments are fetched before the softmax arithmetic)
           float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
           const uint32_t kbase = smem_u32(st) + lrow * 128;
-          const uint32_t vbase = kbase + kVBox * kStBoxBytes;
+          const uint32_t vbase = kbase + kStBoxBytes;
           uint32_t fr[8][4];
           if constexpr (KV8) {
             // matrices of one ldmatrix: tokens 0-7 x piece 2j, tokens 0-7 x piece 2j+1, tokens 8-15 x the same
@@ -673,7 +696,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk) {
               const int chk = ((2 * kk) & 7) + lchk;
-              ldmatrix_x4(kbase + (kk >> 2) * kStBoxBytes + ((chk ^ (lrow & 7)) << 4), fr[kk][0], fr[kk][1], fr[kk][2], fr[kk][3]);
+              ldmatrix_x4(kbase + (kk >> 2) * kHalf + ((chk ^ (lrow & 7)) << 4), fr[kk][0], fr[kk][1], fr[kk][2], fr[kk][3]);
             }
 #pragma unroll
             for (int kk = 0; kk < 8; kk += 2) {
@@ -683,7 +706,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
 #pragma unroll
             for (int mb = 0; mb < 8; ++mb) {
               const int chk = ((2 * mb) & 7) + lchk;
-              ldmatrix_x4_trans(vbase + (mb >> 2) * kStBoxBytes + ((chk ^ (lrow & 7)) << 4), fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3]);
+              ldmatrix_x4_trans(vbase + (mb >> 2) * kHalf + ((chk ^ (lrow & 7)) << 4), fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3]);
             }
           }
           // a3: online softmax.  This thread holds tokens gid and gid+8 of heads 2tig and 2tig+1.
@@ -741,7 +764,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar_empty + 8 * stage);
+        if (lane == 0) mbar_arrive(bar_empty + 8 * (stage / kGS));
       }
 
       // ---- segment end: warp partials -> CTA partial ---------------------------------------------

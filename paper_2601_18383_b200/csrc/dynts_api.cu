@@ -136,7 +136,7 @@ struct dynts_cache {
   bool attr_generic_f32 = false, attr_generic_bf16 = false, attr_generic_kv8 = false, attr_mma = false, attr_select = false;
   bool attr_stream = false, attr_fused = false, attr_prefill = false;
   bool have_maps = false;    // tensor maps of the K and V slabs for the streaming kernel
-  CUtensorMap map_K, map_V;
+  CUtensorMap map_KV;
   int sm_count = 0;
 
   void* K() const { return base + lay.K; }
@@ -163,8 +163,8 @@ namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Tensor maps (TMA descriptors) over all K rows and all V rows: a [slabs * cap][128] bf16 matrix
-// read in boxes of 32 rows x 64 columns with the 128-byte shared-memory swizzle.
+// Tensor map (TMA descriptor) over all K rows and all V rows, read in boxes of 32 rows with the
+// 128-byte shared-memory swizzle.
 typedef CUresult (*tensor_map_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                          const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                          CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -177,21 +177,20 @@ dynts_status_t make_slab_maps(dynts_cache* c) {
   tensor_map_encode_fn encode = reinterpret_cast<tensor_map_encode_fn>(fn);
   const cuuint64_t rows = (cuuint64_t)c->slabs() * c->cap;
   if (rows >= ((cuuint64_t)1 << 31)) return DYNTS_OK;  // row coordinates are 32-bit: keep the cluster kernels
-  // bf16 rows: 256 bytes read as two boxes of 64 elements; 8-bit rows: 128 bytes, one box of 128 codes
+  // One map over both tensors, [2 (K, V)][slabs * cap rows][128 elements], so that one tile load
+  // brings the K box and the V box of a chunk.  bf16 rows: 256 bytes read as boxes of 64 elements;
+  // 8-bit rows: 128 bytes, one box of 128 codes.
   const bool kv8 = c->cfg.dtype == DYNTS_BF16_KV8;
-  const cuuint64_t dims[2] = {128, rows};
-  const cuuint64_t strides[1] = {kv8 ? 128u : 256u};
-  const cuuint32_t box[2] = {kv8 ? 128u : 64u, (cuuint32_t)dynts::kStRows};
-  const cuuint32_t estr[2] = {1, 1};
+  const cuuint64_t kv_stride = (cuuint64_t)(static_cast<char*>(c->V()) - static_cast<char*>(c->K()));
+  if (kv_stride == 0 || (kv_stride & 15u) != 0 || kv_stride >= ((cuuint64_t)1 << 40)) return DYNTS_OK;  // keep the cluster kernels
+  const cuuint64_t dims[3] = {128, rows, 2};
+  const cuuint64_t strides[2] = {kv8 ? 128u : 256u, kv_stride};
+  const cuuint32_t box[3] = {kv8 ? 128u : 64u, (cuuint32_t)dynts::kStRows, 2};
+  const cuuint32_t estr[3] = {1, 1, 1};
   const CUtensorMapDataType mtype = kv8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-  CUresult r1 = encode(&c->map_K, mtype, 2, c->K(), dims, strides, box, estr,
-                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  CUresult r2 = encode(&c->map_V, mtype, 2, c->V(), dims, strides, box, estr,
-                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r1 != CUDA_SUCCESS || r2 != CUDA_SUCCESS)
-    return fail(DYNTS_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d, %d)", (int)r1, (int)r2);
+  CUresult r1 = encode(&c->map_KV, mtype, 3, c->K(), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r1 != CUDA_SUCCESS) return fail(DYNTS_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r1);
   int dev = 0;
   CUDA_TRY(cudaGetDevice(&dev));
   CUDA_TRY(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev));
@@ -385,7 +384,7 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
     sc.gridDim = dim3((unsigned)ctas, 1, 1);
     sc.blockDim = dim3(dynts::kStThreads, 1, 1);
     sc.dynamicSmemBytes = smem;
-    cudaError_t e = cudaLaunchKernelEx(&sc, stream_kernel, p, c->map_K, c->map_V);
+    cudaError_t e = cudaLaunchKernelEx(&sc, stream_kernel, p, c->map_KV);
     if (e != cudaSuccess) return fail(DYNTS_ERR_CUDA, "decode launch (streaming, %d CTAs): %s", ctas, cudaGetErrorString(e));
     c->launches += 1;
     if (advance)
