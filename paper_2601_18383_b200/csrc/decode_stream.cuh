@@ -91,6 +91,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Non-blocking test of a phase: the answer takes a few hundred cycles to come back, so it is asked
+// one unit of work ahead and only read when that work is done.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // Polls with an iteration limit.  On expiry the status word gets the timeout bit and the CTA-wide
 // abort flag is raised; every later wait of the CTA then returns at once, so the kernel ends (its
 // results are void, which the status word says).
@@ -555,6 +566,11 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
     cursor_seek(c, g_begin, s_off, s_cnt, Nb);
     int it = 0;
     int n_posted = 0;  // score passes handed to the scorer warp (thread 0's copy counts)
+    // The warp's next item is item + 2; whether its tile has landed is asked while this item is
+    // being worked on (a wait costs about 300 cycles even when the tile is long there).
+    bool peek_ok = false;  // the tile of this warp's next item was seen to have landed
+    int cs = pair;         // ring stage and phase parity of this warp's next item (its items are pair, pair + 2, ...)
+    uint32_t cp = 0;
     while (it < cnt) {
       // ---- one segment: chunks [c.chunk, c.chunk + seg) of one slab -----------------------------
       const int seg = min(c.cb - c.chunk, cnt - it);
@@ -604,10 +620,16 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
 
       for (int k = (pair ^ it) & 1; k < seg; k += 2) {
         const int item = it + k;  // item & 1 == pair
-        const int stage = item % NS;
+        const int stage = cs;     // == item % NS
         const int row0 = (c.chunk + k) * kStRows;
-        mbar_wait(bar_full + 8 * stage, (uint32_t)(item / NS) & 1u, s_abort, p.err);
+        if (!peek_ok) mbar_wait(bar_full + 8 * stage, cp, s_abort, p.err);
         __syncwarp();
+        cs += 2;
+        if (cs >= NS) {
+          cs -= NS;
+          cp ^= 1u;
+        }
+        if constexpr (KV8) peek_ok = item + 2 < cnt && mbar_test_wait(bar_full + 8 * cs, cp);  // (bf16 rows: HBM-bound, no gain)
         uint8_t* st = s_stage + (size_t)stage * kTxBytes;
         const int t0 = row0 + u16;  // first row of this warp's unit
         if (t0 < n) {
