@@ -122,7 +122,12 @@ dynts_status_t dynts_prefill_seq(dynts_cache_t* c, int seq, const void* k, const
  *   scores:        NULL, or device [L, Nb, Hkv, cap] fp32 that additionally receives this step's
  *                  mass per row (rows [0, n] of each slab are overwritten, the rest untouched).
  * The cache length of each active sequence grows by one.  DYNTS_ERR_CAPACITY if any active
- * sequence is already at capacity.  Rows of inactive sequences in `out` are left untouched. */
+ * sequence is already at capacity.  Rows of inactive sequences in `out` are left untouched.
+ * Stream capture: the library keeps a host copy of every sequence's length and hands it to the
+ * kernel with the launch; while the stream is being captured the kernel reads the lengths from
+ * device memory instead, so a captured step can be replayed.  Replays do not update the host
+ * copy: capture whole cycles that return to the lengths they started from (decode steps + the
+ * eviction), or do not mix replays that change the lengths with direct calls on the same cache. */
 dynts_status_t dynts_decode_attn(dynts_cache_t* c, const void* q, const void* k_new, const void* v_new,
                                  void* out, float* scores);
 

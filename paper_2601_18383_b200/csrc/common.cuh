@@ -9,6 +9,7 @@
 namespace dynts {
 
 constexpr int kMaxGroup = 8;        // query heads per KV head handled by the kernels
+constexpr int kHostLens = 64;       // batches up to this size get their lengths with the launch
 constexpr int kErrTileOverflow = 1; // device status bits
 constexpr int kErrLenOverflow = 2;
 constexpr int kErrEvictSmem = 4;
@@ -44,6 +45,12 @@ struct DecodeParams {
   float scale_log2;   // log2(e) / sqrt(d); times k_scale when the slabs hold 8-bit rows
   float k_scale, v_scale;  // 8-bit slabs: a row is stored as e4m3(x / scale) and read as code value x scale
   float out_scale;    // factor of the output (v_scale for 8-bit slabs, else 1)
+  // Streaming kernel: n_host > 0 => the rows per slab and the tokens seen so far of every sequence
+  // come with the launch (the host's mirror; -1 = inactive sequence) instead of being read from
+  // len / tot / active, and block 0 writes the advanced values back at once (no ticket at the end).
+  int n_host;
+  int len_host[kHostLens];
+  int tot_host[kHostLens];
 };
 
 struct EvictParams {

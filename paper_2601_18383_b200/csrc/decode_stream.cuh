@@ -67,7 +67,7 @@ constexpr uint32_t kStSpinLimit = 1u << 22;      // bounded mbarrier polling
 __host__ __device__ inline size_t stream_smem_bytes(int Nb) {
   return 1024 /* alignment slack */ + (size_t)kStStages * kStStageBytes + sizeof(float) * kStCombFloats +
          sizeof(float) * (2 * kStConsumerWarps * 8 + kStConsumerWarps * 8 + 4 * 8) + 16 * kStStages8 + 128 + 256 +
-         sizeof(int) * (2 * (size_t)Nb + 2);
+         sizeof(int) * (4 * (size_t)Nb + 2);
 }
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -425,8 +425,10 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
   int* s_flags = reinterpret_cast<int*>(s_bar + 2 * NS);      // [0] abort, [1] last arriver, [8] uniform chunk count, [10] pass handed off, [16+s] armed phase of stage s
   int* s_cnt = s_flags + 32;                                         // [Nb]
   int* s_off = s_cnt + Nb;                                           // [Nb + 1]
+  int* s_len = s_off + Nb + 1;                                       // [Nb] rows per slab before this step, -1: inactive
+  int* s_tot = s_len + Nb;                                           // [Nb] tokens seen so far (next position id)
   // hand-off of score passes to the scorer warp: two task slots and their full/empty barriers
-  uint64_t* s_tbar = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(s_off + Nb + 1) + 15) & ~(uintptr_t)15);
+  uint64_t* s_tbar = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(s_tot + Nb) + 15) & ~(uintptr_t)15);
   StScoreTask* s_task = reinterpret_cast<StScoreTask*>(s_tbar + 4);
   volatile int* s_abort = s_flags;
 
@@ -459,8 +461,23 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
     int carry = 0, cmin = 0x7fffffff, cmax = 0;
     for (int b0 = 0; b0 < Nb; b0 += 32) {
       const int b = b0 + lane;
-      int c = 0;
-      if (b < Nb && p.active[b]) c = (p.len[b] + 1 + kStRows - 1) / kStRows;
+      int ln = -1, tt = 0;
+      if (b < Nb) {
+        if (p.n_host > 0) {  // (constant indices: the parameter block is not copied to local memory)
+#pragma unroll
+          for (int i = 0; i < kHostLens; ++i)
+            if (i == b) {
+              ln = p.len_host[i];
+              tt = p.tot_host[i];
+            }
+        } else if (p.active[b]) {
+          ln = p.len[b];
+          tt = p.tot[b];
+        }
+        s_len[b] = ln;
+        s_tot[b] = tt;
+      }
+      const int c = ln >= 0 ? (ln + 1 + kStRows - 1) / kStRows : 0;
       if (c > 0) {
         cmin = min(cmin, c);
         cmax = max(cmax, c);
@@ -488,6 +505,14 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
     }
   }
   __syncthreads();
+  if (p.n_host > 0 && p.advance && blockIdx.x == 0 && warp == 0) {
+    // nobody in this launch reads the lengths from global memory: publish the advanced values now
+    for (int b = lane; b < Nb; b += 32)
+      if (s_len[b] >= 0) {
+        p.len[b] = s_len[b] + 1;
+        p.tot[b] = s_tot[b] + 1;
+      }
+  }
 
   const long long per_layer = s_off[Nb];
   const long long total = per_layer * p.n_layers;
@@ -514,7 +539,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
       const uint32_t sbase = smem_u32(s_stage);
       int stage = 0, grp = 0, in_grp = 0;
       uint32_t ph = 0;  // parity of the round (it / NS)
-      int n_old = p.len[c.b];
+      int n_old = s_len[c.b];
       int row = (int)((((size_t)(p.layer0 + c.lrel) * Nb + c.b) * Hkv + c.h) * (size_t)p.cap) + c.chunk * kStRows;
       bool ok = c.lrel < p.n_layers && c.b < Nb && c.h < Hkv && n_old + 1 <= p.cap && c.cb * kStRows <= p.cap + kStRows &&
                 (sbase & 1023u) == 0u;
@@ -549,7 +574,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         }
         if (++c.chunk == c.cb && it + 1 < cnt) {
           cursor_next_slab(c, s_cnt, Nb, Hkv);
-          n_old = p.len[c.b];
+          n_old = s_len[c.b];
           row = (int)((((size_t)(p.layer0 + c.lrel) * Nb + c.b) * Hkv + c.h) * (size_t)p.cap);
           ok = c.lrel < p.n_layers && c.b < Nb && c.h < Hkv && n_old + 1 <= p.cap && c.cb * kStRows <= p.cap + kStRows;
         }
@@ -576,7 +601,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
       const int seg = min(c.cb - c.chunk, cnt - it);
       const size_t unit = ((size_t)c.lrel * Nb + c.b) * Hkv + c.h;
       const size_t slab = ((size_t)(p.layer0 + c.lrel) * Nb + c.b) * Hkv + c.h;
-      const int n_old = p.len[c.b];
+      const int n_old = s_len[c.b];
       const int n = n_old + 1;
       float* lg = p.logit + slab * (size_t)G * p.cap;  // [G][cap]
       const bool need_pass = p.accumulate || p.delta_out != nullptr;  // else the logits are not needed again
@@ -669,7 +694,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
               reinterpret_cast<uint4*>(grow)[ch] = val;
             }
             if (lane == 0) {
-              p.pos[slab * (size_t)p.cap + n_old] = p.tot[c.b];
+              p.pos[slab * (size_t)p.cap + n_old] = s_tot[c.b];
               if (!p.accumulate) {  // external scores: the new row starts at 0 until the caller sets it
                 p.score[slab * (size_t)p.cap + n_old] = 0.f;
                 p.comp[slab * (size_t)p.cap + n_old] = 0.f;
@@ -961,7 +986,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         if (mbar_try_wait(bar_full + 8 * s, (uint32_t)(armed - 1))) break;
     }
   }
-  finish_ticket(p);
+  if (p.n_host == 0) finish_ticket(p);
 }
 
 }  // namespace dynts

@@ -125,7 +125,7 @@ struct dynts_cache {
   cudaStream_t stream = nullptr;
   int* err_host = nullptr;   // pinned, mapped
   int* err_dev = nullptr;
-  std::vector<int> seq_budget, len_h, pinned_h, target_h, active_h;
+  std::vector<int> seq_budget, len_h, tot_h, pinned_h, target_h, active_h;  // host mirrors of the per-sequence state
   int layer_cursor = 0;      // next layer expected by dynts_decode_attn_layer
   int cluster = 0, variant = 0;
   int score_source = 0;      // 0: attention mass accumulates (Eq. 6); 1: the caller supplies scores (Eq. 7)
@@ -239,6 +239,7 @@ dynts_status_t materialise(dynts_cache* c) {
     for (int b = 0; b < Nb; ++b) c->seq_budget[b] = c->cfg.seq_budgets[b];
   c->cfg.seq_budgets = nullptr;  // the caller's array is not kept
   c->len_h.assign(Nb, 0);
+  c->tot_h.assign(Nb, 0);
   c->pinned_h.assign(Nb, 0);
   c->active_h.assign(Nb, 1);
   c->target_h = c->seq_budget;
@@ -329,6 +330,19 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
     p.out_scale = c->v_scale;
   }
 
+  // Lengths with the launch (streaming kernel): not while the stream is being captured, since a
+  // replayed graph would carry the lengths of the capture.
+  p.n_host = 0;
+  if (Nb <= dynts::kHostLens) {
+    cudaStreamCaptureStatus cap_status = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(c->stream, &cap_status) == cudaSuccess && cap_status == cudaStreamCaptureStatusNone) {
+      p.n_host = Nb;
+      for (int b = 0; b < dynts::kHostLens; ++b) {
+        p.len_host[b] = (b < Nb && c->active_h[b]) ? c->len_h[b] : -1;
+        p.tot_host[b] = b < Nb ? c->tot_h[b] : 0;
+      }
+    }
+  }
   const bool mma_ok = f.dtype == DYNTS_BF16 && f.head_dim == 128 && c->G <= 8;
   const bool stream_ok = (mma_ok || (kv8 && f.head_dim == 128 && c->G <= 8)) && c->have_maps;
   int variant = c->variant;
@@ -389,7 +403,10 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
     c->launches += 1;
     if (advance)
       for (int b = 0; b < Nb; ++b)
-        if (c->active_h[b]) c->len_h[b] += 1;
+        if (c->active_h[b]) {
+          c->len_h[b] += 1;
+          c->tot_h[b] += 1;
+        }
     return DYNTS_OK;
   }
 
@@ -441,7 +458,10 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
   c->launches += 1;
   if (advance)
     for (int b = 0; b < Nb; ++b)
-      if (c->active_h[b]) c->len_h[b] += 1;
+      if (c->active_h[b]) {
+          c->len_h[b] += 1;
+          c->tot_h[b] += 1;
+        }
   return DYNTS_OK;
 }
 
@@ -497,6 +517,7 @@ dynts_status_t do_prefill(dynts_cache* c, int seq, const void* k, const void* v,
   for (int b = 0; b < c->cfg.batch; ++b) {
     if (seq >= 0 && b != seq) continue;
     c->len_h[b] = T;
+    c->tot_h[b] = T;
     c->pinned_h[b] = n_pinned;
     c->active_h[b] = 1;
   }
@@ -810,6 +831,7 @@ dynts_status_t dynts_seq_reset(dynts_cache_t* c, int seq) {
   CUDA_TRY(cudaMemsetAsync(c->pinned() + seq, 0, sizeof(int), c->stream));
   CUDA_TRY(cudaMemsetAsync(c->active() + seq, 0, sizeof(int), c->stream));
   c->len_h[seq] = 0;
+  c->tot_h[seq] = 0;
   c->pinned_h[seq] = 0;
   c->active_h[seq] = 0;
   return DYNTS_OK;
@@ -873,6 +895,7 @@ dynts_status_t dynts_cache_import(dynts_cache_t* c, int layer, int seq, int head
   CUDA_TRY(cudaMemcpy(c->pinned() + seq, &n_pinned, sizeof(int), cudaMemcpyHostToDevice));
   CUDA_TRY(cudaMemcpy(c->active() + seq, &one, sizeof(int), cudaMemcpyHostToDevice));
   c->len_h[seq] = n;
+  c->tot_h[seq] = next;
   c->pinned_h[seq] = n_pinned;
   c->active_h[seq] = 1;
   return DYNTS_OK;
