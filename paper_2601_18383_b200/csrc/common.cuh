@@ -49,6 +49,14 @@ struct DecodeParams {
   // come with the launch (the host's mirror; -1 = inactive sequence) instead of being read from
   // len / tot / active, and block 0 writes the advanced values back at once (no ticket at the end).
   int n_host;
+  // Streaming kernel, whole-slab pieces: defer = 1 => the score pass of a CTA's last slab is not run
+  // at the end of the launch (where nothing overlaps it) but recorded in pend[slab] = {n, n_old,
+  // M[8], 1/L[8]} and run by the scorer warp of the next launch, beside its streaming, from the
+  // other half of the logit scratch (logit_prev).  The host runs the recorded passes itself
+  // (flush_pending_kernel) before anything else touches the scores.
+  int defer;
+  float* logit_prev;
+  int* pend;          // [slabs][20]
   int len_host[kHostLens];
   int tot_host[kHostLens];
 };

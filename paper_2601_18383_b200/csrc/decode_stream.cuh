@@ -63,6 +63,7 @@ constexpr int kStMaxCtas = 320;                  // partial slots exist for this
 constexpr int kStPartStride = 8 * 128 + 16;      // floats per partial: O[8][128], m[8], l[8]
 constexpr int kStMaxBatch = 512;                 // sequences whose chunk prefix fits shared memory
 constexpr uint32_t kStSpinLimit = 1u << 22;      // bounded mbarrier polling
+constexpr int kStPendWords = 20;                 // a recorded score pass: n, n_old, M[8], 1/L[8], 2 spare
 
 __host__ __device__ inline size_t stream_smem_bytes(int Nb) {
   return 1024 /* alignment slack */ + (size_t)kStStages * kStStageBytes + sizeof(float) * kStCombFloats +
@@ -429,7 +430,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
   int* s_tot = s_len + Nb;                                           // [Nb] tokens seen so far (next position id)
   // hand-off of score passes to the scorer warp: two task slots and their full/empty barriers
   uint64_t* s_tbar = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(s_tot + Nb) + 15) & ~(uintptr_t)15);
-  StScoreTask* s_task = reinterpret_cast<StScoreTask*>(s_tbar + 4);
+  StScoreTask* s_task = reinterpret_cast<StScoreTask*>(s_tbar + 5);  // (s_tbar[4]: the recorded passes of this CTA's slabs are done)
   volatile int* s_abort = s_flags;
 
   const uint32_t bar_full = smem_u32(s_bar), bar_empty = smem_u32(s_bar + NS);
@@ -445,6 +446,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
       mbar_init(tbar_full + 8 * s, 1);
       mbar_init(tbar_empty + 8 * s, 1);
     }
+    mbar_init(smem_u32(s_tbar + 4), 1);
     for (int i = 0; i < 8; ++i) s_flags[i] = 0;  // (s_flags[8] belongs to the prefix warp below)
     for (int i = 16; i < 32; ++i) s_flags[i] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -520,6 +522,12 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
   // (no slab is then shared between CTAs), else an equal share of the chunk list.
   const long long per_cta = (p.slabs_per_cta > 0 && s_flags[8] > 0) ? (long long)p.slabs_per_cta * s_flags[8]
                                                                    : (total + gridDim.x - 1) / gridDim.x;
+  // (whole-slab pieces only; evaluated where it is used: the consumer loop has no register to spare)
+  // (bf16 rows only: the 8-bit instantiation is bound by its consumers and every extra live value costs it)
+  auto defer_on = [&]() {
+    if constexpr (KV8) return false;
+    else return p.defer != 0 && p.slabs_per_cta > 0 && s_flags[8] > 0;
+  };
   const long long g_begin = per_cta * blockIdx.x;
   long long g_end = g_begin + per_cta;
   if (g_end > total) g_end = total;
@@ -941,7 +949,19 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           consumer_sync();
           handed = s_flags[10] != 0;
         }
-        if (!handed) {
+        if (!handed && it + seg >= cnt && defer_on()) {
+          // the CTA's last slab: nothing is left to overlap the pass with; record it for the next launch
+          int* rec = p.pend + slab * kStPendWords;
+          if (tid < 8) {
+            reinterpret_cast<float*>(rec)[2 + tid] = s_finM[tid];
+            reinterpret_cast<float*>(rec)[10 + tid] = s_finf[tid];
+          } else if (tid == 8) {
+            rec[1] = n_old;
+            rec[0] = n;
+          }
+        } else if (!handed) {
+          // (the recorded pass of this slab, if any, must have been applied first)
+          if (defer_on()) mbar_wait(smem_u32(s_tbar + 4), 0u, s_abort, p.err);
           float* dout = p.delta_out ? p.delta_out + slab * (size_t)p.cap : nullptr;
           DYNTS_DISPATCH_GROUP(G, score_pass<GG>(p.accumulate != 0, score, p.comp + slab * (size_t)p.cap, dout, lg, p.cap, n,
                                                  n_old, s_finM, s_finf, tid, kStConsumers));
@@ -959,6 +979,30 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
     }
   } else if (cnt > 0) {
     // ================= scorer: score passes of finished slabs, beside the streaming =================
+    if (defer_on()) {
+      // first the passes the previous launch recorded for this CTA's slabs (their logits are in the
+      // other half of the scratch)
+      StCursor c2;
+      cursor_seek(c2, g_begin, s_off, s_cnt, Nb);
+      const int n_sl = cnt / s_flags[8];
+      for (int i = 0; i < n_sl; ++i) {
+        const size_t slab = ((size_t)(p.layer0 + c2.lrel) * Nb + c2.b) * Hkv + c2.h;
+        if (c2.lrel >= p.n_layers || c2.b >= Nb || c2.h >= Hkv) break;
+        int* rec = p.pend + slab * kStPendWords;
+        const int rn = rec[0];
+        if (rn > 0 && rn <= p.cap) {
+          const int rn_old = rec[1];
+          const float* rM = reinterpret_cast<const float*>(rec) + 2;
+          DYNTS_DISPATCH_GROUP(G, score_pass<GG>(true, p.score + slab * (size_t)p.cap, p.comp + slab * (size_t)p.cap, nullptr,
+                                                 p.logit_prev + slab * (size_t)G * p.cap, p.cap, rn, rn_old, rM, rM + 8, lane, 32));
+          __syncwarp();
+          if (lane == 0) rec[0] = 0;
+        }
+        if (i + 1 < n_sl) cursor_next_slab(c2, s_cnt, Nb, Hkv);
+      }
+      __threadfence_block();
+    }
+    if (lane == 0) mbar_arrive(smem_u32(s_tbar + 4));
     for (int t = 0;; ++t) {
       const int slot = t & 1;
       mbar_wait(tbar_full + 8 * slot, (uint32_t)(t >> 1) & 1u, s_abort, p.err);
@@ -987,6 +1031,27 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
     }
   }
   if (p.n_host == 0) finish_ticket(p);
+}
+
+// Applies the score passes recorded by the last streaming launch (see DecodeParams::defer): one
+// CTA per slab.  logit = the half of the scratch those launches wrote.
+__global__ void __launch_bounds__(128) flush_pending_kernel(float* score, float* comp, const float* logit, int* pend, int G,
+                                                            int cap) {
+  const size_t slab = blockIdx.x;
+  int* rec = pend + slab * kStPendWords;
+  const int n = rec[0];
+  if (n <= 0 || n > cap) return;  // uniform over the CTA
+  const int n_old = rec[1];
+  __shared__ float sM[8], sf[8];
+  if (threadIdx.x < 8) {
+    sM[threadIdx.x] = reinterpret_cast<const float*>(rec)[2 + threadIdx.x];
+    sf[threadIdx.x] = reinterpret_cast<const float*>(rec)[10 + threadIdx.x];
+  }
+  __syncthreads();
+  DYNTS_DISPATCH_GROUP(G, score_pass<GG>(true, score + slab * (size_t)cap, comp + slab * (size_t)cap, nullptr,
+                                         logit + slab * (size_t)G * cap, cap, n, n_old, sM, sf, (int)threadIdx.x, 128));
+  __syncthreads();
+  if (threadIdx.x == 0) rec[0] = 0;
 }
 
 }  // namespace dynts

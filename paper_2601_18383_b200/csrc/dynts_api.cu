@@ -43,7 +43,7 @@ dynts_status_t fail(dynts_status_t st, const char* fmt, ...) {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  size_t K, V, pos, score, comp, agg, src, hdr, len, tot, pinned, target, active, ticket, logit, part, arrive, total;
+  size_t K, V, pos, score, comp, agg, src, hdr, len, tot, pinned, target, active, ticket, logit, logit_half, part, arrive, pend, total;
 };
 
 // The streaming decode kernel covers bf16 and 8-bit slabs with head_dim 128.
@@ -99,11 +99,15 @@ Layout make_layout(const dynts_config_t* c, int cap) {
   L.target = take((size_t)c->batch * 4);
   L.active = take((size_t)c->batch * 4);
   L.ticket = take(256);
-  L.logit = L.part = L.arrive = off;
+  L.logit = L.part = L.arrive = L.pend = off;
+  L.logit_half = 0;
   if (stream_capable(c)) {
-    L.logit = take(slabs * (size_t)(c->q_heads / c->kv_heads) * cap * 4);
+    // two halves: a step writes one while the recorded score passes of the step before read the other
+    L.logit_half = align_up(slabs * (size_t)(c->q_heads / c->kv_heads) * cap * 4, 256);
+    L.logit = take(2 * L.logit_half);
     L.part = take((size_t)dynts::kStMaxCtas * 2 * dynts::kStPartStride * 4);
     L.arrive = take(slabs * 4);
+    L.pend = take(slabs * (size_t)dynts::kStPendWords * 4);
   }
   L.total = off;
   return L;
@@ -129,6 +133,8 @@ struct dynts_cache {
   int layer_cursor = 0;      // next layer expected by dynts_decode_attn_layer
   int cluster = 0, variant = 0;
   int score_source = 0;      // 0: attention mass accumulates (Eq. 6); 1: the caller supplies scores (Eq. 7)
+  int parity = 0;            // half of the logit scratch the next decode step writes
+  bool pending = false;      // the last streaming launches recorded score passes that are not applied yet
   long long launches = 0;
   // staging for the host-buffer entry point
   char* stage_dev = nullptr;
@@ -153,7 +159,8 @@ struct dynts_cache {
   int* target() const { return reinterpret_cast<int*>(base + lay.target); }
   int* active() const { return reinterpret_cast<int*>(base + lay.active); }
   unsigned int* ticket() const { return reinterpret_cast<unsigned int*>(base + lay.ticket); }
-  float* logit() const { return reinterpret_cast<float*>(base + lay.logit); }
+  float* logit(int half) const { return reinterpret_cast<float*>(base + lay.logit + (size_t)half * lay.logit_half); }
+  int* pend() const { return reinterpret_cast<int*>(base + lay.pend); }
   float* part() const { return reinterpret_cast<float*>(base + lay.part); }
   int* arrive() const { return reinterpret_cast<int*>(base + lay.arrive); }
   size_t slabs() const { return (size_t)cfg.layers * cfg.batch * cfg.kv_heads; }
@@ -269,6 +276,18 @@ int pick_cluster(const dynts_cache* c, int units, int n_max) {
   return s;
 }
 
+// Applies the score passes that streaming launches left recorded (DecodeParams::defer).  Called
+// before anything but the next deferring decode launch reads or writes the scores.
+dynts_status_t flush_pending(dynts_cache* c) {
+  if (!c->pending) return DYNTS_OK;
+  dynts::flush_pending_kernel<<<(unsigned)c->slabs(), 128, 0, c->stream>>>(c->score(), c->comp(), c->logit(c->parity ^ 1), c->pend(),
+                                                                       c->G, c->cap);
+  CUDA_TRY(cudaGetLastError());
+  c->launches += 1;
+  c->pending = false;
+  return DYNTS_OK;
+}
+
 dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const void* q, const void* k_new,
                              const void* v_new, void* out, float* scores, bool advance) {
   const dynts_config_t& f = c->cfg;
@@ -305,7 +324,10 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
   p.active = c->active();
   p.ticket = c->ticket();
   p.err = c->err_dev;
-  p.logit = c->logit();
+  p.logit = c->logit(c->parity);
+  p.logit_prev = c->logit(c->parity ^ 1);
+  p.pend = c->pend();
+  p.defer = 0;
   p.part = c->part();
   p.arrive = c->arrive();
   p.dbg = reinterpret_cast<int*>(c->ticket()) + 8;  // spare words of the ticket block
@@ -387,6 +409,16 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
         ctas = (int)used;
       }
     }
+    // The score pass of every CTA's last slab moves into the next launch when the pieces are whole
+    // slabs, the lengths travel with the launch (so the piece shape is certain), the scores
+    // accumulate and nobody asked for this step's mass.
+    // (Only launches that cover all layers: the records of a step then sit in one half of the scratch.)
+    const bool defer = !kv8 && n_layers == f.layers && p.slabs_per_cta > 0 && p.n_host > 0 && p.accumulate && scores == nullptr;
+    if (!defer) {
+      dynts_status_t fs = flush_pending(c);
+      if (fs != DYNTS_OK) return fs;
+    }
+    p.defer = defer ? 1 : 0;
     cudaLaunchConfig_t sc;
     memset(&sc, 0, sizeof(sc));
     cudaLaunchAttribute sattr[1];
@@ -401,13 +433,20 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
     cudaError_t e = cudaLaunchKernelEx(&sc, stream_kernel, p, c->map_KV);
     if (e != cudaSuccess) return fail(DYNTS_ERR_CUDA, "decode launch (streaming, %d CTAs): %s", ctas, cudaGetErrorString(e));
     c->launches += 1;
-    if (advance)
+    if (defer) c->pending = true;
+    if (advance) {
+      if (defer) c->parity ^= 1;  // the next step must not overwrite the logits of the recorded passes
       for (int b = 0; b < Nb; ++b)
         if (c->active_h[b]) {
           c->len_h[b] += 1;
           c->tot_h[b] += 1;
         }
+    }
     return DYNTS_OK;
+  }
+  {
+    dynts_status_t fs = flush_pending(c);  // the cluster kernels update the scores themselves
+    if (fs != DYNTS_OK) return fs;
   }
 
   cudaLaunchConfig_t lc;
@@ -484,6 +523,10 @@ dynts_status_t do_prefill(dynts_cache* c, int seq, const void* k, const void* v,
   if (n_pinned < 0 || n_pinned > T) return fail(DYNTS_ERR_INVALID_ARG, "n_pinned %d outside [0, %d]", n_pinned, T);
   if (seq >= c->cfg.batch) return fail(DYNTS_ERR_INVALID_ARG, "sequence %d out of range", seq);
   if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "prefill in the middle of a layer-by-layer step");
+  {
+    dynts_status_t fs_ = flush_pending(c);
+    if (fs_ != DYNTS_OK) return fs_;
+  }
   dynts::PrefillParams p;
   p.k = k;
   p.v = v;
@@ -525,6 +568,10 @@ dynts_status_t do_prefill(dynts_cache* c, int seq, const void* k, const void* v,
 }
 
 dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validated */, bool global = false) {
+  {
+    dynts_status_t fs_ = flush_pending(c);
+    if (fs_ != DYNTS_OK) return fs_;
+  }
   const int Nb = c->cfg.batch;
   bool any = false;
   for (int b = 0; b < Nb; ++b) {
@@ -687,6 +734,10 @@ void dynts_cache_destroy(dynts_cache_t* c) {
 
 dynts_status_t dynts_cache_set_stream(dynts_cache_t* c, void* stream) {
   if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (c->ready) {  // score passes still recorded are applied on the stream they belong to
+    dynts_status_t fs_ = flush_pending(c);
+    if (fs_ != DYNTS_OK) return fs_;
+  }
   c->stream = static_cast<cudaStream_t>(stream);
   return DYNTS_OK;
 }
@@ -826,6 +877,10 @@ dynts_status_t dynts_seq_reset(dynts_cache_t* c, int seq) {
   if (!c || seq < 0 || seq >= c->cfg.batch) return fail(DYNTS_ERR_INVALID_ARG, "bad cache or sequence");
   if (!c->ready) return fail(DYNTS_ERR_STATE, "cache holds nothing yet");
   if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "reset in the middle of a layer-by-layer step");
+  {
+    dynts_status_t fs_ = flush_pending(c);
+    if (fs_ != DYNTS_OK) return fs_;
+  }
   CUDA_TRY(cudaMemsetAsync(c->len() + seq, 0, sizeof(int), c->stream));
   CUDA_TRY(cudaMemsetAsync(c->tot() + seq, 0, sizeof(int), c->stream));
   CUDA_TRY(cudaMemsetAsync(c->pinned() + seq, 0, sizeof(int), c->stream));
@@ -850,13 +905,21 @@ int dynts_cache_capacity(const dynts_cache_t* c) {
   return config_ok(&c->cfg, &cap) ? cap : -1;
 }
 
-float* dynts_cache_scores(dynts_cache_t* c) { return (c && c->ready) ? c->score() : nullptr; }
+float* dynts_cache_scores(dynts_cache_t* c) {
+  if (!c || !c->ready) return nullptr;
+  if (flush_pending(c) != DYNTS_OK) return nullptr;  // score passes still recorded are applied on the stream first
+  return c->score();
+}
 
 dynts_status_t dynts_cache_export(dynts_cache_t* c, int layer, int seq, int head, void* K, void* V, int* pos,
                                   float* score, int* n) {
   if (!c || !c->ready) return fail(DYNTS_ERR_STATE, "cache holds nothing yet");
   if (layer < 0 || layer >= c->cfg.layers || seq < 0 || seq >= c->cfg.batch || head < 0 || head >= c->cfg.kv_heads)
     return fail(DYNTS_ERR_INVALID_ARG, "slab index out of range");
+  {
+    dynts_status_t fs_ = flush_pending(c);
+    if (fs_ != DYNTS_OK) return fs_;
+  }
   CUDA_TRY(cudaStreamSynchronize(c->stream));
   const size_t slab = ((size_t)layer * c->cfg.batch + seq) * c->cfg.kv_heads + head;
   const int rows = c->len_h[seq];
@@ -880,6 +943,10 @@ dynts_status_t dynts_cache_import(dynts_cache_t* c, int layer, int seq, int head
   if (n < 0 || n > c->cap) return fail(DYNTS_ERR_CAPACITY, "%d rows exceed capacity %d", n, c->cap);
   if (n_pinned < 0 || n_pinned > n) return fail(DYNTS_ERR_INVALID_ARG, "n_pinned out of range");
   if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "import in the middle of a layer-by-layer step");
+  {
+    dynts_status_t fs_ = flush_pending(c);
+    if (fs_ != DYNTS_OK) return fs_;
+  }
   CUDA_TRY(cudaStreamSynchronize(c->stream));
   const size_t slab = ((size_t)layer * c->cfg.batch + seq) * c->cfg.kv_heads + head;
   const size_t row_bytes = (size_t)c->cfg.head_dim * c->kv_elt;
@@ -919,6 +986,10 @@ dynts_status_t dynts_poll_error(dynts_cache_t* c) {
 
 dynts_status_t dynts_synchronize(dynts_cache_t* c) {
   if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  {
+    dynts_status_t fs_ = flush_pending(c);
+    if (fs_ != DYNTS_OK) return fs_;
+  }
   CUDA_TRY(cudaStreamSynchronize(c->stream));
   return DYNTS_OK;
 }
@@ -940,6 +1011,10 @@ dynts_status_t dynts_cache_set_score_source(dynts_cache_t* c, int source) {
   if (source != DYNTS_SCORE_ATTENTION && source != DYNTS_SCORE_EXTERNAL)
     return fail(DYNTS_ERR_INVALID_ARG, "score source must be DYNTS_SCORE_ATTENTION or DYNTS_SCORE_EXTERNAL");
   if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "a layer-by-layer step is in progress");
+  {
+    dynts_status_t fs_ = flush_pending(c);
+    if (fs_ != DYNTS_OK) return fs_;
+  }
   c->score_source = source;
   return DYNTS_OK;
 }
@@ -961,6 +1036,10 @@ dynts_status_t dynts_append_scores(dynts_cache_t* c, const float* s_new) {
   if (!c || !s_new) return fail(DYNTS_ERR_INVALID_ARG, "NULL argument");
   if (!c->ready) return fail(DYNTS_ERR_STATE, "cache holds nothing yet");
   if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "a layer-by-layer step is in progress");
+  {
+    dynts_status_t fs_ = flush_pending(c);
+    if (fs_ != DYNTS_OK) return fs_;
+  }
   const int n_slabs = (int)c->slabs();
   dynts::append_scores_kernel<<<(n_slabs + 255) / 256, 256, 0, c->stream>>>(c->score(), c->comp(), c->len(), c->active(), s_new,
                                                                           n_slabs, c->cfg.batch, c->cfg.kv_heads, c->cap);

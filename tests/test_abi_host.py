@@ -60,7 +60,7 @@ def test_cache_bytes_accounts_for_slabs(D):
     cfg = D.make_config(32, 1, 32, 8, 128, 2048, 128, 64)
     nbytes = D.dynts_cache_bytes(cfg)
     kv = 32 * 8 * 2112 * 128 * 2 * 2
-    assert kv < nbytes < kv * 1.1
+    assert kv < nbytes < kv * 1.12      # + positions, scores, compensation, gather list (16 B) and two halves of fp32 logits (32 B) per 512 B row
     assert D.dynts_cache_bytes(D.make_config(32, 1, 32, 8, 128, 2048, 4096, 64)) == 0   # window > budget
     assert D.dynts_cache_bytes(D.make_config(1, 1, 18, 2, 128, 64, 8, 8)) == 0          # G = 9 unsupported
     ragged = D.make_config(2, 3, 8, 2, 128, 1024, 128, 64, seq_budgets=[1024, 2048, 3072])
