@@ -951,6 +951,8 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         }
         if (!handed && it + seg >= cnt && defer_on()) {
           // the CTA's last slab: nothing is left to overlap the pass with; record it for the next launch
+          // (once the scorer warp is done with the record the previous launch left in the same place)
+          mbar_wait(smem_u32(s_tbar + 4), 0u, s_abort, p.err);
           int* rec = p.pend + slab * kStPendWords;
           if (tid < 8) {
             reinterpret_cast<float*>(rec)[2 + tid] = s_finM[tid];

@@ -250,3 +250,76 @@ def test_two_caches_on_two_streams_do_not_interfere():
     for a, b in zip(*results):
         assert torch.equal(a[0].view(torch.int16), b[0].view(torch.int16))
         assert torch.equal(H.bits(a[1]), H.bits(b[1])) and torch.equal(a[2], b[2]) and torch.equal(H.bits(a[3]), H.bits(b[3]))
+
+
+def test_config2_scores_when_the_last_pass_moves_into_the_next_launch():
+    """Decode steps that do not ask for the step's mass, on equally long slabs that fill the grid:
+    the launch then leaves the score pass of every CTA's last slab to the next launch.  The scores
+    read back (which applies what is still recorded) must equal the oracle's after every read, in
+    the middle of the run, after the run and across an eviction."""
+    cfg = W.get_config("c2_llama8b")
+    gpu = _steady_state(cfg, 2300, cfg.budget + 3)
+    slabs = _sample_slabs(cfg, 6, 3)
+    orc = H.oracle_from_gpu(gpu, cfg, slabs=slabs)
+    steps = 24
+    ring = gen.torch_step_ring(cfg, 2300, steps, "cuda:0")
+    out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda:0")
+    G = cfg.group
+    launches0 = gpu.launch_count()
+    for s in range(steps):
+        q, k, v = ring[0][s], ring[1][s], ring[2][s]
+        gpu.decode_attn(q, k, v, out)
+        qh, kh, vh = q.double().cpu().numpy(), k.double().cpu().numpy(), v.double().cpu().numpy()
+        for (l, b, h) in slabs:
+            sl = orc.slab(l, b, h)
+            sl.K[sl.n], sl.V[sl.n], sl.score[sl.n] = kh[l, b, h], vh[l, b, h], 0.0
+            sl.n += 1
+            alpha = O.attention_weights(qh[l, b, h * G:(h + 1) * G], sl.K[:sl.n])
+            sl.score[:sl.n] += alpha.sum(axis=0)
+            if s in (6, steps - 1):
+                o_ref = O.attention_output(alpha, sl.V[:sl.n])
+                assert H.rel_err_vectors(out.float().cpu().numpy()[l, b, h * G:(h + 1) * G], o_ref) <= H.TOL_OUT["bf16"]
+        if s in (6, steps - 1):
+            sc = gpu.scores_tensor().cpu().numpy()
+            for (l, b, h) in slabs:
+                sl = orc.slab(l, b, h)
+                fin = np.isfinite(sl.score[:sl.n])
+                assert np.abs(sc[l, b, h, :sl.n][fin] - sl.score[:sl.n][fin]).max() <= H.TOL_DELTA, (s, l, b, h)
+    # one launch per step plus the two that applied the recorded passes when the scores were read
+    assert gpu.launch_count() - launches0 == steps + 2
+    gpu.poll_error()
+    while gpu.len(0) < cfg.capacity:
+        gpu.decode_attn(ring[0][0], ring[1][0], ring[2][0], out)
+    H.check_evict_bit_exact(gpu, cfg, 0, slabs=slabs)
+    assert gpu.len(0) == cfg.budget
+    gpu.close()
+
+
+@pytest.mark.parametrize("every", [2, 3])
+def test_recorded_pass_on_short_slabs(every):
+    """The same hand-over on slabs so short that a CTA finishes its slab before its scorer warp has
+    applied the record of the previous launch: the new record must not be lost."""
+    cfg = W.get_config("c2_llama8b").scaled(budget=256, window=16, evict_interval=64, prompt=32)
+    gpu = _steady_state(cfg, 2400, cfg.budget + 3)
+    slabs = [(0, 0, 0), (5, 0, 3), (31, 0, 7)]
+    orc = H.oracle_from_gpu(gpu, cfg, slabs=slabs)
+    ring = gen.torch_step_ring(cfg, 2400, 12, "cuda:0")
+    out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda:0")
+    G = cfg.group
+    for s in range(12):
+        q, k, v = ring[0][s], ring[1][s], ring[2][s]
+        gpu.decode_attn(q, k, v, out)
+        qh, kh, vh = q.double().cpu().numpy(), k.double().cpu().numpy(), v.double().cpu().numpy()
+        for (l, b, h) in slabs:
+            sl = orc.slab(l, b, h)
+            sl.K[sl.n], sl.V[sl.n], sl.score[sl.n] = kh[l, b, h], vh[l, b, h], 0.0
+            sl.n += 1
+            sl.score[:sl.n] += O.attention_weights(qh[l, b, h * G:(h + 1) * G], sl.K[:sl.n]).sum(axis=0)
+        if (s + 1) % every == 0:
+            sc = gpu.scores_tensor().cpu().numpy()
+            for (l, b, h) in slabs:
+                sl = orc.slab(l, b, h)
+                fin = np.isfinite(sl.score[:sl.n])
+                assert np.abs(sc[l, b, h, :sl.n][fin] - sl.score[:sl.n][fin]).max() <= H.TOL_DELTA, (s, l, b, h)
+    gpu.poll_error()
+    gpu.close()
