@@ -250,7 +250,12 @@ int dynts_cache_capacity(const dynts_cache_t* c);
  * stream to drive the eviction with external scores (e.g. a predictor's).  NULL before storage
  * exists.  (The decode step adds each step's mass with compensated summation; the compensation
  * terms live beside the scores inside the cache, move with them at an eviction, and are at most
- * one ulp of the score, so overwriting the scores needs no further call.) */
+ * one ulp of the score, so overwriting the scores needs no further call.)
+ * A decode launch may leave the score update of some slabs to the next decode launch (the update
+ * has nothing to overlap with at the end of a launch).  Every call of this function first enqueues
+ * what is still outstanding on the cache's stream, as do eviction, export, import, prefill,
+ * dynts_append_scores and dynts_synchronize: read the accumulator through a pointer obtained
+ * after the decode calls whose effect you want to see, not through one kept from before. */
 float* dynts_cache_scores(dynts_cache_t* c);
 
 /* Copy one slab to host buffers (any may be NULL): K, V [n][d] in the cache dtype, pos [n] int32,

@@ -90,3 +90,26 @@ def test_noalloc_rejects_oversize_and_bad_arguments():
     with pytest.raises(D.DyntsError):
         D.dynts_evict_noalloc(None, K, pos, sc, 1, 128, D.DYNTS_BF16, 16, 16, 0, 0, 8, None)
     D.dynts_evict_noalloc(K, K, pos, sc, 1, 128, D.DYNTS_BF16, 16, 10, 0, 0, 12, None)   # n <= target: no-op
+
+
+def test_noalloc_moves_rows_of_8_bit_codes():
+    """Slabs of E4M3 codes (128-byte rows): the selection is the oracle's, the rows move bit for bit."""
+    import paper_2601_18383_b200 as D
+    from oracle import dynts_oracle as O
+    slabs, cap, d, rows, pinned, window, target = 5, 400, 128, 389, 24, 32, 200
+    g = torch.Generator(device="cuda").manual_seed(21)
+    K = torch.randint(0, 256, (slabs, cap, d), generator=g, device="cuda", dtype=torch.uint8)
+    V = torch.randint(0, 256, (slabs, cap, d), generator=g, device="cuda", dtype=torch.uint8)
+    pos = torch.arange(cap, dtype=torch.int32, device="cuda").repeat(slabs, 1).contiguous()
+    score = (torch.randint(0, 40, (slabs, cap), generator=g, device="cuda").float() / 3.0).contiguous()   # ties
+    score[:, :pinned] = float("inf")
+    K0, V0, s0 = K.cpu(), V.cpu(), score.cpu()
+    D.dynts_evict_noalloc(K, V, pos, score, slabs, d, D.DYNTS_BF16_KV8, cap, rows, pinned, window, target,
+                          torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    for i in range(slabs):
+        kept = torch.from_numpy(O.select_keep(s0[i, :rows].numpy(), rows, pinned, window, target))
+        assert len(kept) == target
+        assert torch.equal(pos[i, :target].cpu(), kept.to(torch.int32))
+        assert torch.equal(K[i, :target].cpu(), K0[i][kept]) and torch.equal(V[i, :target].cpu(), V0[i][kept])
+        assert torch.equal(H.bits(score[i, :target].cpu()), H.bits(s0[i][kept]))
