@@ -189,8 +189,15 @@ struct StCursor {
 
 __device__ __forceinline__ void cursor_seek(StCursor& c, long long g, const int* s_off, const int* s_cnt, int Nb) {
   const int per_layer = s_off[Nb];
-  c.lrel = (int)(g / per_layer);
-  int r = (int)(g % per_layer);
+  int r;
+  if (g <= 0x7fffffffLL) {  // (64-bit division costs a lone thread several hundred cycles)
+    const unsigned g32 = (unsigned)g, pl = (unsigned)per_layer;
+    c.lrel = (int)(g32 / pl);
+    r = (int)(g32 - (unsigned)c.lrel * pl);
+  } else {
+    c.lrel = (int)(g / per_layer);
+    r = (int)(g % per_layer);
+  }
   int lo = 0, hi = Nb;  // largest b with s_off[b] <= r and s_cnt[b] > 0
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
@@ -465,13 +472,36 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
       const int b = b0 + lane;
       int ln = -1, tt = 0;
       if (b < Nb) {
-        if (p.n_host > 0) {  // (constant indices: the parameter block is not copied to local memory)
+        if (p.n_host > 0) {
+          // Constant indices, so that the parameter block is not copied to local memory; the uniform
+          // bounds keep the launch from touching more of it than the batch needs (every first touch
+          // of a line of the block is a constant-cache miss of a few hundred cycles).
+          ln = p.len_host[0];
+          tt = p.tot_host[0];
+          if (Nb > 1) {
 #pragma unroll
-          for (int i = 0; i < kHostLens; ++i)
-            if (i == b) {
-              ln = p.len_host[i];
-              tt = p.tot_host[i];
-            }
+            for (int i = 1; i < 8; ++i)
+              if (i == b) {
+                ln = p.len_host[i];
+                tt = p.tot_host[i];
+              }
+          }
+          if (Nb > 8) {
+#pragma unroll
+            for (int i = 8; i < 32; ++i)
+              if (i == b) {
+                ln = p.len_host[i];
+                tt = p.tot_host[i];
+              }
+          }
+          if (Nb > 32) {
+#pragma unroll
+            for (int i = 32; i < kHostLens; ++i)
+              if (i == b) {
+                ln = p.len_host[i];
+                tt = p.tot_host[i];
+              }
+          }
         } else if (p.active[b]) {
           ln = p.len[b];
           tt = p.tot[b];
@@ -836,7 +866,15 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
       }
       // Who else works on this slab?  Chunk g0 is its first one.
       const long long g0 = g_begin + it - c.chunk;
-      const int p_first = (int)(g0 / per_cta), p_last = (int)((g0 + c.cb - 1) / per_cta);
+      int p_first, p_last;
+      if (total <= 0x7fffffffLL) {  // 32-bit division: this sits between a slab's last tile and its output
+        const unsigned pc = (unsigned)per_cta;
+        p_first = (int)((unsigned)g0 / pc);
+        p_last = (int)(((unsigned)g0 + (unsigned)c.cb - 1u) / pc);
+      } else {
+        p_first = (int)(g0 / per_cta);
+        p_last = (int)((g0 + c.cb - 1) / per_cta);
+      }
       const bool exclusive = p_first == p_last;
       if (p_first < 0 || p_last >= (int)gridDim.x || (int)blockIdx.x < p_first || (int)blockIdx.x > p_last) {
         if (tid == 0) {
@@ -975,7 +1013,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
     }
     if (tid == 0 && it >= cnt) {  // tell the scorer warp that nothing more will come
       const int slot = n_posted & 1;
-      mbar_wait(tbar_empty + 8 * slot, (((uint32_t)n_posted >> 1) & 1u) ^ 1u, s_abort, p.err);
+      if (n_posted >= 2) mbar_wait(tbar_empty + 8 * slot, (((uint32_t)n_posted >> 1) & 1u) ^ 1u, s_abort, p.err);  // (else never used)
       s_task[slot].slab = -1;
       mbar_arrive(tbar_full + 8 * slot);
     }
