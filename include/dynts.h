@@ -138,9 +138,12 @@ dynts_status_t dynts_decode_attn(dynts_cache_t* c, const void* q, const void* k_
 dynts_status_t dynts_decode_attn_layer(dynts_cache_t* c, int layer, const void* q, const void* k_new,
                                        const void* v_new, void* out, float* scores);
 
-/* dynts_decode_attn with HOST buffers: copies q, k_new, v_new to the device, runs the step,
- * copies out back and synchronises the stream.  Pinned host memory makes the copies asynchronous
- * up to that synchronisation.  (Staging buffers are allocated at the first call.) */
+/* dynts_decode_attn with HOST buffers: brings q, k_new, v_new to the device, runs the step,
+ * copies out back and synchronises the stream.  Inputs in pinned, mapped host memory
+ * (cudaHostAlloc, cudaHostRegister) that is 16-byte aligned are read by the kernel in place over
+ * the bus -- every input element is read once -- and, if out is such memory too, the output rows are
+ * written there by the kernel; any other host memory goes through device staging buffers and
+ * copies.  (Staging buffers are allocated at the first call.) */
 dynts_status_t dynts_decode_attn_host(dynts_cache_t* c, const void* q, const void* k_new, const void* v_new,
                                       void* out);
 

@@ -836,10 +836,35 @@ dynts_status_t dynts_decode_attn_host(dynts_cache_t* c, const void* q, const voi
   char* dout = dv + kb;
   const size_t qn = (size_t)f.layers * f.batch * f.q_heads * f.head_dim * c->elt;
   const size_t kn = (size_t)f.layers * f.batch * f.kv_heads * f.head_dim * c->elt;
-  CUDA_TRY(cudaMemcpyAsync(dq, q, qn, cudaMemcpyHostToDevice, c->stream));
-  CUDA_TRY(cudaMemcpyAsync(dk, k_new, kn, cudaMemcpyHostToDevice, c->stream));
-  CUDA_TRY(cudaMemcpyAsync(dv, v_new, kn, cudaMemcpyHostToDevice, c->stream));
-  st = launch_decode(c, 0, f.layers, dq, dk, dv, dout, nullptr, true);
+  // Pinned, mapped host buffers (cudaHostAlloc / cudaHostRegister; what PyTorch's pin_memory gives)
+  // are read by the kernel in place: each input element is read exactly once, so a staging copy
+  // would only add three transfers' latency.  Other host memory is staged.
+  auto device_view = [](const void* h) -> const void* {
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, h) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    if (a.type != cudaMemoryTypeHost || !a.devicePointer || !aligned16(a.devicePointer)) return nullptr;
+    return a.devicePointer;
+  };
+  const void* vq = device_view(q);
+  const void* vk = device_view(k_new);
+  const void* vv = device_view(v_new);
+  void* vo = const_cast<void*>(device_view(out));
+  if (vq && vk && vv && vo) {  // the output rows are written to the host buffer by the kernel as well
+    st = launch_decode(c, 0, f.layers, vq, vk, vv, vo, nullptr, true);
+    if (st != DYNTS_OK) return st;
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    return DYNTS_OK;
+  } else if (vq && vk && vv) {
+    st = launch_decode(c, 0, f.layers, vq, vk, vv, dout, nullptr, true);
+  } else {
+    CUDA_TRY(cudaMemcpyAsync(dq, q, qn, cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(cudaMemcpyAsync(dk, k_new, kn, cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(cudaMemcpyAsync(dv, v_new, kn, cudaMemcpyHostToDevice, c->stream));
+    st = launch_decode(c, 0, f.layers, dq, dk, dv, dout, nullptr, true);
+  }
   if (st != DYNTS_OK) return st;
   CUDA_TRY(cudaMemcpyAsync(out, dout, qn, cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(cudaStreamSynchronize(c->stream));
