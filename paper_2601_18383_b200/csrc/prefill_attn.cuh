@@ -21,7 +21,7 @@ namespace dynts {
 constexpr int kPfRows = 64;      // query rows per CTA and key rows per tile
 constexpr int kPfThreads = 128;
 constexpr int kPfTileBytes = kPfRows * 256;  // 64 rows x 128 bf16
-constexpr int kPfSmemBytes = 5 * kPfTileBytes;  // Q, K x 2, V x 2
+constexpr int kPfSmemBytes = 4 * kPfTileBytes;  // K x 2, V x 2; the Q tile borrows the second K buffer until its fragments are in registers
 
 struct PrefillAttnParams {
   const __nv_bfloat16* q;  // [L, Nb, Hq, T, 128]
@@ -66,7 +66,7 @@ __device__ __forceinline__ void pf_load_tile(uint32_t tile, const __nv_bfloat16*
 }
 
 // grid = (query tiles, Hq, L * Nb); tiles are taken from the last (longest) to the first.
-__global__ void __launch_bounds__(kPfThreads) prefill_attn_kernel(const PrefillAttnParams p) {
+__global__ void __launch_bounds__(kPfThreads, 3) prefill_attn_kernel(const PrefillAttnParams p) {
   extern __shared__ __align__(128) uint8_t pf_smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int gid = lane >> 2, tig = lane & 3;
@@ -78,8 +78,8 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attn_kernel(const PrefillA
   const __nv_bfloat16* K = p.k + ((size_t)lb * p.Hkv + h) * T * 128;
   const __nv_bfloat16* V = p.v + ((size_t)lb * p.Hkv + h) * T * 128;
   __nv_bfloat16* O = p.out + ((size_t)lb * p.Hq + hq) * T * 128;
-  const uint32_t sQ = (uint32_t)__cvta_generic_to_shared(pf_smem);
-  const uint32_t sK = sQ + kPfTileBytes, sV = sQ + 3 * kPfTileBytes;  // two buffers each
+  const uint32_t sK = (uint32_t)__cvta_generic_to_shared(pf_smem), sV = sK + 2 * kPfTileBytes;  // two buffers each
+  const uint32_t sQ = sK + kPfTileBytes;  // = K buffer 1, free until the first prefetch
   const int q0 = qt * kPfRows;
 
   pf_load_tile(sQ, Q, q0, T, tid);
@@ -99,6 +99,7 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attn_kernel(const PrefillA
       pf_ldmatrix_x4(sQ + r * 256 + ((c ^ (r & 7)) << 4), qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3]);
     }
   }
+  __syncthreads();  // every warp has its Q fragments: the buffer may be overwritten by the first prefetch
   float o[16][4];
 #pragma unroll
   for (int db = 0; db < 16; ++db)
