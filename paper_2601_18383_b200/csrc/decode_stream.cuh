@@ -765,17 +765,11 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
               e4m3x4_to_half2x2(kr[j][3], a1, a3);
               mma_f16_m16n8k16(s1, a0, a1, a2, a3, qa[2 * j + 1][0], qa[2 * j + 1][1]);
             }
-            // V: the transposed load gives (token 2tig, columns 2gid, 2gid+1 | token 2tig+1, the same columns)
+            // V: the transposed load gives (token 2tig, columns 2gid, 2gid+1 | token 2tig+1, the same
+            // columns); the codes stay packed (16 registers instead of 32) until the second product.
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              uint32_t v0, v1, v2, v3;  // tokens 0-7 x pieces 2j, 2j+1; tokens 8-15 x pieces 2j, 2j+1
-              ldmatrix_x4_trans(vbase + (((2 * j + lchk) ^ (lrow & 7)) << 4), v0, v1, v2, v3);
-              // -> (token, token+1) pairs of column 2gid (low half) and 2gid+1 (high half)
-              e4m3x4_to_half2x2(__byte_perm(v0, 0u, 0x3120), fr[2 * j][0], fr[2 * j][1]);
-              e4m3x4_to_half2x2(__byte_perm(v2, 0u, 0x3120), fr[2 * j][2], fr[2 * j][3]);
-              e4m3x4_to_half2x2(__byte_perm(v1, 0u, 0x3120), fr[2 * j + 1][0], fr[2 * j + 1][1]);
-              e4m3x4_to_half2x2(__byte_perm(v3, 0u, 0x3120), fr[2 * j + 1][2], fr[2 * j + 1][3]);
-            }
+            for (int j = 0; j < 4; ++j)  // fr[j][0..3]: tokens 0-7 x pieces 2j, 2j+1; tokens 8-15 x pieces 2j, 2j+1
+              ldmatrix_x4_trans(vbase + (((2 * j + lchk) ^ (lrow & 7)) << 4), fr[j][0], fr[j][1], fr[j][2], fr[j][3]);
           } else {
             // registers of one ldmatrix: tokens 0-7 x k 0-7, tokens 0-7 x k 8-15, tokens 8-15 x the same
 #pragma unroll
@@ -844,8 +838,15 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           }
 #pragma unroll
           for (int mb = 0; mb < 8; ++mb) {
-            if constexpr (KV8) mma_f16_m16n8k16(o[mb], fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3], pb0, pb1);
-            else mma_bf16_m16n8k16(o[mb], fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3], pb0, pb1);
+            if constexpr (KV8) {
+              // -> (token, token+1) pairs of column 2gid (low half) and 2gid+1 (high half)
+              uint32_t a0, a1, a2, a3;
+              e4m3x4_to_half2x2(__byte_perm(fr[mb >> 1][mb & 1], 0u, 0x3120), a0, a1);
+              e4m3x4_to_half2x2(__byte_perm(fr[mb >> 1][2 + (mb & 1)], 0u, 0x3120), a2, a3);
+              mma_f16_m16n8k16(o[mb], a0, a1, a2, a3, pb0, pb1);
+            } else {
+              mma_bf16_m16n8k16(o[mb], fr[mb][0], fr[mb][1], fr[mb][2], fr[mb][3], pb0, pb1);
+            }
           }
         }
         __syncwarp();
