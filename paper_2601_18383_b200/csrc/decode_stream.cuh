@@ -404,7 +404,10 @@ struct StScoreTask {
     default: { constexpr int GG = 8; CALL; } break; \
   }
 
-template <bool KV8>
+// DEFER: the instantiation that can record / apply deferred score passes (DecodeParams::defer).  The
+// 8-bit instantiation has no register to spare, so it carries that code only in the variant the
+// host launches for whole-slab pieces.
+template <bool KV8, bool DEFER = !KV8>
 __global__ void __launch_bounds__(kStThreads, 2)
 decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmKV) {
   constexpr int d = 128;
@@ -553,9 +556,8 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
   const long long per_cta = (p.slabs_per_cta > 0 && s_flags[8] > 0) ? (long long)p.slabs_per_cta * s_flags[8]
                                                                    : (total + gridDim.x - 1) / gridDim.x;
   // (whole-slab pieces only; evaluated where it is used: the consumer loop has no register to spare)
-  // (bf16 rows only: the 8-bit instantiation is bound by its consumers and every extra live value costs it)
   auto defer_on = [&]() {
-    if constexpr (KV8) return false;
+    if constexpr (!DEFER) return false;
     else return p.defer != 0 && p.slabs_per_cta > 0 && s_flags[8] > 0;
   };
   const long long g_begin = per_cta * blockIdx.x;

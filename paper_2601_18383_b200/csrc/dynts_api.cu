@@ -377,10 +377,14 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
 
   if (variant == 3) {
     const size_t smem = dynts::stream_smem_bytes(Nb);
-    auto* stream_kernel = kv8 ? dynts::decode_attn_stream_kernel<true> : dynts::decode_attn_stream_kernel<false>;
     if (!c->attr_stream) {
-      CUDA_TRY(cudaFuncSetAttribute(stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)dynts::stream_smem_bytes(dynts::kStMaxBatch)));
+      const int smem_max = (int)dynts::stream_smem_bytes(dynts::kStMaxBatch);
+      if (kv8) {
+        CUDA_TRY(cudaFuncSetAttribute(dynts::decode_attn_stream_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
+        CUDA_TRY(cudaFuncSetAttribute(dynts::decode_attn_stream_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
+      } else {
+        CUDA_TRY(cudaFuncSetAttribute(dynts::decode_attn_stream_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
+      }
       c->attr_stream = true;
     }
     int ctas = ((c->cluster == 1 || c->cluster == 2) ? c->cluster : 2) * c->sm_count;
@@ -413,12 +417,14 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
     // slabs, the lengths travel with the launch (so the piece shape is certain), the scores
     // accumulate and nobody asked for this step's mass.
     // (Only launches that cover all layers: the records of a step then sit in one half of the scratch.)
-    const bool defer = !kv8 && n_layers == f.layers && p.slabs_per_cta > 0 && p.n_host > 0 && p.accumulate && scores == nullptr;
+    const bool defer = n_layers == f.layers && p.slabs_per_cta > 0 && p.n_host > 0 && p.accumulate && scores == nullptr;
     if (!defer) {
       dynts_status_t fs = flush_pending(c);
       if (fs != DYNTS_OK) return fs;
     }
     p.defer = defer ? 1 : 0;
+    auto* stream_kernel = !kv8 ? dynts::decode_attn_stream_kernel<false, true>
+                               : (defer ? dynts::decode_attn_stream_kernel<true, true> : dynts::decode_attn_stream_kernel<true, false>);
     cudaLaunchConfig_t sc;
     memset(&sc, 0, sizeof(sc));
     cudaLaunchAttribute sattr[1];

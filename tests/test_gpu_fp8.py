@@ -198,3 +198,35 @@ def test_config3_full_size_8_bit():
     assert worst["out"] <= H.TOL_OUT["bf16"] and worst["delta"] <= H.TOL_DELTA, worst
     gpu.close()
     torch.cuda.empty_cache()
+
+
+def test_recorded_last_pass_with_8_bit_rows():
+    """Equally long slabs that fill the grid, no per-step mass requested: the launch leaves the score
+    pass of every CTA's last slab to the next launch.  Scores read back every third step must equal
+    the oracle's (which accumulates every step at once)."""
+    import paper_2601_18383_b200 as D
+    from workloads import gen
+    cfg = W.get_config("c2_llama8b").scaled(budget=256, window=16, evict_interval=64, prompt=32)
+    ks, vs = 0.03125, 0.0625
+    gpu, orc = _make(cfg, ks, vs)
+    k, v = gen.torch_keys_values(cfg, 2500, cfg.budget + 3, "cuda:0")
+    gpu.prefill(k, v, n_pinned=cfg.prompt)
+    O.prefill(orc, k.float().cpu().numpy(), v.float().cpu().numpy(), n_pinned=cfg.prompt)
+    ring = gen.torch_step_ring(cfg, 2500, 9, "cuda:0")
+    out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda:0")
+    launches0 = gpu.launch_count()
+    for s in range(9):
+        q, kk, vv = ring[0][s], ring[1][s], ring[2][s]
+        gpu.decode_attn(q, kk, vv, out)
+        o_ref, _ = O.decode_step(orc, q.double().cpu().numpy(), kk.float().cpu().numpy(), vv.float().cpu().numpy())
+        if (s + 1) % 3 == 0:
+            assert H.rel_err_vectors(out.float().cpu().numpy(), o_ref) <= H.TOL_OUT["bf16"]
+            sc = gpu.scores_tensor().cpu().numpy()
+            worst = 0.0
+            for l, b, h, sl in orc.units():
+                fin = np.isfinite(sl.score[:sl.n])
+                worst = max(worst, float(np.abs(sc[l, b, h, :sl.n][fin] - sl.score[:sl.n][fin]).max()))
+            assert worst <= H.TOL_DELTA, (s, worst)
+    assert gpu.launch_count() - launches0 == 9 + 3      # three reads applied what was still recorded
+    gpu.poll_error()
+    gpu.close()
