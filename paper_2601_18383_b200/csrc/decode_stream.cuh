@@ -1082,6 +1082,7 @@ __global__ void __launch_bounds__(128) flush_pending_kernel(float* score, float*
                                                             int cap) {
   const size_t slab = blockIdx.x;
   int* rec = pend + slab * kStPendWords;
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // (launched with programmatic stream serialisation)
   const int n = rec[0];
   if (n <= 0 || n > cap) return;  // uniform over the CTA
   const int n_old = rec[1];

@@ -280,9 +280,18 @@ int pick_cluster(const dynts_cache* c, int units, int n_max) {
 // before anything but the next deferring decode launch reads or writes the scores.
 dynts_status_t flush_pending(dynts_cache* c) {
   if (!c->pending) return DYNTS_OK;
-  dynts::flush_pending_kernel<<<(unsigned)c->slabs(), 128, 0, c->stream>>>(c->score(), c->comp(), c->logit(c->parity ^ 1), c->pend(),
-                                                                       c->G, c->cap);
-  CUDA_TRY(cudaGetLastError());
+  cudaLaunchConfig_t fc;
+  memset(&fc, 0, sizeof(fc));
+  cudaLaunchAttribute fattr[1];
+  fattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see griddepcontrol.wait in the kernel
+  fattr[0].val.programmaticStreamSerializationAllowed = 1;
+  fc.attrs = fattr;
+  fc.numAttrs = 1;
+  fc.stream = c->stream;
+  fc.gridDim = dim3((unsigned)c->slabs(), 1, 1);
+  fc.blockDim = dim3(128, 1, 1);
+  CUDA_TRY(cudaLaunchKernelEx(&fc, dynts::flush_pending_kernel, c->score(), c->comp(), (const float*)c->logit(c->parity ^ 1),
+                              c->pend(), c->G, c->cap));
   c->launches += 1;
   c->pending = false;
   return DYNTS_OK;
