@@ -75,6 +75,11 @@ struct EvictParams {
   const int* target;  // [Nb]
   int* err;
   int L, Nb, Hkv, d, cap, window, elt_bytes;
+  // Fused kernel: score passes the last streaming decode launch left recorded (DecodeParams::defer)
+  // are applied by each slab's CTA before it reads the scores.  pend == NULL: nothing recorded.
+  int* pend = nullptr;
+  const float* logit_prev = nullptr;
+  int G = 0;
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {

@@ -385,6 +385,26 @@ __device__ __forceinline__ void combine_partials(const float* part, int p_first,
   }
 }
 
+// The same pass with one group of loads in flight per thread: for callers that must stay small in
+// registers (the eviction kernel applies recorded passes with it).
+template <int GG>
+__device__ __forceinline__ void score_pass_lean(float* score, float* comp, const float* lg, int cap, int n, int n_old,
+                                                const float* s_finM, const float* s_finf, int tid, int nthr) {
+  if ((cap & 3) == 0 && cap >= 4) {
+    score_pass_vec<GG, 1>(true, score, comp, nullptr, lg, cap, n, n_old, s_finM, s_finf, tid, nthr);
+  } else {
+    for (int j = tid; j < n; j += nthr) {
+      float dl = 0.f;
+#pragma unroll
+      for (int g = 0; g < GG; ++g) dl += fast_exp2(__ldcg(lg + (size_t)g * cap + j) - s_finM[g]) * s_finf[g];
+      float sj = j == n_old ? 0.f : score[j], cj = j == n_old ? 0.f : comp[j];
+      kahan_add(sj, cj, dl);
+      score[j] = sj;
+      comp[j] = cj;
+    }
+  }
+}
+
 // A score pass handed from the consumer warps to the scorer warp.
 struct StScoreTask {
   long long slab;  // < 0: no more tasks

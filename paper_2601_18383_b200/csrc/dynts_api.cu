@@ -583,7 +583,10 @@ dynts_status_t do_prefill(dynts_cache* c, int seq, const void* k, const void* v,
 }
 
 dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validated */, bool global = false) {
-  {
+  // Recorded score passes: the fused kernel applies them slab by slab before it reads the scores;
+  // the other paths (aggregated keys, very long slabs) need them applied beforehand.
+  const bool fused_path = c->cap <= 12800;
+  if (global || !fused_path) {
     dynts_status_t fs_ = flush_pending(c);
     if (fs_ != DYNTS_OK) return fs_;
   }
@@ -633,8 +636,14 @@ dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validat
     c->launches += 1;
     p.key = c->agg();
   }
-  if (c->cap <= 12800) {
+  if (fused_path) {
     // one launch: selection and compaction of a slab by the same CTA
+    if (c->pending) {
+      p.pend = c->pend();
+      p.logit_prev = c->logit(c->parity ^ 1);
+      p.G = c->G;
+      c->pending = false;
+    }
     const size_t smem = (size_t)c->cap * (global ? 20 : 16);
     dynts_status_t st = ensure_smem_attr(dynts::evict_fused_kernel, smem, &c->attr_fused, false);
     if (st != DYNTS_OK) return st;

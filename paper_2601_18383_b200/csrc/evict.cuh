@@ -18,6 +18,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "decode_stream.cuh"  // score_pass_lean, kStPendWords: recorded score passes are applied here
 
 namespace dynts {
 
@@ -253,6 +254,25 @@ __global__ void __launch_bounds__(kFusedThreads) evict_fused_kernel(const EvictP
   const int tid = threadIdx.x;
   // Launched with programmatic stream serialisation: wait here for the kernel before this one.
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (p.pend != nullptr) {
+    // a score pass of this slab that the last decode launch recorded instead of running it
+    int* rec = p.pend + (size_t)slab * kStPendWords;
+    const int rn = rec[0];
+    if (rn > 0 && rn <= p.cap) {  // uniform over the CTA
+      __shared__ float s_recM[8], s_recf[8];
+      if (tid < 8) {
+        s_recM[tid] = reinterpret_cast<const float*>(rec)[2 + tid];
+        s_recf[tid] = reinterpret_cast<const float*>(rec)[10 + tid];
+      }
+      const int rn_old = rec[1];
+      __syncthreads();
+      DYNTS_DISPATCH_GROUP(p.G, score_pass_lean<GG>(p.score + (size_t)slab * p.cap, p.comp + (size_t)slab * p.cap,
+                                                    p.logit_prev + (size_t)slab * p.G * p.cap, p.cap, rn, rn_old, s_recM,
+                                                    s_recf, tid, kFusedThreads));
+      __syncthreads();  // the updated scores are read back below
+      if (tid == 0) rec[0] = 0;
+    }
+  }
   const int n = p.len[b];
   const int tgt = p.target[b];
   int* hdr = p.hdr + (size_t)slab * 4;
