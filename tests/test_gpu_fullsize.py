@@ -323,3 +323,43 @@ def test_recorded_pass_on_short_slabs(every):
                 assert np.abs(sc[l, b, h, :sl.n][fin] - sl.score[:sl.n][fin]).max() <= H.TOL_DELTA, (s, l, b, h)
     gpu.poll_error()
     gpu.close()
+
+
+@pytest.mark.parametrize("kv8", [False, True])
+def test_eviction_right_after_recorded_passes_equals_the_eager_path(kv8):
+    """Two caches on the same inputs: one is asked for every step's mass (so every score pass runs
+    inside its launch), the other is not (whole-slab pieces: the last pass of every CTA is recorded
+    and, at the eviction, applied by the eviction kernel itself).  After the eviction both must hold
+    the same bits: scores, positions, K, V."""
+    import paper_2601_18383_b200 as D
+    cfg = W.get_config("c2_llama8b").scaled(budget=256, window=16, evict_interval=32, prompt=32)
+    caches = []
+    for _ in range(2):
+        g = D.Cache(cfg.layers, cfg.batch, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.budget, cfg.window, cfg.evict_interval,
+                    dtype="bf16_kv8" if kv8 else "bf16")
+        if kv8:
+            g.set_kv_scale(0.03125, 0.0625)
+        k, v = gen.torch_keys_values(cfg, 2600, cfg.budget, "cuda:0")
+        g.prefill(k, v, n_pinned=cfg.prompt)
+        caches.append(g)
+    eager, lazy = caches
+    ring = gen.torch_step_ring(cfg, 2600, cfg.evict_interval, "cuda:0")
+    oe = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda:0")
+    ol = torch.empty_like(oe)
+    delta = torch.zeros((cfg.layers, cfg.batch, cfg.kv_heads, eager.capacity), dtype=torch.float32, device="cuda:0")
+    for cycle in range(2):
+        for s in range(cfg.evict_interval):
+            eager.decode_attn(ring[0][s], ring[1][s], ring[2][s], oe, delta)
+            lazy.decode_attn(ring[0][s], ring[1][s], ring[2][s], ol)
+        n0 = lazy.launch_count()
+        eager.evict(0)
+        lazy.evict(0)
+        assert lazy.launch_count() - n0 == 1            # no separate launch for the recorded passes
+        assert torch.equal(oe.view(torch.int16), ol.view(torch.int16))
+        for sl in [(0, 0, 0), (7, 0, 3), (31, 0, 7), (16, 0, 5)]:
+            Ke, Ve, pe, se = eager.export_slab(*sl)
+            Kl, Vl, pl, sl_ = lazy.export_slab(*sl)
+            assert torch.equal(pe, pl) and torch.equal(H.bits(se), H.bits(sl_)), (cycle, sl)
+            assert torch.equal(H.bits(Ke), H.bits(Kl)) and torch.equal(H.bits(Ve), H.bits(Vl))
+    eager.poll_error(); lazy.poll_error()
+    eager.close(); lazy.close()
