@@ -105,8 +105,12 @@ class PresetRun:
 
     def __init__(self, preset: Preset, layers, batch, q_heads, kv_heads, head_dim, dtype="bf16", device="cuda:0"):
         self.preset = preset
+        # One spare row is enough for the trigger-at-B schedule; the row count of a slab is rounded up
+        # to a multiple of 32 so that the kernels' vector paths apply (16-byte score accesses, whole
+        # 128-byte lines of the logit scratch).
+        capacity = (preset.budget + 1 + 31) // 32 * 32
         self.cache = _b.Cache(layers, batch, q_heads, kv_heads, head_dim, preset.budget, preset.window, 1,
-                              dtype=dtype, device=device)
+                              dtype=dtype, capacity=capacity, device=device)
         self.cache.set_score_source(preset.score_source)
         self.events = 0
 
