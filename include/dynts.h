@@ -56,7 +56,9 @@ typedef struct dynts_config {
   int budget;         /* B: default eviction target (rows kept per slab) */
   int window;         /* W_l: most recent rows, always kept */
   int evict_interval; /* E: decode steps between evictions; slab capacity = max budget + E */
-  int capacity;       /* rows per slab; 0 => max budget + evict_interval */
+  int capacity;       /* rows per slab; 0 => max budget + evict_interval.  A multiple of 32 lets the
+                         kernels use 16-byte score accesses and whole lines of their scratch: an odd
+                         row count costs the score update about 4x its loads */
   int dtype;          /* dynts_dtype_t of q, k, v, out and of the slab rows */
   const int* seq_budgets; /* host [batch] per-sequence targets, or NULL => budget for all */
   void* storage;          /* device memory for the whole cache, 256-byte aligned, or NULL:
