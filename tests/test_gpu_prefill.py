@@ -73,3 +73,31 @@ def test_prefill_attention_rejects_other_shapes():
         gpu.prefill_attn(x, kv, kv, x)
     assert e.value.status == D.DYNTS_ERR_INVALID_ARG and gpu.len(0) == 0
     gpu.close()
+
+
+def test_prefill_attention_into_a_cache_of_8_bit_rows():
+    """The prompt attention reads the caller's bf16 k, v (so its output equals the bf16 cache's bit
+    for bit); the fill stores the oracle's E4M3 codes."""
+    import paper_2601_18383_b200 as D
+    T = 150
+    cfg = W.get_config("c2_llama8b").scaled(layers=2, batch=1, kv_heads=2, q_heads=8, prompt=T, budget=256, window=8,
+                                             evict_interval=16)
+    q, k, v = _qkv(cfg, T, 91)
+    ks, vs = 0.02, 0.07
+    a = H.make_gpu(cfg)
+    b = D.Cache(cfg.layers, cfg.batch, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.budget, cfg.window, cfg.evict_interval,
+                dtype="bf16_kv8")
+    b.set_kv_scale(ks, vs)
+    oa = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, T, 128), dtype=torch.bfloat16, device="cuda:0")
+    ob = torch.empty_like(oa)
+    a.prefill_attn(H.dev(q, cfg), H.dev(k, cfg), H.dev(v, cfg), oa)
+    b.prefill_attn(H.dev(q, cfg), H.dev(k, cfg), H.dev(v, cfg), ob)
+    torch.cuda.synchronize()
+    assert torch.equal(oa.view(torch.int16), ob.view(torch.int16))
+    assert H.rel_err_vectors(ob.float().cpu().numpy().astype(np.float64), O.prefill_attention(q, k, v)) <= H.TOL_OUT["bf16"]
+    for (l, h) in [(0, 0), (1, 1)]:
+        Kc, Vc, pos, score = b.export_slab(l, 0, h)
+        assert np.array_equal(Kc.numpy(), O.fp8_e4m3_encode(k[l, 0, h] / np.float32(ks)))
+        assert np.array_equal(Vc.numpy(), O.fp8_e4m3_encode(v[l, 0, h] / np.float32(vs)))
+        assert np.array_equal(pos.numpy(), np.arange(T)) and np.isinf(score.numpy()).all()
+    a.close(); b.close()
