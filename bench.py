@@ -161,17 +161,22 @@ def run_ours(args, cfg, rank, world, device):
         if external:
             cache.append_scores(s_ring[j])
 
+    cycle = {"since": 0}      # decode steps since the last eviction, kept across the phases below
+
     def step(i):
         decode(i % ring_n)
-        if (i + 1) % E == 0:
+        cycle["since"] += 1
+        if cycle["since"] == E:
             evict_call(0)
+            cycle["since"] = 0
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize(device)
 
-    # warm-up: at least one full eviction cycle so that scores and selection are non-trivial
+    # warm-up: the requested steps rounded up to whole eviction cycles (at least one), so that scores and
+    # selection are non-trivial and the timed region starts at the beginning of a cycle
     warm = max(args.warmup, 3)
     warm = (warm + E - 1) // E * E
     for i in range(warm):
@@ -215,7 +220,7 @@ def run_ours(args, cfg, rank, world, device):
     dec_events, ev_events, dec_bytes = [], [], []
     i = 0
     while i < Kp:
-        run = min(E - (i % E), Kp - i)
+        run = min(E - cycle["since"], Kp - i)   # (the timed region may have stopped in the middle of a cycle)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
         for j in range(i, i + run):
@@ -224,7 +229,9 @@ def run_ours(args, cfg, rank, world, device):
         b.record(stream)
         dec_events.append((a, b, run))
         i += run
-        if i % E == 0:
+        cycle["since"] += run
+        if cycle["since"] == E:
+            cycle["since"] = 0
             a2, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a2.record(stream)
             evict_call(0)
@@ -304,12 +311,12 @@ def run_ours(args, cfg, rank, world, device):
         cpu = oracle_baseline(cfg, cache, q_ring, k_ring, v_ring, budget_s=args.cpu_seconds)
 
     result = {
-        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": warm,
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
         "ms_per_step": round(ms / K, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": cfg.name, "layers": cfg.layers, "batch": cfg.batch, "q_heads": cfg.q_heads,
                    "kv_heads": cfg.kv_heads, "head_dim": cfg.head_dim, "budget": cfg.budget, "window": cfg.window,
-                   "evict_interval": E, "prompt_pinned": cfg.prompt, "dist": cfg.dist, "score_source": args.score_source, "selection": args.selection, "kv_dtype": "e4m3 codes, scale 1/32" if kv8 else cfg.dtype, "accumulate": "fp32 (softmax, output, scores)",
+                   "evict_interval": E, "warmup_steps_run": warm, "prompt_pinned": cfg.prompt, "dist": cfg.dist, "score_source": args.score_source, "selection": args.selection, "kv_dtype": "e4m3 codes, scale 1/32" if kv8 else cfg.dtype, "accumulate": "fp32 (softmax, output, scores)",
                    "cache_bytes": cache.nbytes, "l2_policy": "inputs larger than L2 (KV cache %.0f MB vs 126 MB L2)" % (cache.nbytes / 1e6),
                    "replicas": world},
         "hbm_gbs_decode": round(dec_gbs, 1), "roofline": roofline, "evict": evict, "e2e": e2e,

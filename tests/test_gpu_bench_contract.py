@@ -11,8 +11,8 @@ pytestmark = pytest.mark.gpu
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-def _run(*extra):
-    cmd = [sys.executable, "bench.py", "--steps", "128", "--warmup", "64", "--cpu-seconds", "1"] + list(extra)
+def _run(*extra, steps=128, warmup=64):
+    cmd = [sys.executable, "bench.py", "--steps", str(steps), "--warmup", str(warmup), "--cpu-seconds", "1"] + list(extra)
     res = subprocess.run(cmd, cwd=ROOT, capture_output=True, text=True, timeout=600)
     assert res.returncode == 0, res.stderr[-3000:]
     lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
@@ -24,7 +24,7 @@ def _run(*extra):
 def test_bench_line_contract(extra):
     d = _run(*extra)
     assert d["metric"] == "decode tokens/s at budget B" and d["unit"] == "tokens/s" and d["higher_is_better"] is True
-    assert d["n_gpus"] == 1 and d["steps"] == 128 and d["warmup"] >= 64 and d["scaling"] == "weak"
+    assert d["n_gpus"] == 1 and d["steps"] == 128 and d["warmup"] == 64 and d["config"]["warmup_steps_run"] >= 64 and d["scaling"] == "weak"
     assert d["vs_baseline"] is None and d["data"] == "synthetic" and d["dtype"] in ("bf16", "f32")
     assert d["value"] > 0 and abs(d["value"] - d["config"]["batch"] / (d["ms_per_step"] * 1e-3)) <= 0.01 * d["value"]
     assert "workload" in d["config"] and "model" not in d["config"]
@@ -40,3 +40,13 @@ def test_bench_line_contract(extra):
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
     if d["evict"] is not None:
         assert d["evict"]["bound"] == "hbm" and d["evict"]["achieved"] >= 0
+
+
+@pytest.mark.parametrize("steps,warmup", [(100, 5), (2, 1), (70, 3)])
+def test_step_counts_off_the_eviction_cycle(steps, warmup):
+    """K and W need not be multiples of the eviction interval: the eviction cycle carries over from
+    the timed region into the per-kernel pass and the end-to-end arm."""
+    d = _run("--no-cpu-baseline", steps=steps, warmup=warmup)
+    assert d["steps"] == steps and d["warmup"] == warmup and d["config"]["warmup_steps_run"] >= max(3, warmup)
+    assert d["value"] > 0 and d["roofline"]["achieved"] > 0 and d["e2e"]["value"] > 0
+    assert d["gpu_launches"] >= steps
