@@ -8,7 +8,7 @@
 // stops in the middle of another; when all slabs are equally long and there are at least about as
 // many as CTAs, a piece is a whole number of slabs instead and no slab is shared).  Inside a CTA
 // one producer thread walks the piece and issues
-// TMA tile loads (cp.async.bulk.tensor, 128-byte swizzle, no multicast) of the K and V rows of
+// TMA tile loads (cp.async.bulk.tensor, 128-byte swizzle, each tile to one CTA only) of the K and V rows of
 // each chunk into a 6-stage shared-memory ring guarded by mbarriers, running ahead of the four
 // consumer warps across chunk and slab boundaries, so the HBM stream never pauses for an
 // epilogue.  Chunk i of a CTA goes to stage i mod 6 and to the warp pair i mod 2; with an even
