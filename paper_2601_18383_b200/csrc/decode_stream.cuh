@@ -7,17 +7,23 @@
 // ("stream-K": a CTA usually starts in the middle of one slab, covers some slabs completely and
 // stops in the middle of another; when all slabs are equally long and there are at least about as
 // many as CTAs, a piece is a whole number of slabs instead and no slab is shared).  Inside a CTA
-// one producer thread walks the piece and issues
-// TMA tile loads (cp.async.bulk.tensor, 128-byte swizzle, each tile to one CTA only) of the K and V rows of
-// each chunk into a 6-stage shared-memory ring guarded by mbarriers, running ahead of the four
-// consumer warps across chunk and slab boundaries, so the HBM stream never pauses for an
-// epilogue.  Chunk i of a CTA goes to stage i mod 6 and to the warp pair i mod 2; with an even
-// stage count every stage is always consumed by the same two warps, which is what makes the
-// parity wait on its barrier unambiguous (a waiter is never two phases away from the barrier).
-// The consumer warps take 16 rows each: K Q^T (the unit's 16 tokens on M, the heads on N) and
-// V^T P (head_dim on M, the heads on N) run on the tensor pipe (mma.sync m16n8k16, fp32
-// accumulate: 16 mma per unit, which is what bounds the consumers) with operands fetched by
-// ldmatrix from the swizzled tiles; online softmax in registers, P transposed by movmatrix.
+// one producer thread walks the piece and issues TMA tile loads (cp.async.bulk.tensor.3d over one
+// tensor map [K|V][rows][128], 128-byte swizzle, each tile to one CTA only): one load brings the K
+// box and the V box of a chunk (two loads for bf16 rows, one per half of head_dim) into a
+// shared-memory ring (6 stages of 16 KB; 12 of 8 KB for 8-bit rows) with a "full" mbarrier per
+// stage and an "empty" mbarrier per group of stages, running ahead of the four consumer warps
+// across chunk and slab boundaries, so the HBM stream never pauses for an epilogue.  The producer
+// thread's own latency bounds a CTA (a barrier wait costs it about 300 cycles even on a completed
+// phase, arming a stage and issuing a load about 100), hence the grouped waits, the combined
+// loads and a per-chunk loop that carries only counters.  Chunk i of a CTA goes to stage
+// i mod NS and to the warp pair i mod 2; with an even stage count every stage is always consumed
+// by the same two warps, which is what makes the parity wait on its barrier unambiguous (a
+// waiter is never two phases away from the barrier).  The consumer warps take 16 rows each:
+// K Q^T (the unit's 16 tokens on M, the heads on N) and V^T P (head_dim on M, the heads on N) run
+// on the tensor pipe (mma.sync m16n8k16, fp32 accumulate, 16 mma per unit) with operands
+// fetched by ldmatrix from the swizzled tiles; online softmax in registers, P transposed by
+// movmatrix.  The rows per slab of every sequence normally come with the launch (DecodeParams::
+// n_host), so the kernel reads no length from global memory and needs no ticket at its end.
 //
 // The final softmax normaliser of a slab is known only when all its chunks are done, and the
 // importance score needs the normalised weights (Eq. 6).  So every row's scaled logits go to a
@@ -28,7 +34,9 @@
 // every score row.  Nobody ever waits for another CTA: there is no inter-CTA spin, no float
 // atomic, one writer per score row and per output element.  While a CTA still has chunks to
 // stream, that pass is handed to a sixth warp (the scorer) through a two-slot task queue in shared
-// memory, so the consumer warps go straight on to the next slab.
+// memory, so the consumer warps go straight on to the next slab.  The pass after a CTA's last chunk
+// has nothing left to overlap with: with whole-slab pieces it is recorded instead (DecodeParams::
+// defer) and applied by the scorer warp of the next launch, or by the eviction kernel.
 //
 // 8-bit slabs (KV8 = true): a stage holds one 32 x 128-byte box of K codes and one of V codes.
 // ldmatrix moves bytes, so the same 8 x 16-byte matrices are fetched; a thread's 32-bit register
