@@ -212,3 +212,33 @@ def test_capacity_error_and_inactive_sequences():
     assert out[0, 1].abs().max().item() == 0.0 and out[0, 0].abs().max().item() > 0.0
     gpu.poll_error()
     gpu.close()
+
+
+def test_batch_larger_than_the_launch_carries_lengths_for():
+    """More than 64 sequences: the streaming kernel then reads the lengths from device memory and
+    the last block advances them through the ticket, as under stream capture."""
+    cfg = W.get_config("c2_llama8b").scaled(layers=1, batch=70, kv_heads=1, q_heads=4, prompt=20, budget=96, window=8,
+                                             evict_interval=16)
+    gpu = H.make_gpu(cfg)
+    orc = H.make_oracle(cfg)
+    pk, pv = W.prompt_kv(cfg, 17)
+    gpu.prefill(H.dev(pk, cfg), H.dev(pv, cfg))
+    O.prefill(orc, pk.astype(np.float64), pv.astype(np.float64))
+    stream = W.DecodeStream(cfg, 17)
+    out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda:0")
+    delta = torch.zeros((cfg.layers, cfg.batch, cfg.kv_heads, gpu.capacity), dtype=torch.float32, device="cuda:0")
+    for s in range(1, 40):
+        q, k, v = stream.step(s)
+        gpu.decode_attn(H.dev(q, cfg), H.dev(k, cfg), H.dev(v, cfg), out, delta if s % 2 else None)
+        o_ref, d_ref = O.decode_step(orc, q.astype(np.float64), k.astype(np.float64), v.astype(np.float64))
+        assert gpu.len(69) == orc.length(69) == 20 + s
+        if s % 5 == 0:
+            assert H.rel_err_vectors(out.float().cpu().numpy(), o_ref) <= H.TOL_OUT["bf16"]
+    sc = gpu.scores_tensor().cpu().numpy()
+    for l, b, h, sl in orc.units():
+        fin = np.isfinite(sl.score[:sl.n])
+        assert np.abs(sc[l, b, h, :sl.n][fin] - sl.score[:sl.n][fin]).max() <= H.TOL_DELTA
+        pos = gpu.export_slab(l, b, h)[2].numpy()
+        assert np.array_equal(pos, sl.pos[:sl.n])
+    gpu.poll_error()
+    gpu.close()
