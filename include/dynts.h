@@ -159,12 +159,18 @@ dynts_status_t dynts_decode_attn_host(dynts_cache_t* c, const void* q, const voi
 dynts_status_t dynts_evict(dynts_cache_t* c, int budget);
 
 /* Eviction with one selection per sequence (Appendix B.1 aggregates a token's importance across
- * all layers and heads): the scores of all slabs of a sequence are summed row by row (float32,
- * layer-major then KV head) and every slab ranks its selection window by that sum, so all
- * layers and heads keep the same tokens.  Requires that all slabs of a sequence hold the same
- * tokens, i.e. that every eviction of this cache is of this kind (or driven by shared external
- * scores).  Otherwise as dynts_evict.  Up to 10000 rows per slab. */
+ * all layers and heads): the scores of all slabs of a sequence are summed row by row (see
+ * dynts_aggregate_scores) and every slab ranks its selection window by that sum, so all layers
+ * and heads keep the same tokens.  Requires that all slabs of a sequence hold the same tokens,
+ * i.e. that every eviction of this cache is of this kind (or driven by shared external scores).
+ * Otherwise as dynts_evict. */
 dynts_status_t dynts_evict_global(dynts_cache_t* c, int budget);
+
+/* Appendix B.1's aggregate on its own: agg[b][j] = sum over all layers and KV heads of the score
+ * of row j of sequence b, the fp32 slab scores added in double precision and rounded to fp32 once.
+ *   agg: device [Nb, cap] fp32, caller-owned; rows [0, len(b)) of each active sequence are
+ *   written, the rest left untouched.  These are the keys dynts_evict_global ranks by. */
+dynts_status_t dynts_aggregate_scores(dynts_cache_t* c, float* agg);
 
 /* Eviction with one target per sequence; seq_targets: host [Nb]. */
 dynts_status_t dynts_evict_ex(dynts_cache_t* c, const int* seq_targets);

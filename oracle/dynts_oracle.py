@@ -315,31 +315,33 @@ def evict(cache: OracleCache, target, scores32=None):
 # Appendix B.1: one importance score per token, aggregated across all layers and heads
 # ----------------------------------------------------------------------------------------------
 
-def aggregate_scores(cache: OracleCache, seq: int, scores32=None) -> np.ndarray:
+def aggregate_scores(cache: OracleCache, seq: int) -> np.ndarray:
     """Appendix B.1 aggregates the attention a token receives across all layers and heads into one
-    importance score per token.  Online form: sum over (layer, KV head) of the slab scores of
-    sequence ``seq``, row by row (all slabs of a sequence must hold the same tokens).  The sum is
-    taken in float32, layer-major then head, because it decides an integer ranking and the device
-    adds float32 scores in that order."""
+    importance score per token.  Online form: agg[j] = sum over every layer l and KV head h of
+    score[l][seq][h][j] (all slabs of a sequence must hold the same tokens).  Plain float64 sum;
+    pinned rows (+inf) stay +inf."""
     n = cache.length(seq)
-    agg = np.zeros(n, dtype=np.float32)
+    agg = np.zeros(n, dtype=np.float64)
     for l in range(cache.layers):
         for h in range(cache.kv_heads):
             s = cache.slab(l, seq, h)
             assert s.n == n, "slabs of one sequence differ in length"
-            sc = s.score[:n].astype(np.float32) if scores32 is None else np.asarray(scores32(l, seq, h)[:n], dtype=np.float32)
-            agg = (agg + sc).astype(np.float32)
+            agg += s.score[:n]
     return agg
 
 
-def evict_global(cache: OracleCache, target, scores32=None):
+def evict_global(cache: OracleCache, target, keys32=None):
     """Section 4.2's selection taken once per sequence on the aggregated score and applied to every
-    layer and KV head: all slabs of a sequence keep the same rows.  Returns kept[b]."""
+    layer and KV head: all slabs of a sequence keep the same rows.  ``keys32(b)`` may supply the
+    float32 array the decision for sequence b is taken from (used to replay the device's decisions
+    from the device's own aggregated scores); by default the float64 aggregate, rounded once to
+    float32, decides.  Returns kept[b]."""
     kept_all = []
     for b in range(cache.batch):
         tgt = int(target if np.isscalar(target) else target[b])
         n = cache.length(b)
-        kept = select_keep(aggregate_scores(cache, b, scores32), n, cache.n_pinned[b], cache.window, tgt)
+        keys = aggregate_scores(cache, b).astype(np.float32) if keys32 is None else np.asarray(keys32(b)[:n], dtype=np.float32)
+        kept = select_keep(keys, n, cache.n_pinned[b], cache.window, tgt)
         m = len(kept)
         for l in range(cache.layers):
             for h in range(cache.kv_heads):

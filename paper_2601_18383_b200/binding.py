@@ -52,7 +52,7 @@ class dynts_config_t(C.Structure):
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
-        f"{LIB_PATH} is missing: build it with `python -m paper_2601_18383_b200.build` "
+        f"{LIB_PATH} is missing: build it with `python paper_2601_18383_b200/build.py` "
         "(there is no CPU fallback)")
 
 lib = C.CDLL(LIB_PATH)
@@ -73,6 +73,7 @@ _sigs = {
     "dynts_decode_attn_host": (C.c_int, [_P, _P, _P, _P, _P]),
     "dynts_evict": (C.c_int, [_P, C.c_int]),
     "dynts_evict_global": (C.c_int, [_P, C.c_int]),
+    "dynts_aggregate_scores": (C.c_int, [_P, _P]),
     "dynts_evict_ex": (C.c_int, [_P, C.POINTER(C.c_int)]),
     "dynts_evict_noalloc": (C.c_int, [_P, _P, _P, _P] + [C.c_int] * 8 + [_P]),
     "dynts_seq_reset": (C.c_int, [_P, C.c_int]),
@@ -201,6 +202,10 @@ def dynts_evict(c, budget=0):
 
 def dynts_evict_global(c, budget=0):
     return _check(lib.dynts_evict_global(c, budget))
+
+
+def dynts_aggregate_scores(c, agg):
+    return _check(lib.dynts_aggregate_scores(c, _ptr(agg)))
 
 
 def dynts_evict_ex(c, seq_targets: Sequence[int]):
@@ -356,6 +361,9 @@ class Cache:
 
     def evict_global(self, budget=0):
         return dynts_evict_global(self.handle, budget)
+
+    def aggregate_scores(self, agg):
+        return dynts_aggregate_scores(self.handle, agg)
 
     def evict_ex(self, targets):
         return dynts_evict_ex(self.handle, targets)

@@ -10,7 +10,6 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdynts.so")
 SOURCES = ["dynts_api.cu"]
-HEADERS = ["common.cuh", "decode_attn.cuh", "evict.cuh"]
 
 
 def _nvcc() -> str:
@@ -24,7 +23,7 @@ def _stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in SOURCES + HEADERS]
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh", ".h"))]   # every source and header
     deps.append(os.path.join(os.path.dirname(HERE), "include", "dynts.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 

@@ -585,7 +585,7 @@ dynts_status_t do_prefill(dynts_cache* c, int seq, const void* k, const void* v,
 dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validated */, bool global = false) {
   // Recorded score passes: the fused kernel applies them slab by slab before it reads the scores;
   // the other paths (aggregated keys, very long slabs) need them applied beforehand.
-  const bool fused_path = c->cap <= 12800;
+  const bool fused_path = c->cap <= (global ? 10000 : 12800);  // (the shared keys take a fifth array of the CTA's shared memory)
   if (global || !fused_path) {
     dynts_status_t fs_ = flush_pending(c);
     if (fs_ != DYNTS_OK) return fs_;
@@ -629,7 +629,6 @@ dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validat
   p.elt_bytes = c->kv_elt;
   if (global) {
     // one score per token: sum the slab scores of each sequence, every slab then ranks by the sum
-    if (c->cap > 10000) return fail(DYNTS_ERR_CAPACITY, "sequence-wide selection supports up to 10000 rows per slab");
     dynts::aggregate_scores_kernel<<<dim3((unsigned)((c->cap + 255) / 256), (unsigned)Nb, 1), 256, 0, c->stream>>>(
         c->score(), c->agg(), c->len(), c->active(), c->cfg.layers, Nb, c->cfg.kv_heads, c->cap);
     CUDA_TRY(cudaGetLastError());
@@ -911,6 +910,21 @@ dynts_status_t dynts_evict_global(dynts_cache_t* c, int budget) {
   std::vector<int> t(c->cfg.batch);
   for (int b = 0; b < c->cfg.batch; ++b) t[b] = budget > 0 ? budget : c->seq_budget[b];
   return do_evict(c, t.data(), true);
+}
+
+dynts_status_t dynts_aggregate_scores(dynts_cache_t* c, float* agg) {
+  if (!c || !agg) return fail(DYNTS_ERR_INVALID_ARG, "NULL argument");
+  if (!c->ready) return fail(DYNTS_ERR_STATE, "cache holds nothing yet");
+  if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "a layer-by-layer step is in progress");
+  {
+    dynts_status_t fs_ = flush_pending(c);
+    if (fs_ != DYNTS_OK) return fs_;
+  }
+  dynts::aggregate_scores_kernel<<<dim3((unsigned)((c->cap + 255) / 256), (unsigned)c->cfg.batch, 1), 256, 0, c->stream>>>(
+      c->score(), agg, c->len(), c->active(), c->cfg.layers, c->cfg.batch, c->cfg.kv_heads, c->cap);
+  CUDA_TRY(cudaGetLastError());
+  c->launches += 1;
+  return DYNTS_OK;
 }
 
 dynts_status_t dynts_evict_ex(dynts_cache_t* c, const int* seq_targets) {

@@ -86,6 +86,9 @@ __global__ void __launch_bounds__(kSelectThreads) evict_select_kernel(const Evic
   int* pos = p.pos + (size_t)slab * p.cap;
   int* src = p.src + (size_t)slab * p.cap;
   float* comp = p.comp ? p.comp + (size_t)slab * p.cap : nullptr;
+  // bit patterns the selection ranks by: the slab's own scores, or keys shared by all slabs of the
+  // sequence (read from global memory: such slabs may leave no shared memory for a copy)
+  const uint32_t* sel = p.key ? reinterpret_cast<const uint32_t*>(p.key + (size_t)b * p.cap) : raw;
   for (int j = tid; j < n; j += kSelectThreads) {
     raw[j] = __float_as_uint(score[j]);
     posbuf[j] = pos[j];
@@ -108,7 +111,7 @@ __global__ void __launch_bounds__(kSelectThreads) evict_select_kernel(const Evic
       const uint32_t prefix = s_prefix;
       const int krem = s_krem;  // read by everyone before warp 0 updates it below
       for (int j = lo + tid; j < hi; j += kSelectThreads) {
-        const uint32_t key = order_key(raw[j]);
+        const uint32_t key = order_key(sel[j]);
         if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
       }
       __syncthreads();
@@ -150,7 +153,7 @@ __global__ void __launch_bounds__(kSelectThreads) evict_select_kernel(const Evic
     const bool in = j < n;
     const bool cand = in && j >= lo && j < hi;
     uint32_t key = 0u;
-    if (cand) key = order_key(raw[j]);
+    if (cand) key = order_key(sel[j]);
     const bool gt = cand && k > 0 && key > T;
     const bool eq = cand && k > 0 && key == T;
     int tot_eq, tot_keep;
@@ -455,18 +458,19 @@ __global__ void __launch_bounds__(kFusedThreads) evict_fused_kernel(const EvictP
 
 // ---------------------------------------------------------------------------------------------
 // One importance score per token, aggregated across all layers and KV heads (Appendix B.1):
-// agg[b][j] = sum over (layer, head) of score[layer][b][head][j], added in float32 in that order
-// (the order is part of the result: it decides a ranking).  grid = (row blocks, sequences).
+// agg[b][j] = sum over (layer, head) of score[layer][b][head][j].  The fp32 slab scores are added
+// in double precision and the sum is rounded to fp32 once, so the key a ranking is decided by is
+// within half an ulp of the exact sum whatever the number of slabs.  grid = (row blocks, sequences).
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) aggregate_scores_kernel(const float* score, float* agg, const int* len,
                                                                const int* active, int L, int Nb, int Hkv, int cap) {
   const int b = blockIdx.y;
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (!active[b] || j >= len[b] || j >= cap) return;
-  float acc = 0.f;
+  double acc = 0.0;
   for (int l = 0; l < L; ++l)
-    for (int h = 0; h < Hkv; ++h) acc = __fadd_rn(acc, score[(((size_t)l * Nb + b) * Hkv + h) * cap + j]);
-  agg[(size_t)b * cap + j] = acc;
+    for (int h = 0; h < Hkv; ++h) acc += (double)score[(((size_t)l * Nb + b) * Hkv + h) * cap + j];
+  agg[(size_t)b * cap + j] = (float)acc;
 }
 
 // ---------------------------------------------------------------------------------------------

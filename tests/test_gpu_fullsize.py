@@ -363,3 +363,122 @@ def test_eviction_right_after_recorded_passes_equals_the_eager_path(kv8):
             assert torch.equal(H.bits(Ke), H.bits(Kl)) and torch.equal(H.bits(Ve), H.bits(Vl))
     eager.poll_error(); lazy.poll_error()
     eager.close(); lazy.close()
+
+
+def _fill(cfg, gpu, seed):
+    """Steady-state rows for every sequence: capacity - 3 rows (equal budgets) or, for a ragged
+    batch, each sequence's budget plus a seeded number of rows below the eviction interval."""
+    if cfg.seq_budgets:
+        one = cfg.scaled(batch=1)
+        r = np.random.default_rng(seed)
+        for b in range(cfg.batch):
+            n = int(cfg.seq_budgets[b] + r.integers(1, cfg.evict_interval - 3))
+            k, v = gen.torch_keys_values(one, seed + b, n, "cuda:0")
+            gpu.prefill_seq(b, k[:, 0], v[:, 0], n_pinned=cfg.prompt)
+    else:
+        k, v = gen.torch_keys_values(cfg, seed, cfg.capacity - 3, "cuda:0")
+        gpu.prefill(k, v, n_pinned=cfg.prompt)
+
+
+@pytest.mark.parametrize("name", ["c3_qwen7b", "c4_ragged"])
+def test_the_benchmarks_exact_call_at_full_size(name):
+    """decode_attn(..., scores = NULL) followed by evict, as bench.py issues them (config 3: whole-slab
+    pieces of 7 slabs per CTA whose last score pass is recorded and applied by the next launch or by
+    the eviction kernel; config 4: stream-K pieces over a ragged batch).  Sampled slabs against the
+    oracle: outputs every step, accumulated scores in the middle of the run (Eq. 6).  The eviction
+    is checked through a second cache on the same inputs that is asked for every step's mass, so
+    that all its score passes run inside their launches: its eviction must equal the oracle's
+    selection from its own float32 scores bit for bit (Section 4.2), and the first cache, evicted
+    without any read in between, must hold the same bits."""
+    cfg = W.get_config(name)
+    lazy, eager = H.make_gpu(cfg), H.make_gpu(cfg)
+    _fill(cfg, lazy, 8100)
+    _fill(cfg, eager, 8100)
+    slabs = _sample_slabs(cfg, 8, 11)
+    orc = H.oracle_from_gpu(lazy, cfg, slabs=slabs)
+    steps = 3
+    ring = gen.torch_step_ring(cfg, 8100, steps, "cuda:0")
+    ol = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda:0")
+    oe = torch.empty_like(ol)
+    delta = torch.zeros((cfg.layers, cfg.batch, cfg.kv_heads, eager.capacity), dtype=torch.float32, device="cuda:0")
+    G = cfg.group
+    for s in range(steps):
+        q, k, v = ring[0][s], ring[1][s], ring[2][s]
+        lazy.decode_attn(q, k, v, ol)                       # the benchmark's call
+        eager.decode_attn(q, k, v, oe, delta)
+        assert torch.equal(ol.view(torch.int16), oe.view(torch.int16))
+        qh, kh, vh = q.double().cpu().numpy(), k.double().cpu().numpy(), v.double().cpu().numpy()
+        og = ol.float().cpu().numpy()
+        for (l, b, h) in slabs:
+            sl = orc.slab(l, b, h)
+            sl.K[sl.n], sl.V[sl.n], sl.score[sl.n] = kh[l, b, h], vh[l, b, h], 0.0
+            sl.n += 1
+            alpha = O.attention_weights(qh[l, b, h * G:(h + 1) * G], sl.K[:sl.n])
+            sl.score[:sl.n] += alpha.sum(axis=0)
+            o_ref = O.attention_output(alpha, sl.V[:sl.n])
+            assert H.rel_err_vectors(og[l, b, h * G:(h + 1) * G], o_ref) <= H.TOL_OUT["bf16"], (s, l, b, h)
+        if s == steps - 2:                                  # a read in the middle applies what is recorded
+            sc = lazy.scores_tensor().cpu().numpy()
+            for (l, b, h) in slabs:
+                sl = orc.slab(l, b, h)
+                fin = np.isfinite(sl.score[:sl.n])
+                assert np.abs(sc[l, b, h, :sl.n][fin] - sl.score[:sl.n][fin]).max() <= H.TOL_DELTA, (s, l, b, h)
+            del sc
+    lazy.poll_error()
+    n0 = lazy.launch_count()
+    lazy.evict(0)                                           # straight after the last decode launch
+    assert lazy.launch_count() - n0 == 1
+    lazy.synchronize()
+    lazy.poll_error()
+    # the eager cache: scores against the oracle, then its eviction against the oracle's selection
+    sc = eager.scores_tensor().cpu().numpy()
+    for (l, b, h) in slabs:
+        sl = orc.slab(l, b, h)
+        fin = np.isfinite(sl.score[:sl.n])
+        assert np.abs(sc[l, b, h, :sl.n][fin] - sl.score[:sl.n][fin]).max() <= H.TOL_DELTA, (l, b, h)
+    del sc
+    H.check_evict_bit_exact(eager, cfg, 0, slabs=slabs)
+    targets = list(cfg.seq_budgets) if cfg.seq_budgets else [cfg.budget] * cfg.batch
+    assert [lazy.len(b) for b in range(cfg.batch)] == targets == [eager.len(b) for b in range(cfg.batch)]
+    for sl in slabs:
+        Ke, Ve, pe, se = eager.export_slab(*sl)
+        Kl, Vl, pl, s_l = lazy.export_slab(*sl)
+        assert torch.equal(pe, pl) and torch.equal(H.bits(se), H.bits(s_l)), sl
+        assert torch.equal(H.bits(Ke), H.bits(Kl)) and torch.equal(H.bits(Ve), H.bits(Vl)), sl
+    lazy.close()
+    eager.close()
+    torch.cuda.empty_cache()
+
+
+def test_sequence_wide_selection_on_full_kv_length_slabs():
+    """dynts_evict_global on slabs too long for the fused kernel (16640 rows): the two-kernel path
+    ranks every slab by the keys shared across the sequence (Appendix B.1)."""
+    cfg = W.get_config("c2_llama8b").scaled(name="full_kv_global", layers=2, batch=1, kv_heads=2, q_heads=8, budget=16640,
+                                             window=128, evict_interval=64, prompt=256, density=0.01)
+    gpu = _steady_state(cfg, 6200, 16640 - 2)
+    ring = gen.torch_step_ring(cfg, 6200, 2, "cuda:0")
+    out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda:0")
+    for s in range(2):
+        gpu.decode_attn(ring[0][s], ring[1][s], ring[2][s], out)
+    n = gpu.len(0)
+    assert n == 16640
+    keys_t = torch.zeros((cfg.batch, gpu.capacity), dtype=torch.float32, device="cuda:0")
+    gpu.aggregate_scores(keys_t)
+    keys = keys_t.cpu().numpy()
+    sc = gpu.scores_tensor().cpu().numpy()
+    exact = sc[:, 0, :, :n].astype(np.float64).sum(axis=(0, 1))
+    fin = np.isfinite(exact)
+    assert np.abs(keys[0, :n][fin] - exact[fin]).max() <= 1e-4 * cfg.layers * cfg.kv_heads
+    pre = H.export_all(gpu, cfg)
+    gpu.evict_global(12000)
+    gpu.synchronize()
+    gpu.poll_error()
+    kept = O.select_keep(keys[0, :n], n, cfg.prompt, cfg.window, 12000)
+    idx = torch.from_numpy(kept)
+    assert gpu.len(0) == 12000 == len(kept)
+    for key, (K0, V0, p0, s0) in pre.items():
+        K1, V1, p1, s1 = gpu.export_slab(*key)
+        assert torch.equal(p1, p0[idx]) and torch.equal(H.bits(s1), H.bits(s0[idx])), key
+        assert torch.equal(H.bits(K1), H.bits(K0[idx])) and torch.equal(H.bits(V1), H.bits(V0[idx])), key
+    gpu.close()
+    torch.cuda.empty_cache()

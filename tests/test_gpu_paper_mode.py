@@ -121,7 +121,7 @@ def test_sequence_wide_selection_on_aggregated_scores(name):
     stream = W.DecodeStream(cfg, 31)
     out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=H.tdtype(cfg), device="cuda:0")
     events = moved = 0
-    worst_score = 0.0
+    worst_score = worst_key = 0.0
     for s in range(1, 225):
         q, k, v = stream.step(s)
         gpu.decode_attn(H.dev(q, cfg), H.dev(k, cfg), H.dev(v, cfg), out)
@@ -134,10 +134,22 @@ def test_sequence_wide_selection_on_aggregated_scores(name):
             fin = np.isfinite(sl.score[:sl.n])
             worst_score = max(worst_score, float(np.abs(sc[l, b, h, :sl.n][fin] - sl.score[:sl.n][fin]).max()))
         n_before = gpu.len(0)
+        # the device's aggregated keys: within rounding of the float64 sum of its own slab scores
+        # (Appendix B.1), and the array the oracle's selection is taken from
+        keys_t = torch.full((cfg.batch, gpu.capacity), float("nan"), dtype=torch.float32, device="cuda:0")
+        gpu.aggregate_scores(keys_t)
+        keys = keys_t.cpu().numpy()
+        n_slabs = cfg.layers * cfg.kv_heads
+        for b in range(cfg.batch):
+            exact = sc[:, b, :, :n_before].astype(np.float64).sum(axis=(0, 1))
+            fin = np.isfinite(exact)
+            assert np.array_equal(np.isinf(keys[b, :n_before]), ~fin)
+            worst_key = max(worst_key, float(np.abs(keys[b, :n_before][fin] - exact[fin]).max()))
+            assert np.isnan(keys[b, n_before:]).all()              # rows beyond the length are left alone
         gpu.evict_global(0)
         gpu.synchronize()
         gpu.poll_error()
-        kept = O.evict_global(orc, cfg.budget, scores32=lambda l, b, h: sc[l, b, h])
+        kept = O.evict_global(orc, cfg.budget, keys32=lambda b: keys[b])
         for l, b, h, sl in orc.units():
             K0, V0, p0, s0 = pre[(l, b, h)]
             K1, V1, p1, s1 = gpu.export_slab(l, b, h)
@@ -151,4 +163,5 @@ def test_sequence_wide_selection_on_aggregated_scores(name):
             events += 1
             moved += sum(int((kk != np.arange(len(kk))).sum()) for kk in kept)
     assert events >= 3 and moved > 0 and worst_score <= H.TOL_DELTA, (events, moved, worst_score)
+    assert worst_key <= 1e-4 * cfg.layers * cfg.kv_heads, worst_key
     gpu.close()

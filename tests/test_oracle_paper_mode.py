@@ -134,27 +134,69 @@ def test_accumulate_off_leaves_scores_alone():
     assert sl.score[12] == np.float32(0.25)
 
 
+def _decoded_cache(cfg, seed, steps, n_pinned=None, cap=80):
+    orc = O.OracleCache(cfg.layers, cfg.batch, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.window, cap)
+    pk, pv = W.prompt_kv(cfg, seed)
+    O.prefill(orc, pk.astype(np.float64), pv.astype(np.float64), n_pinned=n_pinned)
+    st = W.DecodeStream(cfg, seed)
+    for s in range(1, steps + 1):
+        O.decode_step(orc, *[x.astype(np.float64) for x in st.step(s)])
+    return orc
+
+
+def test_aggregated_mass_is_conserved_across_layers_and_heads():
+    """Appendix B.1 / Eq. 6: every decode step hands out a mass of 1 per query head, so with no
+    pinned row and no eviction the aggregate over all layers and heads sums to
+    layers x q_heads x steps.  A dropped layer or head breaks the total."""
+    cfg = _small_cfg(layers=3, batch=2, kv_heads=2, q_heads=4)
+    steps = 25
+    orc = _decoded_cache(cfg, 8, steps, n_pinned=0)
+    for b in range(cfg.batch):
+        agg = O.aggregate_scores(orc, b)
+        assert agg.dtype == np.float64 and agg.shape == (cfg.prompt + steps,)
+        assert np.all(agg >= 0)
+        assert abs(agg.sum() - cfg.layers * cfg.q_heads * steps) < 1e-9
+        # the row appended by the last step has been attended to once, by every head of every layer
+        assert 0 < agg[-1] <= cfg.layers * cfg.q_heads
+
+
+def test_aggregate_of_hand_set_scores_has_the_closed_form_and_ignores_slab_order():
+    """score[l][h][j] = 10 (l + 1) + h + j / 2 has the aggregate
+    Hkv * 10 * L (L + 1) / 2 + L * Hkv (Hkv - 1) / 2 + L * Hkv * j / 2; it equals the library sum over
+    the stacked slabs and does not change when layers and heads are permuted."""
+    L, Hkv, n = 3, 2, 20
+    cfg = _small_cfg(layers=L, batch=1, kv_heads=Hkv, q_heads=4)
+    orc = _decoded_cache(cfg, 11, n - cfg.prompt, n_pinned=0)
+    j = np.arange(n, dtype=np.float64)
+    for l in range(L):
+        for h in range(Hkv):
+            orc.slab(l, 0, h).score[:n] = 10.0 * (l + 1) + h + j / 2
+    expect = Hkv * 10.0 * L * (L + 1) / 2 + L * Hkv * (Hkv - 1) / 2 + L * Hkv * j / 2
+    agg = O.aggregate_scores(orc, 0)
+    assert np.array_equal(agg, expect)
+    stacked = np.stack([orc.slab(l, 0, h).score[:n] for l in range(L) for h in range(Hkv)])
+    assert np.array_equal(agg, stacked.sum(axis=0))
+    perm = np.random.default_rng(3).permutation(L * Hkv)
+    rows = stacked[perm]
+    for i, (l, h) in enumerate((l, h) for l in range(L) for h in range(Hkv)):
+        orc.slab(l, 0, h).score[:n] = rows[i]
+    assert np.array_equal(O.aggregate_scores(orc, 0), expect)
+    # one pinned row in one slab pins the token's aggregate
+    orc.slab(1, 0, 1).score[4] = np.inf
+    assert O.aggregate_scores(orc, 0)[4] == np.inf
+
+
 def test_global_selection_shares_one_retained_set_and_matches_brute_force():
     cfg = _small_cfg(layers=3, batch=2, kv_heads=2, q_heads=4)
-    orc = O.OracleCache(cfg.layers, cfg.batch, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.window, 80)
-    pk, pv = W.prompt_kv(cfg, 8)
-    O.prefill(orc, pk.astype(np.float64), pv.astype(np.float64))
-    st = W.DecodeStream(cfg, 8)
-    for s in range(1, 41):
-        O.decode_step(orc, *[x.astype(np.float64) for x in st.step(s)])
+    orc = _decoded_cache(cfg, 8, 40)
     n = orc.length(0)
-    # brute force: sum the float32 scores of all slabs of a sequence, rank the selection window
+    # brute force on the float64 aggregate: rank the selection window by (sum descending, index)
     expect = []
     for b in range(cfg.batch):
-        tot = np.zeros(n, dtype=np.float32)
-        for l in range(cfg.layers):
-            for h in range(cfg.kv_heads):
-                tot = (tot + orc.slab(l, b, h).score[:n].astype(np.float32)).astype(np.float32)
-        assert np.array_equal(tot, O.aggregate_scores(orc, b))
-        # every step adds G mass per KV head: layers * q_heads per step in total, over the finite rows
-        fin = np.isfinite(tot)
-        assert abs(float(tot[fin].sum()) + 0 - 0) > 0
+        tot = np.stack([orc.slab(l, b, h).score[:n] for l in range(cfg.layers) for h in range(cfg.kv_heads)]).sum(axis=0)
         cand = list(range(cfg.prompt, n - cfg.window))
+        gaps = np.diff(np.sort(tot[cand]))
+        assert gaps.min() > 1e-4 * tot[cand].max()       # well separated: rounding to float32 cannot reorder them
         k = 40 - cfg.prompt - cfg.window
         best = sorted(sorted(cand, key=lambda j: (-tot[j], j))[:k])
         expect.append(list(range(cfg.prompt)) + best + list(range(n - cfg.window, n)))
@@ -166,6 +208,28 @@ def test_global_selection_shares_one_retained_set_and_matches_brute_force():
             for h in range(cfg.kv_heads):
                 sl = orc.slab(l, b, h)
                 assert sl.n == 40 and np.array_equal(sl.pos[:40], pos_before[b][kept[b]])
+
+
+def test_global_selection_sees_every_slab_and_takes_supplied_keys():
+    """A row that only ONE slab rates highly (by a margin above all other sums) must survive in all
+    slabs; keys handed in replace the aggregate."""
+    cfg = _small_cfg(layers=3, batch=1, kv_heads=2, q_heads=4)
+    for (l, h) in [(0, 0), (2, 1), (1, 0)]:
+        orc = _decoded_cache(cfg, 13, 40)
+        n = orc.length(0)
+        cand = np.arange(cfg.prompt, n - cfg.window)
+        low = cand[np.argmin(O.aggregate_scores(orc, 0)[cand])]      # would be evicted first ...
+        kept0 = O.evict_global(_decoded_cache(cfg, 13, 40), 40)[0]
+        assert low not in kept0
+        orc.slab(l, 0, h).score[low] += 1e6                           # ... unless this one slab says otherwise
+        kept = O.evict_global(orc, 40)[0]
+        assert low in kept
+    orc = _decoded_cache(cfg, 13, 40)
+    n = orc.length(0)
+    keys = np.arange(n, dtype=np.float32)                             # supplied keys: later rows rank higher
+    kept = O.evict_global(orc, 40, keys32=lambda b: keys)[0]
+    k = 40 - cfg.prompt - cfg.window
+    assert kept.tolist() == list(range(cfg.prompt)) + list(range(n - cfg.window - k, n))
 
 
 def test_global_selection_with_one_slab_is_the_per_slab_selection():
