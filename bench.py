@@ -51,7 +51,7 @@ class ClockSampler(threading.Thread):
     def __init__(self, index: int, period_s: float = 0.02):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.times, self.reasons, self.max_mhz = [], [], set(), None
         self._stop_evt = threading.Event()
         self.ok = False
         try:
@@ -77,6 +77,7 @@ class ClockSampler(threading.Thread):
         while not self._stop_evt.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                self.times.append(time.perf_counter())
                 r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
                 for bit, name in names.items():
                     if r & bit:
@@ -106,8 +107,25 @@ def physical_gpu_index(local_index: int) -> int:
     return local_index
 
 
-def setup_cache(cfg, seed, device, kv8=False):
-    """A cache in steady state: every sequence holds `budget` rows (the prompt rows pinned)."""
+def workload_config(cfg, args, world):
+    """The `config` object of the JSON line: a description of the workload that both arms print
+    alike (nothing in it depends on which implementation ran)."""
+    kv8 = args.kv_dtype == "fp8"
+    elt = 1 if kv8 else (2 if cfg.dtype == "bf16" else 4)
+    kv_bytes = cfg.layers * cfg.batch * cfg.kv_heads * cfg.capacity * 2 * cfg.head_dim * elt
+    return {"workload": cfg.name, "layers": cfg.layers, "batch": cfg.batch, "q_heads": cfg.q_heads,
+            "kv_heads": cfg.kv_heads, "head_dim": cfg.head_dim, "budget": cfg.budget, "window": cfg.window,
+            "evict_interval": cfg.evict_interval, "prompt_pinned": cfg.prompt, "dist": cfg.dist,
+            "score_source": args.score_source, "selection": args.selection,
+            "kv_dtype": "e4m3 codes, scale 1/32" if kv8 else cfg.dtype,
+            "kv_bytes": kv_bytes,
+            "l2_policy": "inputs larger than L2 (K/V slabs %.0f MB vs 126 MB L2)" % (kv_bytes / 1e6),
+            "replicas": world}
+
+
+def setup_cache(cfg, seed, device, kv8=False, u=None):
+    """A cache in steady state: every sequence holds `budget` rows (the prompt rows pinned).  u: the
+    planted directions the decode queries will be aligned with (the fill's critical keys use them)."""
     import torch
     import paper_2601_18383_b200 as D
     cache = D.Cache(cfg.layers, cfg.batch, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.budget, cfg.window,
@@ -117,10 +135,10 @@ def setup_cache(cfg, seed, device, kv8=False):
     if cfg.seq_budgets:
         one = cfg.scaled(batch=1)
         for b in range(cfg.batch):
-            k, v = gen.torch_keys_values(one, seed + b, cfg.seq_budgets[b], device)
+            k, v = gen.torch_keys_values(one, seed + b, cfg.seq_budgets[b], device, u=None if u is None else u[:, b:b + 1])
             cache.prefill_seq(b, k[:, 0], v[:, 0], n_pinned=cfg.prompt)
     else:
-        k, v = gen.torch_keys_values(cfg, seed, cfg.budget, device)
+        k, v = gen.torch_keys_values(cfg, seed, cfg.budget, device, u=u)
         cache.prefill(k, v, n_pinned=cfg.prompt)
     del k, v
     torch.cuda.empty_cache()
@@ -140,8 +158,13 @@ def run_ours(args, cfg, rank, world, device):
     kv8 = args.kv_dtype == "fp8"
     if kv8 and (cfg.dtype != "bf16" or cfg.head_dim % 16):
         raise SystemExit("--kv-dtype fp8 needs a bf16 workload")
-    cache = setup_cache(cfg, 1000 * int(cfg.name[1]) + rank, device, kv8)
-    q_ring, k_ring, v_ring = gen.torch_step_ring(cfg, 77 + rank, ring_n, device)
+    seed = 1000 * int(cfg.name[1]) + rank
+    # one set of planted directions for the steady-state fill and for the decode queries
+    u = gen.torch_unit_dirs(cfg, seed, device) if cfg.dist == "planted" else None
+    cache = setup_cache(cfg, seed, device, kv8, u=u)
+    if args.evict_split:
+        cache.set_evict_launch(args.evict_split)
+    q_ring, k_ring, v_ring = gen.torch_step_ring(cfg, 77 + rank, ring_n, device, u=u)
     out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, cfg.head_dim), dtype=q_ring.dtype, device=device)
     stream = torch.cuda.current_stream(device)
     external = args.score_source == "external"
@@ -155,32 +178,47 @@ def run_ours(args, cfg, rank, world, device):
         s_ring = torch.randn((ring_n, cfg.batch), generator=g, device=device)   # stand-in for predictor outputs
 
     evict_call = cache.evict_global if args.selection == "global" else cache.evict
+    peak, peak_kind = measured_peaks()
+    elt = 1 if kv8 else (2 if cfg.dtype == "bf16" else 4)
+    row_move_bytes = 2 * (2 * cfg.head_dim * elt + 8)      # K row + V row + pos + score, read and written
 
     def decode(j):
         cache.decode_attn(q_ring[j], k_ring[j], v_ring[j], out)
         if external:
             cache.append_scores(s_ring[j])
 
-    cycle = {"since": 0}      # decode steps since the last eviction, kept across the phases below
+    state = {"since": 0, "i": 0, "evictions": 0}      # decode steps since the last eviction, kept across the phases below
 
-    def step(i):
-        decode(i % ring_n)
-        cycle["since"] += 1
-        if cycle["since"] == E:
+    def step():
+        decode(state["i"] % ring_n)
+        state["i"] += 1
+        state["since"] += 1
+        if state["since"] == E:
             evict_call(0)
-            cycle["since"] = 0
+            state["since"] = 0
+            state["evictions"] += 1
+
+    def finish_cycle():
+        while state["since"] != 0:
+            step()
+
+    def step_bytes():
+        return bytes_per_slot * slots_in_step(cfg, [cache.len(bb) + 1 for bb in range(cfg.batch)])
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize(device)
 
+    def event():
+        return torch.cuda.Event(enable_timing=True)
+
     # warm-up: the requested steps rounded up to whole eviction cycles (at least one), so that scores and
     # selection are non-trivial and the timed region starts at the beginning of a cycle
     warm = max(args.warmup, 3)
     warm = (warm + E - 1) // E * E
-    for i in range(warm):
-        step(i)
+    for _ in range(warm):
+        step()
     barrier()
     cache.poll_error()
 
@@ -189,19 +227,18 @@ def run_ours(args, cfg, rank, world, device):
     sampler = ClockSampler(physical_gpu_index(torch.cuda.current_device()))
     sampler.start()
     launches0 = cache.launch_count()
-    lens = [cache.len(b) for b in range(cfg.batch)]
-    slot_steps = 0
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev_before = state["evictions"]
+    ev0, ev1 = event(), event()
     barrier()
     ev0.record(stream)
-    for i in range(K):
-        slot_steps += slots_in_step(cfg, [cache.len(b) + 1 for b in range(cfg.batch)])
-        step(i)
+    for _ in range(K):
+        step()
     ev1.record(stream)
     barrier()
     ms = ev0.elapsed_time(ev1)
     clocks = sampler.stop()
     launches = cache.launch_count() - launches0
+    evictions_in_region = state["evictions"] - ev_before
     cache.poll_error()
     if world > 1:
         t = torch.tensor([ms], device=device)
@@ -210,40 +247,52 @@ def run_ours(args, cfg, rank, world, device):
     tokens = cfg.batch * K * world
     value = tokens / (ms * 1e-3)
 
-    # ---- per-kernel durations (separate pass: event pairs around every launch) -----------------
-    Kp = min(K, 8 * E)
-    elt = 1 if kv8 else (2 if cfg.dtype == "bf16" else 4)
-    row_move_bytes = 2 * (2 * cfg.head_dim * elt + 8)      # K row + V row + pos + score, read and written
-    # One event pair per run of back-to-back decode launches (the E launches between two evictions)
-    # and one per eviction: the average launch duration includes the gaps between launches, as in
-    # the timed region.
-    dec_events, ev_events, dec_bytes = [], [], []
-    i = 0
-    while i < Kp:
-        run = min(E - cycle["since"], Kp - i)   # (the timed region may have stopped in the middle of a cycle)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        for j in range(i, i + run):
-            dec_bytes.append(bytes_per_slot * slots_in_step(cfg, [cache.len(bb) + 1 for bb in range(cfg.batch)]))
-            decode(j % ring_n)
-        b.record(stream)
-        dec_events.append((a, b, run))
-        i += run
-        cycle["since"] += run
-        if cycle["since"] == E:
-            cycle["since"] = 0
-            a2, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a2.record(stream)
+    # ---- per-kernel durations: whole eviction cycles, whatever K is -------------------------------
+    # Every cycle is E back-to-back decode launches (one event pair around the run, so the average
+    # launch duration includes the gaps between launches, as in the timed region) and the eviction
+    # that follows (its own event pair).  At least 4 cycles, so at least 4 eviction events are timed.
+    finish_cycle()
+    n_cyc = max(4, min((K + E - 1) // E, 8))
+
+    def timed_cycles(n):
+        dec_runs, ev_events = [], []
+        for _ in range(n):
+            a, b, c = event(), event(), event()
+            run_bytes = 0
+            a.record(stream)
+            for _j in range(E):
+                run_bytes += step_bytes()
+                decode(state["i"] % ring_n)
+                state["i"] += 1
+            b.record(stream)
             evict_call(0)
-            b2.record(stream)
-            scanned, moved = cache.evict_stats()           # synchronises; outside the event pair
-            ev_events.append((a2, b2, 4 * scanned + row_move_bytes * moved))
-    torch.cuda.synchronize(device)
-    dec_launches = sum(r for _, _, r in dec_events)
-    dec_avg_ms = sum(a.elapsed_time(b) for a, b, _ in dec_events) / dec_launches
-    dec_gbs = (sum(dec_bytes) / len(dec_bytes)) / (dec_avg_ms * 1e-3) / 1e9
-    peak, peak_kind = measured_peaks()
-    algo_bytes = sum(dec_bytes) / len(dec_bytes)
+            c.record(stream)
+            state["evictions"] += 1
+            scanned, moved = cache.evict_stats()           # synchronises; outside the event pairs
+            dec_runs.append((a, b, run_bytes))
+            ev_events.append((b, c, 4 * scanned + row_move_bytes * moved, moved))
+        torch.cuda.synchronize(device)
+        cache.poll_error()
+        return dec_runs, ev_events
+
+    def evict_summary(ev_events):
+        ev_ms = [a.elapsed_time(b) for a, b, _, _ in ev_events]
+        ev_bytes = sum(x for _, _, x, _ in ev_events) / len(ev_events)
+        ev_avg = sum(ev_ms) / len(ev_ms)
+        ev_gbs = ev_bytes / (ev_avg * 1e-3) / 1e9 if ev_avg > 0 else 0.0
+        return {"kernels": "evict (selection + in-place compaction, one launch)", "bound": "hbm", "achieved": round(ev_gbs, 1),
+                "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": round(ev_gbs / peak, 4),
+                "algorithmic_bytes_per_event": int(ev_bytes),
+                "rows_moved_per_event": int(sum(m for _, _, _, m in ev_events) / len(ev_events)),
+                "avg_event_us": round(1e3 * ev_avg, 2), "min_event_us": round(1e3 * min(ev_ms), 2),
+                "evict_per_step_us": round(1e3 * ev_avg / E, 3), "events_timed": len(ev_ms),
+                "decode_steps_before": state["i"]}, ev_avg, ev_bytes
+
+    dec_runs, ev_events = timed_cycles(n_cyc)
+    dec_launches = n_cyc * E
+    dec_avg_ms = sum(a.elapsed_time(b) for a, b, _ in dec_runs) / dec_launches
+    algo_bytes = sum(x for _, _, x in dec_runs) / dec_launches
+    dec_gbs = algo_bytes / (dec_avg_ms * 1e-3) / 1e9
     roofline = {
         "kernel": "decode_attn (fused append + attention" + (" + append of the token's predictor score)" if external
                                                                  else " + importance accumulation)"),
@@ -253,56 +302,122 @@ def run_ours(args, cfg, rank, world, device):
         "algorithmic_bytes_per_launch": int(algo_bytes), "avg_launch_us": round(dec_avg_ms * 1e3, 2),
         "launches_timed": dec_launches,
     }
-    evict = None
-    if ev_events:
-        ev_ms = [a.elapsed_time(b) for a, b, _ in ev_events]
-        ev_bytes = sum(x for _, _, x in ev_events) / len(ev_events)
-        ev_avg = sum(ev_ms) / len(ev_ms)
-        ev_gbs = ev_bytes / (ev_avg * 1e-3) / 1e9 if ev_avg > 0 else 0.0
-        evict = {"kernels": "evict_fused (selection + in-place compaction, one launch)", "bound": "hbm", "achieved": round(ev_gbs, 1), "peak": peak,
-                 "unit": "GB/s", "frac": round(ev_gbs / peak, 4), "algorithmic_bytes_per_event": int(ev_bytes),
-                 "avg_event_us": round(1e3 * ev_avg, 2), "events_timed": len(ev_ms)}
+    evict, ev_avg, ev_bytes = evict_summary(ev_events)
 
-    # ---- end to end through the host-buffer entry point ----------------------------------------
+    # ---- whole cycles without inner events: E decode steps + 1 eviction ----------------------------
+    cyc = []
+    for _ in range(n_cyc):
+        a, c = event(), event()
+        nbytes = 0
+        a.record(stream)
+        for _j in range(E):
+            nbytes += step_bytes()
+            decode(state["i"] % ring_n)
+            state["i"] += 1
+        evict_call(0)
+        c.record(stream)
+        state["evictions"] += 1
+        cyc.append((a, c, nbytes))
+    torch.cuda.synchronize(device)
+    cyc_ms = sum(a.elapsed_time(c) for a, c, _ in cyc) / n_cyc
+    cyc_bytes = sum(x for _, _, x in cyc) / n_cyc + ev_bytes
+    cycle = {"decode_steps": E, "evictions": 1, "ms": round(cyc_ms, 4), "tokens_per_s": round(cfg.batch * E * world / (cyc_ms * 1e-3), 1),
+             "algorithmic_bytes": int(cyc_bytes), "achieved": round(cyc_bytes / (cyc_ms * 1e-3) / 1e9, 1), "unit": "GB/s",
+             "frac": round(cyc_bytes / (cyc_ms * 1e-3) / 1e9 / peak, 4), "evict_share": round(ev_avg / cyc_ms, 4), "cycles_timed": n_cyc}
+
+    # ---- sustained: whole cycles for at least args.sustain_seconds, clocks sampled throughout --------------
+    sustained = evict_aged = None
+    if args.sustain_seconds > 0:
+        n_sus = max(2, int(args.sustain_seconds * 1e3 / cyc_ms) + 1)
+        sus_sampler = ClockSampler(physical_gpu_index(torch.cuda.current_device()))
+        marks = [event() for _ in range(n_sus + 1)]
+        barrier()
+        sus_sampler.start()
+        t_start = time.perf_counter()
+        marks[0].record(stream)
+        for ci in range(n_sus):
+            for _j in range(E):
+                decode(state["i"] % ring_n)
+                state["i"] += 1
+            evict_call(0)
+            state["evictions"] += 1
+            marks[ci + 1].record(stream)
+        barrier()
+        sus_clk = sus_sampler.stop()
+        ends = [marks[0].elapsed_time(m) for m in marks[1:]]            # ms since the start, on the device
+        total_ms = ends[-1]
+        if world > 1:
+            t = torch.tensor([total_ms], device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            total_ms = float(t.item())
+        # each cycle is attributed to the clock sample nearest to its middle, then binned by 50 MHz
+        bins = {}
+        if sus_sampler.samples:
+            ts = np.asarray(sus_sampler.times) - t_start
+            mhz = np.asarray(sus_sampler.samples, dtype=np.float64)
+            prev = 0.0
+            for e_ms in ends:
+                mid = 0.5e-3 * (prev + e_ms)
+                f = float(mhz[int(np.argmin(np.abs(ts - mid)))])
+                key = int(round(f / 50.0) * 50)
+                d = bins.setdefault(key, [0, 0.0])
+                d[0] += 1
+                d[1] += e_ms - prev
+                prev = e_ms
+        med = sus_clk["sm_mhz"]
+        sustained = {"seconds": round(total_ms * 1e-3, 3), "cycles": n_sus, "steps": n_sus * E,
+                     "tokens_per_s": round(cfg.batch * n_sus * E * world / (total_ms * 1e-3), 1),
+                     "ms_per_step": round(total_ms / (n_sus * E), 5),
+                     "clocks": sus_clk,
+                     "step_us_x_sm_ghz": None if not med else round(total_ms * 1e3 / (n_sus * E) * med * 1e-3, 3),
+                     "by_sm_mhz": [{"sm_mhz": k_, "cycles": v_[0], "tokens_per_s": round(cfg.batch * v_[0] * E * world / (v_[1] * 1e-3), 1)}
+                                   for k_, v_ in sorted(bins.items())]}
+        cache.poll_error()
+        # the same eviction measurement on the aged cache: which rows an event evicts, and so how many
+        # rows it moves, changes as the steady-state fill is replaced by decoded rows
+        evict_aged = evict_summary(timed_cycles(4)[1])[0]
+
+    # ---- end to end through the host-buffer entry point: whole cycles, evictions included ---------
     e2e = None
     if rank == 0 or world > 1:
-        Ke = min(K, 4 * E)
+        Ke = min(max(K, E), 4 * E)
+        Ke = (Ke + E - 1) // E * E                     # whole cycles: every E-th step is followed by its eviction
         hq = [q_ring[j].cpu().pin_memory() for j in range(ring_n)]
         hk = [k_ring[j].cpu().pin_memory() for j in range(ring_n)]
         hv = [v_ring[j].cpu().pin_memory() for j in range(ring_n)]
         hout = torch.empty(out.shape, dtype=out.dtype).pin_memory()
-        for i in range(3):
+        for i in range(3):                             # warm-up of the entry point (staging set-up), then back to a cycle start
             cache.decode_attn_host(hq[i], hk[i], hv[i], hout)
-        # re-align to the eviction cycle
-        while cache.len(0) % 1 == 0 and any(cache.len(bb) >= cache.capacity for bb in range(cfg.batch)):
-            evict_call(0)
+        state["since"] = 3
+        finish_cycle()
         barrier()
         t0 = time.perf_counter()
-        steps_done = 0
+        e2e_evictions = 0
         for i in range(Ke):
-            if any(cache.len(bb) + 1 > cache.capacity for bb in range(cfg.batch)):
+            cache.decode_attn_host(hq[i % ring_n], hk[i % ring_n], hv[i % ring_n], hout)   # returns when `out` is on the host
+            if (i + 1) % E == 0:
                 evict_call(0)
-            cache.decode_attn_host(hq[i % ring_n], hk[i % ring_n], hv[i % ring_n], hout)
-            steps_done += 1
+                e2e_evictions += 1
         torch.cuda.synchronize(device)
         dt = time.perf_counter() - t0
         if world > 1:
             t = torch.tensor([dt], device=device)
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             dt = float(t.item())
-        e2e = {"value": round(cfg.batch * steps_done * world / dt, 1), "unit": UNIT,
+        e2e = {"value": round(cfg.batch * Ke * world / dt, 1), "unit": UNIT,
                "h2d_bytes_per_step": int(hq[0].numel() * hq[0].element_size() + 2 * hk[0].numel() * hk[0].element_size()),
-               "d2h_bytes_per_step": int(hout.numel() * hout.element_size()), "steps": steps_done,
-               "api": "dynts_decode_attn_host + dynts_evict"}
+               "d2h_bytes_per_step": int(hout.numel() * hout.element_size()), "steps": Ke, "evictions": e2e_evictions,
+               "api": "dynts_decode_attn_host every step + dynts_evict every %d steps" % E}
+        cache.poll_error()
 
     # ---- Importance Predictor head (Section 4.1): d -> 2d -> d/2 -> 1 at Llama-8B width -----------
     predictor = None
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and not args.no_extras:
         predictor = time_predictor(cfg.batch, device, peak)
 
     # ---- prefill attention of the prompt (dense: tensor-bound) ------------------------------------
     prefill = None
-    if rank == 0 and world == 1 and cfg.dtype == "bf16" and cfg.head_dim == 128:
+    if rank == 0 and world == 1 and cfg.dtype == "bf16" and cfg.head_dim == 128 and not args.no_extras:
         prefill = time_prefill(cfg, device)
 
     # ---- CPU baseline: the oracle, as it stands, on this machine's host cores (rank 0, N = 1) ------
@@ -310,17 +425,17 @@ def run_ours(args, cfg, rank, world, device):
     if rank == 0 and world == 1 and not args.no_cpu_baseline and not kv8:
         cpu = oracle_baseline(cfg, cache, q_ring, k_ring, v_ring, budget_s=args.cpu_seconds)
 
+    config = workload_config(cfg, args, world)
     result = {
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
         "ms_per_step": round(ms / K, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": cfg.name, "layers": cfg.layers, "batch": cfg.batch, "q_heads": cfg.q_heads,
-                   "kv_heads": cfg.kv_heads, "head_dim": cfg.head_dim, "budget": cfg.budget, "window": cfg.window,
-                   "evict_interval": E, "warmup_steps_run": warm, "prompt_pinned": cfg.prompt, "dist": cfg.dist, "score_source": args.score_source, "selection": args.selection, "kv_dtype": "e4m3 codes, scale 1/32" if kv8 else cfg.dtype, "accumulate": "fp32 (softmax, output, scores)",
-                   "cache_bytes": cache.nbytes, "l2_policy": "inputs larger than L2 (KV cache %.0f MB vs 126 MB L2)" % (cache.nbytes / 1e6),
-                   "replicas": world},
-        "hbm_gbs_decode": round(dec_gbs, 1), "roofline": roofline, "evict": evict, "e2e": e2e,
-        "predictor_mlp": predictor, "prefill_attn": prefill, "cpu_baseline": cpu, "clocks": clocks, "gpu_launches": int(launches),
+        "config": config,
+        "run": {"warmup_steps_run": warm, "evictions_in_timed_region": evictions_in_region, "cache_bytes": cache.nbytes,
+                "accumulate": "fp32 (softmax, output, scores)"},
+        "hbm_gbs_decode": round(dec_gbs, 1), "roofline": roofline, "evict": evict, "evict_aged": evict_aged, "cycle": cycle, "sustained": sustained,
+        "e2e": e2e, "predictor_mlp": predictor, "prefill_attn": prefill, "cpu_baseline": cpu, "clocks": clocks,
+        "gpu_launches": int(launches),
     }
     cache.close()
     return result
@@ -494,9 +609,7 @@ def run_reference(args, cfg, rank, world):
         "impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt / args.steps * 1e3 * (total_slabs / used), 3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": cfg.name, "layers": cfg.layers, "batch": cfg.batch, "q_heads": cfg.q_heads,
-                   "kv_heads": cfg.kv_heads, "head_dim": cfg.head_dim, "budget": cfg.budget, "window": cfg.window,
-                   "evict_interval": cfg.evict_interval},
+        "config": workload_config(cfg, args, world),
         "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": int(threads), "kind": "oracle", "sample": sample},
         "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -512,12 +625,16 @@ def main():
     ap.add_argument("--workload", default="c2_llama8b", choices=sorted(W.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--sustain-seconds", type=float, default=2.0,
+                    help="length of the sustained region that follows the K timed steps (0: skip it)")
+    ap.add_argument("--no-extras", action="store_true", help="skip the predictor-head and prefill-attention timings")
     ap.add_argument("--score-source", default="attention", choices=["attention", "external"],
                     help="attention: Eq. 6 mass accumulated online (default); external: one predictor score per token (Eq. 7)")
     ap.add_argument("--selection", default="slab", choices=["slab", "global"],
                     help="slab: every (layer, KV head) selects on its own scores; global: one selection per sequence")
     ap.add_argument("--kv-dtype", default="bf16", choices=["bf16", "fp8"],
                     help="fp8: the slabs hold E4M3 codes (q, k, v, out stay bf16); bf16 workloads only")
+    ap.add_argument("--evict-split", type=int, default=0, help="CTAs per slab of the eviction kernel (0: automatic; tuning)")
     ap.add_argument("--cluster", type=int, default=0)
     ap.add_argument("--variant", type=int, default=0)
     args = ap.parse_args()

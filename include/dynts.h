@@ -294,6 +294,14 @@ dynts_status_t dynts_synchronize(dynts_cache_t* c);
  * 8 or 16; 0 => automatic); for variant 3 the CTAs per SM (1 or 2; anything else => 2). */
 dynts_status_t dynts_cache_set_launch(dynts_cache_t* c, int cluster, int variant);
 
+/* Launch configuration of the eviction kernel, for tuning.  split: 1, 2, 4 or 8 => the kernel that
+ * keeps every thread's rows in registers, with that many CTAs sharing one slab (each takes the
+ * selection decision for itself and moves its own share of the row bytes; slabs of up to 4352
+ * rows, the count is halved until the row size allows it); -1 => the one-CTA-per-slab kernel that
+ * keeps its keys in shared memory; 0 => automatic (the register kernel for slabs of up to 2304
+ * rows, with as many CTAs per slab as still fit the GPU at once).  Results do not depend on it. */
+dynts_status_t dynts_cache_set_evict_launch(dynts_cache_t* c, int split);
+
 /* Bookkeeping of the most recent eviction, read back from the device (synchronises the stream):
  * over the slabs that shrank, the rows whose scores were scanned and the rows that changed place
  * during compaction (rows behind the first evicted one).  For traffic accounting. */

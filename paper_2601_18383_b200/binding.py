@@ -85,6 +85,7 @@ _sigs = {
     "dynts_poll_error": (C.c_int, [_P]),
     "dynts_synchronize": (C.c_int, [_P]),
     "dynts_cache_set_launch": (C.c_int, [_P, C.c_int, C.c_int]),
+    "dynts_cache_set_evict_launch": (C.c_int, [_P, C.c_int]),
     "dynts_cache_launch_count": (C.c_longlong, [_P]),
     "dynts_cache_set_score_source": (C.c_int, [_P, C.c_int]),
     "dynts_cache_set_kv_scale": (C.c_int, [_P, C.c_float, C.c_float]),
@@ -258,6 +259,10 @@ def dynts_cache_set_launch(c, cluster=0, variant=0):
     return _check(lib.dynts_cache_set_launch(c, cluster, variant))
 
 
+def dynts_cache_set_evict_launch(c, split=0):
+    return _check(lib.dynts_cache_set_evict_launch(c, split))
+
+
 def dynts_cache_set_score_source(c, source):
     return _check(lib.dynts_cache_set_score_source(c, source))
 
@@ -376,6 +381,9 @@ class Cache:
 
     def set_launch(self, cluster=0, variant=0):
         return dynts_cache_set_launch(self.handle, cluster, variant)
+
+    def set_evict_launch(self, split=0):
+        return dynts_cache_set_evict_launch(self.handle, split)
 
     def set_stream(self, stream):
         return dynts_cache_set_stream(self.handle, stream.cuda_stream if hasattr(stream, "cuda_stream") else stream)

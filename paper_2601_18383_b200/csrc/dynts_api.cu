@@ -132,6 +132,7 @@ struct dynts_cache {
   std::vector<int> seq_budget, len_h, tot_h, pinned_h, target_h, active_h;  // host mirrors of the per-sequence state
   int layer_cursor = 0;      // next layer expected by dynts_decode_attn_layer
   int cluster = 0, variant = 0;
+  int evict_split = 0;       // CTAs per slab of the eviction: 0 automatic, 1/2/4/8 forced, -1 the one-CTA kernel with shared-memory keys
   int score_source = 0;      // 0: attention mass accumulates (Eq. 6); 1: the caller supplies scores (Eq. 7)
   int parity = 0;            // half of the logit scratch the next decode step writes
   bool pending = false;      // the last streaming launches recorded score passes that are not applied yet
@@ -198,9 +199,6 @@ dynts_status_t make_slab_maps(dynts_cache* c) {
   CUresult r1 = encode(&c->map_KV, mtype, 3, c->K(), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r1 != CUDA_SUCCESS) return fail(DYNTS_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r1);
-  int dev = 0;
-  CUDA_TRY(cudaGetDevice(&dev));
-  CUDA_TRY(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev));
   c->have_maps = true;
   return DYNTS_OK;
 }
@@ -235,6 +233,11 @@ dynts_status_t materialise(dynts_cache* c) {
     CUDA_TRY(cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->err_dev), c->err_host, 0));
   }
   CUDA_TRY(cudaMemsetAsync(c->base, 0, c->lay.total, c->stream));
+  {
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    CUDA_TRY(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev));
+  }
   c->have_maps = false;
   if (stream_capable(&c->cfg)) {
     dynts_status_t ms = make_slab_maps(c);
@@ -636,28 +639,65 @@ dynts_status_t do_evict(dynts_cache* c, const int* targets /* host [Nb], validat
     p.key = c->agg();
   }
   if (fused_path) {
-    // one launch: selection and compaction of a slab by the same CTA
+    // one launch: selection and compaction of a slab by the same CTA, or by a cluster of CTAs that
+    // share the slab's columns
     if (c->pending) {
       p.pend = c->pend();
       p.logit_prev = c->logit(c->parity ^ 1);
       p.G = c->G;
       c->pending = false;
     }
-    const size_t smem = (size_t)c->cap * (global ? 20 : 16);
-    dynts_status_t st = ensure_smem_attr(dynts::evict_fused_kernel, smem, &c->attr_fused, false);
-    if (st != DYNTS_OK) return st;
     cudaLaunchConfig_t fc;
     memset(&fc, 0, sizeof(fc));
-    cudaLaunchAttribute fattr[1];
+    cudaLaunchAttribute fattr[2];
     fattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see griddepcontrol.wait in the kernel
     fattr[0].val.programmaticStreamSerializationAllowed = 1;
     fc.attrs = fattr;
     fc.numAttrs = 1;
     fc.stream = c->stream;
-    fc.gridDim = dim3((unsigned)c->slabs(), 1, 1);
-    fc.blockDim = dim3(dynts::kFusedThreads, 1, 1);
-    fc.dynamicSmemBytes = smem;
-    CUDA_TRY(cudaLaunchKernelEx(&fc, dynts::evict_fused_kernel, p, c->ticket() + 1));
+    const int pieces2 = 2 * c->cfg.head_dim * c->kv_elt / 16;  // 16-byte pieces of a K row followed by a V row
+    // Slabs of up to 2304 rows: the kernel that keeps a thread's rows in registers (its short
+    // selection phase matters there); longer slabs, whose events are dominated by the rows that
+    // move, measured faster on the one-CTA kernel with shared-memory keys.
+    if (c->cap <= 17 * dynts::kSplitThreads && (c->evict_split > 0 || (c->evict_split == 0 && c->cap <= 9 * dynts::kSplitThreads))) {
+      // CTAs per slab: as many as still leave every CTA of the grid resident at once (a second round
+      // of CTAs would start only when the first ends), in shares of at least 64 contiguous bytes
+      const int tier = c->cap <= 5 * dynts::kSplitThreads ? 5 : c->cap <= 9 * dynts::kSplitThreads ? 9 : c->cap <= 13 * dynts::kSplitThreads ? 13 : 17;
+      const long long resident = (long long)(c->sm_count > 0 ? c->sm_count : 148) * dynts::split_ctas_per_sm(tier);
+      int S = 1;
+      if (c->evict_split > 0) {
+        S = c->evict_split;
+      } else {
+        while (S < 8 && (long long)c->slabs() * (2 * S) <= resident) S *= 2;
+      }
+      while (S > 1 && (pieces2 % S != 0 || pieces2 / S < 4)) S /= 2;
+      fattr[1].id = cudaLaunchAttributeClusterDimension;
+      fattr[1].val.clusterDim.x = (unsigned)S;
+      fattr[1].val.clusterDim.y = 1;
+      fattr[1].val.clusterDim.z = 1;
+      fc.numAttrs = 2;
+      fc.gridDim = dim3((unsigned)(c->slabs() * S), 1, 1);
+      fc.blockDim = dim3(dynts::kSplitThreads, 1, 1);
+      fc.dynamicSmemBytes = (size_t)c->cap * 4;
+      cudaError_t e;
+#define DYNTS_SPLIT_LAUNCH(RPT)                                                                                   \
+  (global ? cudaLaunchKernelEx(&fc, dynts::evict_split_kernel<RPT, true>, p, c->ticket() + 1)                     \
+          : cudaLaunchKernelEx(&fc, dynts::evict_split_kernel<RPT, false>, p, c->ticket() + 1))
+      if (tier == 5) e = DYNTS_SPLIT_LAUNCH(5);
+      else if (tier == 9) e = DYNTS_SPLIT_LAUNCH(9);
+      else if (tier == 13) e = DYNTS_SPLIT_LAUNCH(13);
+      else e = DYNTS_SPLIT_LAUNCH(17);
+#undef DYNTS_SPLIT_LAUNCH
+      if (e != cudaSuccess) return fail(DYNTS_ERR_CUDA, "eviction launch (%d CTAs per slab): %s", S, cudaGetErrorString(e));
+    } else {
+      const size_t smem = (size_t)c->cap * (global ? 20 : 16);
+      dynts_status_t st = ensure_smem_attr(dynts::evict_fused_kernel, smem, &c->attr_fused, false);
+      if (st != DYNTS_OK) return st;
+      fc.gridDim = dim3((unsigned)c->slabs(), 1, 1);
+      fc.blockDim = dim3(dynts::kFusedThreads, 1, 1);
+      fc.dynamicSmemBytes = smem;
+      CUDA_TRY(cudaLaunchKernelEx(&fc, dynts::evict_fused_kernel, p, c->ticket() + 1));
+    }
     c->launches += 1;
   } else {
     const size_t smem = (size_t)c->cap * 12;
@@ -1064,6 +1104,14 @@ dynts_status_t dynts_cache_set_launch(dynts_cache_t* c, int cluster, int variant
   if (variant < 0 || variant > 3) return fail(DYNTS_ERR_INVALID_ARG, "variant must be 0, 1, 2 or 3");
   c->cluster = cluster;
   c->variant = variant;
+  return DYNTS_OK;
+}
+
+dynts_status_t dynts_cache_set_evict_launch(dynts_cache_t* c, int split) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (!(split == -1 || split == 0 || split == 1 || split == 2 || split == 4 || split == 8))
+    return fail(DYNTS_ERR_INVALID_ARG, "split must be -1, 0, 1, 2, 4 or 8");
+  c->evict_split = split;
   return DYNTS_OK;
 }
 

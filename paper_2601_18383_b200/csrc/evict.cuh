@@ -457,6 +457,419 @@ __global__ void __launch_bounds__(kFusedThreads) evict_fused_kernel(const EvictP
 }
 
 // ---------------------------------------------------------------------------------------------
+// Split eviction (slabs of up to 256 * RPT rows): a cluster of S CTAs per slab.  Every CTA of the
+// cluster takes the slab's selection decision for itself and then moves its own share of the
+// columns of the K and V rows (16-byte pieces [rank * 2P / S, (rank + 1) * 2P / S) of the 2P pieces
+// of a K row followed by a V row).  Column shares are disjoint, so the CTAs of a slab never wait
+// for one another while rows move, and a slab whose first evicted row lies far from its end no
+// longer keeps one CTA busy long after the rest of the grid has finished.
+//
+// Everything a thread knows about its rows lives in registers: row i * 256 + tid is the thread's
+// row i, with its score, its compensation term and (where the selection ranks by keys shared
+// across the sequence) its key.  A score pass that the last decode launch left recorded is applied
+// right there -- new score = old score + the row's normalised mass, from the logit scratch -- so
+// the pass costs no round trip through memory before the scores can be ranked.
+//
+// Selection, integer-only as above:
+//   - the candidates' smallest and largest key give a shift s with (key - smallest) >> s < 2048;
+//     that monotone map spreads the rows over the 2048 bins of one histogram according to their
+//     values, so a bin rarely holds more than a few rows.  Walking the bins from the top finds the
+//     bin of the k-th largest key; the search ends there if the bin must be taken whole ("key >=
+//     the bin's lower bound" decides), else it repeats inside the bin with s - 11 (at most three
+//     rounds resolve all 32 bits);
+//   - only if the threshold key itself is shared by more rows than may survive do ranks among the
+//     ties (by index, from warp ballots and one scan of the per-warp counts) come into play;
+//   - destinations are the exclusive prefix count of the survivor flags in index order.
+// Score and compensation are written to their destinations from the registers, positions are
+// gathered; each of the three arrays by one CTA of the cluster.  One cluster barrier separates
+// every CTA's read of the old scores from their being overwritten.
+// ---------------------------------------------------------------------------------------------
+constexpr int kSplitThreads = 256;
+constexpr int kSplitBins = 2048;
+// 16-byte loads in flight per thread while rows move, and CTAs per SM: short slabs leave room for
+// four CTAs of 64 registers; longer ones hold more rows per thread and run as two CTAs of 128.
+__host__ __device__ constexpr int split_unroll(int rpt) { return rpt <= 5 ? 8 : 16; }
+__host__ __device__ constexpr int split_ctas_per_sm(int rpt) { return rpt <= 5 ? 4 : 2; }
+
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_cta_count() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+// Per-warp counts of a per-row flag (bit i of `flags` belongs to row i * 256 + tid): cnt[i * 8 + warp].
+template <int RPT>
+__device__ __forceinline__ void rows_count(uint32_t flags, int* cnt, int warp, int lane) {
+#pragma unroll
+  for (int i = 0; i < RPT; ++i) {
+    const unsigned bal = __ballot_sync(0xffffffffu, (flags >> i) & 1u);
+    if (lane == 0) cnt[i * 8 + warp] = __popc(bal);
+  }
+}
+// One warp turns cnt[0 .. RPT * 8) into its exclusive prefix sums (index order of the rows) and
+// leaves the total in cnt[RPT * 8].
+template <int RPT>
+__device__ __forceinline__ void rows_scan(int* cnt, int lane) {
+  constexpr int N = RPT * 8, E = (N + 31) / 32;
+  int v[E], sum = 0;
+#pragma unroll
+  for (int e = 0; e < E; ++e) {
+    const int idx = lane * E + e;
+    v[e] = idx < N ? cnt[idx] : 0;
+    sum += v[e];
+  }
+  int incl = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  int run = incl - sum;
+#pragma unroll
+  for (int e = 0; e < E; ++e) {
+    const int idx = lane * E + e;
+    if (idx < N) cnt[idx] = run;
+    run += v[e];
+  }
+  if (lane == 31) cnt[N] = incl;
+}
+
+// The recorded score pass of a slab (see DecodeParams::defer) on the rows this thread holds: the
+// same arithmetic, in the same order, as score_pass_vec.  The logits and the record's maxima and
+// normalisers are requested before anyone knows whether the record is valid (the addresses always
+// are), so that they travel together with the scores; `valid` decides whether they are used.
+template <int RPT, int GG>
+__device__ __forceinline__ void recorded_pass_rows(float (&sc)[RPT], float (&cc)[RPT], const float* __restrict__ lg, int cap,
+                                                   const int* rec, bool valid, int n, int n_old, int tid) {
+  float M[GG], f[GG];
+#pragma unroll
+  for (int g = 0; g < GG; ++g) {
+    M[g] = __ldcg(reinterpret_cast<const float*>(rec) + 2 + g);
+    f[g] = __ldcg(reinterpret_cast<const float*>(rec) + 10 + g);
+  }
+#pragma unroll
+  for (int i = 0; i < RPT; ++i) {
+    const int j = i * kSplitThreads + tid;
+    float e[GG];
+#pragma unroll
+    for (int g = 0; g < GG; ++g) e[g] = j < cap ? __ldcg(lg + (size_t)g * cap + j) : 0.f;
+    float dl = 0.f;
+#pragma unroll
+    for (int g = 0; g < GG; ++g) dl += fast_exp2(e[g] - M[g]) * f[g];
+    if (valid && j < n) {
+      if (j == n_old) sc[i] = cc[i] = 0.f;  // the appended row starts from zero
+      kahan_add(sc[i], cc[i], dl);
+    }
+  }
+}
+
+// SHARED_KEYS: the selection ranks by p.key (one key per token, shared by all slabs of a sequence)
+// instead of the slab's own scores.
+template <int RPT, bool SHARED_KEYS>
+__global__ void __launch_bounds__(kSplitThreads, split_ctas_per_sm(RPT)) evict_split_kernel(const EvictParams p, unsigned int* ticket) {
+  constexpr int kSplitUnroll = split_unroll(RPT);
+  const uint32_t S = cluster_cta_count(), rank = cluster_cta_rank();
+  const int slab = (int)(blockIdx.x / S);
+  const int b = (slab / p.Hkv) % p.Nb;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  extern __shared__ __align__(16) int split_src[];  // [cap] gather list: split_src[dst] = surviving row
+  __shared__ __align__(16) unsigned int hist[kSplitBins];
+  __shared__ int s_cnt_eq[RPT * 8 + 1], s_cnt_keep[RPT * 8 + 1];
+  __shared__ int s_wtot[kSplitThreads / 32];
+  __shared__ uint32_t s_wmin[kSplitThreads / 32], s_wmax[kSplitThreads / 32];
+  __shared__ uint32_t s_base;
+  __shared__ int s_krem, s_bin_cnt;
+  __shared__ int s_wfirst[kSplitThreads / 32];
+
+  // nothing here touches global memory: it may overlap the tail of the kernel before this one
+#pragma unroll
+  for (int i = 0; i < kSplitBins / 4 / kSplitThreads; ++i)
+    reinterpret_cast<uint4*>(hist)[i * kSplitThreads + tid] = make_uint4(0u, 0u, 0u, 0u);
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // launched with programmatic stream serialisation
+
+  // One round trip: the lengths, the record of a score pass the last decode launch may have left,
+  // and this thread's rows (score, compensation, position; the logits of the recorded pass).
+  float* score = p.score + (size_t)slab * p.cap;
+  float* comp = p.comp ? p.comp + (size_t)slab * p.cap : nullptr;
+  int* pos = p.pos + (size_t)slab * p.cap;
+  const bool have_rec = !SHARED_KEYS && p.pend != nullptr;
+  const int* rec = have_rec ? p.pend + (size_t)slab * kStPendWords : nullptr;
+  const int n = p.len[b];
+  const int tgt = p.target[b];
+  const int M = p.pinned[b];
+  const int rn = have_rec ? rec[0] : 0, rn_old = have_rec ? rec[1] : 0;
+  // Owners of the per-row arrays within the cluster.
+  const bool own_score = rank == 0, own_comp = rank == (2u % S), own_pos = rank == (1u % S);
+  float sc[RPT], cc[RPT];
+  int posv[RPT];
+#pragma unroll
+  for (int i = 0; i < RPT; ++i) {
+    const int j = i * kSplitThreads + tid;
+    sc[i] = j < p.cap ? score[j] : 0.f;
+    cc[i] = (j < p.cap && comp) ? comp[j] : 0.f;
+    posv[i] = (j < p.cap && own_pos) ? pos[j] : 0;
+  }
+  int* hdr = p.hdr + (size_t)slab * 4;
+  const bool fits = n <= p.cap && n <= RPT * kSplitThreads;
+  if (!fits && tid == 0) atomicOr(p.err, kErrEvictSmem);  // (the host chooses RPT from the capacity)
+  const bool evicting = fits && n > tgt;                        // uniform over the cluster
+  bool applied = false;
+  if constexpr (!SHARED_KEYS) {
+    if (have_rec) {
+      applied = fits && rn > 0 && rn == n;                      // uniform over the cluster
+      DYNTS_DISPATCH_GROUP(p.G, (recorded_pass_rows<RPT, GG>(sc, cc, p.logit_prev + (size_t)slab * p.G * p.cap, p.cap, rec, applied, n,
+                                                            rn_old, tid)));
+      if (rn > 0 && !applied && tid == 0) atomicOr(p.err, kErrLenOverflow);  // a record that does not match the slab: the host mirror prevents it
+    }
+  }
+  __syncthreads();  // hist, s_first
+
+  if (evicting) {
+    const int lo = M, hi = n - p.window;  // selection window [lo, hi)
+    const int k = tgt - M - p.window;     // survivors wanted from it (host guarantees 0 <= k < hi - lo)
+
+    // keys of the selection window
+    uint32_t key[RPT];
+    uint32_t candm = 0u;
+    uint32_t tmin = 0xffffffffu, tmax = 0u;
+#pragma unroll
+    for (int i = 0; i < RPT; ++i) {
+      const int j = i * kSplitThreads + tid;
+      const bool cand = j >= lo && j < hi;
+      uint32_t bits = __float_as_uint(sc[i]);
+      if constexpr (SHARED_KEYS) bits = cand ? __float_as_uint(p.key[(size_t)b * p.cap + j]) : 0u;
+      key[i] = cand ? order_key(bits) : 0u;
+      candm |= (cand ? 1u : 0u) << i;
+      if (cand) {
+        tmin = min(tmin, key[i]);
+        tmax = max(tmax, key[i]);
+      }
+    }
+    cluster_arrive();  // this CTA has read the old scores (paired with the wait before any of them is overwritten)
+
+    uint32_t T = 0u;
+    int take_eq = 0;
+    bool whole_bin = true;  // every row with key >= T survives (no tie is split)
+    if (k > 0) {
+      tmin = __reduce_min_sync(0xffffffffu, tmin);
+      tmax = __reduce_max_sync(0xffffffffu, tmax);
+      if (lane == 0) {
+        s_wmin[warp] = tmin;
+        s_wmax[warp] = tmax;
+      }
+      __syncthreads();
+      uint32_t kmin = s_wmin[0], kmax = s_wmax[0];
+#pragma unroll
+      for (int w = 1; w < kSplitThreads / 32; ++w) {
+        kmin = min(kmin, s_wmin[w]);
+        kmax = max(kmax, s_wmax[w]);
+      }
+      // keys in [base, base + width): bin = (key - base) >> s, with width >> s <= 2048
+      uint32_t base = kmin;
+      int s = max(0, 32 - __clz(kmax - kmin) - 11);  // (kmax == kmin: clz = 32, s = 0, every row in bin 0)
+      uint32_t width_m1 = kmax - kmin;                // width - 1 of the current interval
+      int krem = k;
+      whole_bin = false;
+      for (int round = 0; round < 3; ++round) {  // s: <= 21, <= 10, 0
+#pragma unroll
+        for (int i = 0; i < RPT; ++i) {
+          const uint32_t off = key[i] - base;
+          if (((candm >> i) & 1u) && key[i] >= base && off <= width_m1) atomicAdd(&hist[off >> s], 1u);
+        }
+        __syncthreads();
+        // thread t owns bins 2040 - 8t .. 2047 - 8t; walking t upwards walks the bins downwards
+        const int hb = kSplitBins - 8 - 8 * tid;
+        unsigned int hv[8];
+        {
+          const uint4 h0 = reinterpret_cast<const uint4*>(hist)[hb >> 2], h1 = reinterpret_cast<const uint4*>(hist)[(hb >> 2) + 1];
+          hv[0] = h0.x; hv[1] = h0.y; hv[2] = h0.z; hv[3] = h0.w;
+          hv[4] = h1.x; hv[5] = h1.y; hv[6] = h1.z; hv[7] = h1.w;
+          reinterpret_cast<uint4*>(hist)[hb >> 2] = make_uint4(0u, 0u, 0u, 0u);  // clear for the next round
+          reinterpret_cast<uint4*>(hist)[(hb >> 2) + 1] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        const int mine = (int)(hv[0] + hv[1] + hv[2] + hv[3] + hv[4] + hv[5] + hv[6] + hv[7]);
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += t;
+        }
+        if (lane == 31) s_wtot[warp] = incl;
+        __syncthreads();
+#pragma unroll
+        for (int w = 0; w < kSplitThreads / 32; ++w)
+          if (w < warp) incl += s_wtot[w];
+        const int excl = incl - mine;
+        if (excl < krem && krem <= incl) {  // exactly one thread: its bins hold the krem-th largest remaining key
+          int above = excl;
+#pragma unroll
+          for (int i = 7; i >= 0; --i) {
+            const int c = (int)hv[i];
+            if (above < krem && krem <= above + c) {
+              s_base = base + ((uint32_t)(hb + i) << s);
+              s_krem = krem - above;
+              s_bin_cnt = c;
+            }
+            above += c;
+          }
+        }
+        __syncthreads();
+        base = s_base;
+        krem = s_krem;
+        T = base;
+        take_eq = krem;
+        if (krem == s_bin_cnt) {  // the whole bin survives: nothing finer needs to be known
+          whole_bin = true;
+          break;
+        }
+        if (s == 0) break;        // the bin is one key value, shared by more rows than may survive
+        width_m1 = (1u << s) - 1u;
+        s = max(0, s - 11);
+      }
+    }
+
+    // survivor flags
+    uint32_t keepm = 0u;
+    if (whole_bin) {
+#pragma unroll
+      for (int i = 0; i < RPT; ++i) {
+        const int j = i * kSplitThreads + tid;
+        const bool cand = (candm >> i) & 1u;
+        const bool keep = cand ? (k > 0 && key[i] >= T) : (j < n);
+        keepm |= (keep ? 1u : 0u) << i;
+      }
+    } else {
+      // more rows share the threshold key than may survive: the lowest-indexed take_eq of them do
+      uint32_t eqm = 0u;
+#pragma unroll
+      for (int i = 0; i < RPT; ++i) eqm |= ((((candm >> i) & 1u) && key[i] == T) ? 1u : 0u) << i;
+      rows_count<RPT>(eqm, s_cnt_eq, warp, lane);
+      __syncthreads();
+      if (warp == 0) rows_scan<RPT>(s_cnt_eq, lane);
+      __syncthreads();
+#pragma unroll
+      for (int i = 0; i < RPT; ++i) {
+        const int j = i * kSplitThreads + tid;
+        const bool cand = (candm >> i) & 1u;
+        const bool eq = (eqm >> i) & 1u;
+        const unsigned bal = __ballot_sync(0xffffffffu, eq);
+        const int eq_rank = s_cnt_eq[i * 8 + warp] + __popc(bal & ((1u << lane) - 1u));
+        const bool keep = cand ? (key[i] > T || (eq && eq_rank < take_eq)) : (j < n);
+        keepm |= (keep ? 1u : 0u) << i;
+      }
+    }
+    // destinations and the gather list
+    rows_count<RPT>(keepm, s_cnt_keep, warp, lane);
+    __syncthreads();
+    if (warp == 0) rows_scan<RPT>(s_cnt_keep, lane);
+    __syncthreads();
+    int dstv[RPT];  // destination of this thread's surviving rows
+    int wfirst = 0x7fffffff;  // first row of this warp's rows that leaves (the same value in every lane)
+#pragma unroll
+    for (int i = 0; i < RPT; ++i) {
+      const int j = i * kSplitThreads + tid;
+      const bool keep = (keepm >> i) & 1u;
+      const unsigned bal = __ballot_sync(0xffffffffu, keep);
+      dstv[i] = s_cnt_keep[i * 8 + warp] + __popc(bal & ((1u << lane) - 1u));
+      if (keep) split_src[dstv[i]] = j;
+      const unsigned gone = __ballot_sync(0xffffffffu, !keep && j < n);
+      if (gone != 0u) wfirst = min(wfirst, i * kSplitThreads + warp * 32 + __ffs(gone) - 1);
+    }
+    if (lane == 0) s_wfirst[warp] = wfirst;
+    __syncthreads();
+    int first = s_wfirst[0];  // rows below `first` stay where they are
+#pragma unroll
+    for (int w = 1; w < kSplitThreads / 32; ++w) first = min(first, s_wfirst[w]);
+    const int kept = s_cnt_keep[RPT * 8];  // == tgt
+    if (rank == 0 && tid == 0) {
+      hdr[0] = first;
+      hdr[1] = kept;
+      hdr[2] = n;
+    }
+    cluster_wait();  // every CTA of the cluster has read the old scores: they may be overwritten now
+    if (applied && rank == S - 1 && (p.cap & 31) == 0) {
+      // ... and the logits of the recorded pass, which are dead now: drop their L2 lines (32 rows of one
+      // head each) instead of letting them be written back
+      const float* lg = p.logit_prev + (size_t)slab * p.G * p.cap;
+      const int lines = (n + 31) >> 5;
+      for (int x = tid; x < p.G * lines; x += kSplitThreads) {
+        const int g = x / lines, ln = x - g * lines;
+        asm volatile("discard.global.L2 [%0], 128;" ::"l"(lg + (size_t)g * p.cap + 32 * ln) : "memory");
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < RPT; ++i) {
+      const bool keep = (keepm >> i) & 1u;
+      const bool moved = keep && dstv[i] >= first;
+      if (own_score && keep && (moved || applied)) score[dstv[i]] = sc[i];
+      if (own_comp && comp && keep && (moved || applied)) comp[dstv[i]] = cc[i];
+      if (own_pos && moved) pos[dstv[i]] = posv[i];
+    }
+
+    // K and V rows: this CTA's share of the 16-byte pieces of (K row | V row).  Ascending blocks; all
+    // sources of a block are in registers before any destination of it is written (src >= dst).
+    const int row_bytes = p.d * p.elt_bytes;
+    const int P = row_bytes >> 4;               // pieces per row and tensor
+    const int ppc = (2 * P) / (int)S;            // pieces per CTA and row (the host makes S divide 2P)
+    const int rpp = kSplitThreads / ppc;         // rows per pass
+    const bool active = tid < rpp * ppc;
+    const int r_in = tid / ppc;
+    const int q = (int)rank * ppc + (tid - r_in * ppc);
+    const int isv = q >= P ? 1 : 0;
+    char* kvbase = reinterpret_cast<char*>(isv ? p.V : p.K) + (size_t)slab * p.cap * row_bytes + (size_t)(q - isv * P) * 16;
+    for (int c0 = first; c0 < kept; c0 += rpp * kSplitUnroll) {
+      uint4 buf[kSplitUnroll];
+#pragma unroll
+      for (int uu = 0; uu < kSplitUnroll; ++uu) {
+        const int dd = c0 + uu * rpp + r_in;
+        if (active && dd < kept) buf[uu] = *reinterpret_cast<const uint4*>(kvbase + (size_t)split_src[dd] * row_bytes);
+      }
+      __syncthreads();  // every source row of the block is in registers before any row is overwritten
+#pragma unroll
+      for (int uu = 0; uu < kSplitUnroll; ++uu) {
+        const int dd = c0 + uu * rpp + r_in;
+        if (active && dd < kept) *reinterpret_cast<uint4*>(kvbase + (size_t)dd * row_bytes) = buf[uu];
+      }
+    }
+  } else {
+    if (rank == 0 && tid == 0) {
+      hdr[0] = n;
+      hdr[1] = n;
+      hdr[2] = n;
+    }
+    if (applied) {  // no row leaves, but the recorded pass has changed the scores (this launch's CTAs are the only readers)
+#pragma unroll
+      for (int i = 0; i < RPT; ++i) {
+        const int j = i * kSplitThreads + tid;
+        if (j < n && own_score) score[j] = sc[i];
+        if (j < n && own_comp && comp) comp[j] = cc[i];
+      }
+    }
+  }
+  if (applied && rank == 0 && tid == 0) p.pend[(size_t)slab * kStPendWords] = 0;
+
+  // The last CTA to finish publishes the new lengths.
+  __syncthreads();
+  if (tid == 0) {
+    __threadfence();
+    const unsigned int t = atomicAdd(ticket, 1u);
+    if (t == gridDim.x - 1) {
+      *ticket = 0u;
+      for (int bb = 0; bb < p.Nb; ++bb) p.len[bb] = min(p.len[bb], p.target[bb]);
+      __threadfence();
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // One importance score per token, aggregated across all layers and KV heads (Appendix B.1):
 // agg[b][j] = sum over (layer, head) of score[layer][b][head][j].  The fp32 slab scores are added
 // in double precision and the sum is rounded to fp32 once, so the key a ranking is decided by is

@@ -18,6 +18,11 @@ def _check_line(line, n_gpus):
     assert d["value"] > 0 and d["config"]["workload"] == "c1_tiny_fp32" and d["vs_baseline"] is None
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1 and d["cpu_baseline"]["sample"]
     assert d["e2e"] == {"value": d["value"], "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+    # the same description of the workload as the main arm prints (bench.workload_config)
+    assert set(d["config"]) == {"workload", "layers", "batch", "q_heads", "kv_heads", "head_dim", "budget", "window",
+                                "evict_interval", "prompt_pinned", "dist", "score_source", "selection", "kv_dtype",
+                                "kv_bytes", "l2_policy", "replicas"}
+    assert d["config"]["replicas"] == n_gpus
 
 
 def test_reference_arm_single_process():

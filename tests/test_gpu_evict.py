@@ -59,6 +59,29 @@ def test_patterns_bit_exact(pattern, dtype, d):
     gpu.close()
 
 
+@pytest.mark.parametrize("split", [-1, 1, 2, 4, 8])
+@pytest.mark.parametrize("pattern", ["random", "all_equal", "few_levels_many_ties", "negative_and_zero", "first_candidate_lowest",
+                                     "block_before_window_lowest"])
+@pytest.mark.parametrize("dtype,d,rows,budget", [("bf16", 128, 1237, 700), ("fp32", 96, 1000, 300), ("bf16", 128, 2112, 2048),
+                                                 ("bf16", 128, 3136, 3072), ("bf16", 128, 4224, 4096), ("bf16", 128, 4352, 1000)])
+def test_ctas_per_slab_and_row_count_tiers(split, pattern, dtype, d, rows, budget):
+    """The eviction kernel's launch shapes: one CTA per slab with shared-memory keys (-1), or 1, 2,
+    4, 8 CTAs per slab that each decide for themselves and move a share of the row bytes; row
+    counts in each of the kernel's register tiers (up to 1280, 2304, 3328, 4352 rows)."""
+    cfg = W.get_config("c2_llama8b").scaled(layers=2, batch=2, kv_heads=2, q_heads=8, head_dim=d, dtype=dtype,
+                                             prompt=24, budget=budget, window=32, evict_interval=rows - budget)
+    gpu = _filled(cfg, rows, cfg.prompt, seed=1)
+    gpu.set_evict_launch(split)
+    _set_scores(gpu, cfg, rows, cfg.prompt, PATTERNS[pattern], seed=2)
+    kept = H.check_evict_bit_exact(gpu, cfg, cfg.budget)
+    assert all(len(k) == cfg.budget for k in kept.values()) and gpu.len(1) == cfg.budget
+    rows_scanned, rows_moved = gpu.evict_stats()
+    assert rows_scanned == rows * 8
+    assert rows_moved == sum(cfg.budget - int(np.flatnonzero(k != np.arange(len(k)))[0]) if (k != np.arange(len(k))).any() else 0
+                             for k in kept.values())
+    gpu.close()
+
+
 @pytest.mark.parametrize("target", [56, 57, 100, 699, 1236, 1237, 5000])
 def test_targets_from_window_only_to_no_op(target):
     """k = 0 (question + local window only) ... target >= n (nothing moves)."""
