@@ -203,6 +203,13 @@ dynts_status_t dynts_evict_ex(dynts_cache_t* c, const int* seq_targets);
 dynts_status_t dynts_evict_noalloc(void* K, void* V, int* pos, float* score, int n_slabs, int head_dim, int dtype,
                                    int capacity, int n_rows, int n_pinned, int window, int target, void* stream);
 
+/* No counterpart in the paper.  The kernels of dynts_evict_noalloc re-check the lengths they were
+ * given and, if they disagree (memory the caller changed while the call was in flight), record it
+ * in a status word inside the built-in scratch and move nothing for that slab.  This waits for
+ * `stream` and returns DYNTS_ERR_DEVICE if the most recent call on the current device recorded
+ * anything, else DYNTS_OK.  Allocates nothing. */
+dynts_status_t dynts_evict_noalloc_status(void* stream);
+
 /* Scales of a DYNTS_BF16_KV8 cache (default 1, 1).  Host floats; k_scale, v_scale > 0 and finite.
  * Allowed only while no sequence holds rows (DYNTS_ERR_STATE otherwise): stored codes are not
  * re-encoded.  Choose scale ~ max|x| / 448 of the tensor to use the format's range. */
@@ -293,6 +300,18 @@ dynts_status_t dynts_synchronize(dynts_cache_t* c);
  * 2 and 3 need bf16, d = 128, G <= 8.  cluster: for variants 1 and 2 the cluster size (1, 2, 4,
  * 8 or 16; 0 => automatic); for variant 3 the CTAs per SM (1 or 2; anything else => 2). */
 dynts_status_t dynts_cache_set_launch(dynts_cache_t* c, int cluster, int variant);
+
+/* Device-side waits are bounded: a thread that waits for a tile or a hand-over inside the streaming
+ * decode kernel polls at most `polls` times (default 2^22, seconds at worst); when a wait runs
+ * out the CTA raises the timeout bit of the status word, every later wait of that CTA returns at
+ * once, the kernel ends, and dynts_poll_error reports DYNTS_ERR_DEVICE (that step's results are
+ * void; the context stays usable).  polls >= 64. */
+dynts_status_t dynts_cache_set_wait_limit(dynts_cache_t* c, unsigned int polls);
+
+/* For tests of that path only: the next streaming decode launch of this cache omits one tile load
+ * (the item-th 32-row chunk of the first CTA's piece), so that the wait for it runs out.  The
+ * step's results, and the scores of the slabs that CTA covers, are void afterwards. */
+dynts_status_t dynts_debug_drop_tile_load(dynts_cache_t* c, int item);
 
 /* Launch configuration of the eviction kernel, for tuning.  split: 1, 2, 4 or 8 => the kernel that
  * keeps every thread's rows in registers, with that many CTAs sharing one slab (each takes the

@@ -76,6 +76,7 @@ _sigs = {
     "dynts_aggregate_scores": (C.c_int, [_P, _P]),
     "dynts_evict_ex": (C.c_int, [_P, C.POINTER(C.c_int)]),
     "dynts_evict_noalloc": (C.c_int, [_P, _P, _P, _P] + [C.c_int] * 8 + [_P]),
+    "dynts_evict_noalloc_status": (C.c_int, [_P]),
     "dynts_seq_reset": (C.c_int, [_P, C.c_int]),
     "dynts_cache_len": (C.c_int, [_P, C.c_int]),
     "dynts_cache_capacity": (C.c_int, [_P]),
@@ -86,6 +87,8 @@ _sigs = {
     "dynts_synchronize": (C.c_int, [_P]),
     "dynts_cache_set_launch": (C.c_int, [_P, C.c_int, C.c_int]),
     "dynts_cache_set_evict_launch": (C.c_int, [_P, C.c_int]),
+    "dynts_cache_set_wait_limit": (C.c_int, [_P, C.c_uint]),
+    "dynts_debug_drop_tile_load": (C.c_int, [_P, C.c_int]),
     "dynts_cache_launch_count": (C.c_longlong, [_P]),
     "dynts_cache_set_score_source": (C.c_int, [_P, C.c_int]),
     "dynts_cache_set_kv_scale": (C.c_int, [_P, C.c_float, C.c_float]),
@@ -221,6 +224,11 @@ def dynts_evict_noalloc(K, V, pos, score, n_slabs, head_dim, dtype, capacity, n_
                                           capacity, n_rows, n_pinned, window, target, stream))
 
 
+def dynts_evict_noalloc_status(stream=None):
+    """Waits for the stream; raises if the last allocation-free eviction recorded a device-side check."""
+    return _check(lib.dynts_evict_noalloc_status(stream))
+
+
 def dynts_seq_reset(c, seq):
     return _check(lib.dynts_seq_reset(c, seq))
 
@@ -257,6 +265,14 @@ def dynts_synchronize(c):
 
 def dynts_cache_set_launch(c, cluster=0, variant=0):
     return _check(lib.dynts_cache_set_launch(c, cluster, variant))
+
+
+def dynts_cache_set_wait_limit(c, polls):
+    return _check(lib.dynts_cache_set_wait_limit(c, polls))
+
+
+def dynts_debug_drop_tile_load(c, item):
+    return _check(lib.dynts_debug_drop_tile_load(c, item))
 
 
 def dynts_cache_set_evict_launch(c, split=0):
@@ -381,6 +397,12 @@ class Cache:
 
     def set_launch(self, cluster=0, variant=0):
         return dynts_cache_set_launch(self.handle, cluster, variant)
+
+    def set_wait_limit(self, polls):
+        return dynts_cache_set_wait_limit(self.handle, polls)
+
+    def debug_drop_tile_load(self, item):
+        return dynts_debug_drop_tile_load(self.handle, item)
 
     def set_evict_launch(self, split=0):
         return dynts_cache_set_evict_launch(self.handle, split)

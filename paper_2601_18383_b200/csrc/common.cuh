@@ -57,6 +57,8 @@ struct DecodeParams {
   int defer;
   float* logit_prev;
   int* pend;          // [slabs][20]
+  unsigned int spin_limit;  // streaming kernel: polls after which a wait on a shared-memory barrier gives up (kErrTimeout)
+  int drop_item;            // streaming kernel, tests of the timeout path: CTA 0 omits the tile load of this item (-1: none)
   int len_host[kHostLens];
   int tot_host[kHostLens];
 };

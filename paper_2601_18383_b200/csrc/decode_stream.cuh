@@ -70,7 +70,7 @@ constexpr int kStCombFloats = kStConsumerWarps * 4 * 128;
 constexpr int kStMaxCtas = 320;                  // partial slots exist for this many CTAs
 constexpr int kStPartStride = 8 * 128 + 16;      // floats per partial: O[8][128], m[8], l[8]
 constexpr int kStMaxBatch = 512;                 // sequences whose chunk prefix fits shared memory
-constexpr uint32_t kStSpinLimit = 1u << 22;      // bounded mbarrier polling
+constexpr uint32_t kStSpinLimit = 1u << 22;      // bounded mbarrier polling: the default limit (DecodeParams::spin_limit)
 constexpr int kStPendWords = 20;                 // a recorded score pass: n, n_old, M[8], 1/L[8], 2 spare
 
 __host__ __device__ inline size_t stream_smem_bytes(int Nb) {
@@ -114,9 +114,9 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // Polls with an iteration limit.  On expiry the status word gets the timeout bit and the CTA-wide
 // abort flag is raised; every later wait of the CTA then returns at once, so the kernel ends (its
 // results are void, which the status word says).
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err) {
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err, uint32_t limit) {
   if (*abort_flag) return;
-  for (uint32_t i = 0; i < kStSpinLimit; ++i) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return;
     if ((i & 1023u) == 1023u && *abort_flag) return;
   }
@@ -613,7 +613,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
                 (sbase & 1023u) == 0u;
       for (int it = 0; it < cnt; ++it) {
         if (in_grp == 0) {  // the group's stages of the previous round have all been consumed
-          mbar_wait(bar_empty + 8 * grp, ph ^ 1u, s_abort, p.err);
+          mbar_wait(bar_empty + 8 * grp, ph ^ 1u, s_abort, p.err, p.spin_limit);
           if (*s_abort) break;
         }
         if (!ok) {
@@ -626,10 +626,14 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         }
         const uint32_t full = bar_full + 8 * stage;
         const uint32_t dst = sbase + (uint32_t)stage * kTxBytes;
-        mbar_arrive_expect_tx(full, kTxBytes);
-        s_flags[16 + stage] = 1 + (int)ph;  // phase of the loads now in flight, for the drain below
-        tma_load_3d(dst, &tmKV, 0, row, 0, full, pol);
-        if constexpr (!KV8) tma_load_3d(dst + kHalf, &tmKV, 64, row, 0, full, pol);
+        // (p.drop_item >= 0, for tests of the timeout path: CTA 0 neither arms nor loads that item, so
+        // the consumers' bounded wait for it runs out)
+        if (!(p.drop_item == it && blockIdx.x == 0)) {
+          mbar_arrive_expect_tx(full, kTxBytes);
+          s_flags[16 + stage] = 1 + (int)ph;  // phase of the loads now in flight, for the drain below
+          tma_load_3d(dst, &tmKV, 0, row, 0, full, pol);
+          if constexpr (!KV8) tma_load_3d(dst + kHalf, &tmKV, 64, row, 0, full, pol);
+        }
         row += kStRows;
         ++stage;
         if (++in_grp == kGS) {
@@ -715,7 +719,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         const int item = it + k;  // item & 1 == pair
         const int stage = cs;     // == item % NS
         const int row0 = (c.chunk + k) * kStRows;
-        if (!peek_ok) mbar_wait(bar_full + 8 * stage, cp, s_abort, p.err);
+        if (!peek_ok) mbar_wait(bar_full + 8 * stage, cp, s_abort, p.err, p.spin_limit);
         __syncwarp();
         cs += 2;
         if (cs >= NS) {
@@ -1021,7 +1025,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         if (!handed && it + seg >= cnt && defer_on()) {
           // the CTA's last slab: nothing is left to overlap the pass with; record it for the next launch
           // (once the scorer warp is done with the record the previous launch left in the same place)
-          mbar_wait(smem_u32(s_tbar + 4), 0u, s_abort, p.err);
+          mbar_wait(smem_u32(s_tbar + 4), 0u, s_abort, p.err, p.spin_limit);
           int* rec = p.pend + slab * kStPendWords;
           if (tid < 8) {
             reinterpret_cast<float*>(rec)[2 + tid] = s_finM[tid];
@@ -1032,7 +1036,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
           }
         } else if (!handed) {
           // (the recorded pass of this slab, if any, must have been applied first)
-          if (defer_on()) mbar_wait(smem_u32(s_tbar + 4), 0u, s_abort, p.err);
+          if (defer_on()) mbar_wait(smem_u32(s_tbar + 4), 0u, s_abort, p.err, p.spin_limit);
           float* dout = p.delta_out ? p.delta_out + slab * (size_t)p.cap : nullptr;
           DYNTS_DISPATCH_GROUP(G, score_pass<GG>(p.accumulate != 0, score, p.comp + slab * (size_t)p.cap, dout, lg, p.cap, n,
                                                  n_old, s_finM, s_finf, tid, kStConsumers));
@@ -1044,7 +1048,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
     }
     if (tid == 0 && it >= cnt) {  // tell the scorer warp that nothing more will come
       const int slot = n_posted & 1;
-      if (n_posted >= 2) mbar_wait(tbar_empty + 8 * slot, (((uint32_t)n_posted >> 1) & 1u) ^ 1u, s_abort, p.err);  // (else never used)
+      if (n_posted >= 2) mbar_wait(tbar_empty + 8 * slot, (((uint32_t)n_posted >> 1) & 1u) ^ 1u, s_abort, p.err, p.spin_limit);  // (else never used)
       s_task[slot].slab = -1;
       mbar_arrive(tbar_full + 8 * slot);
     }
@@ -1076,7 +1080,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
     if (lane == 0) mbar_arrive(smem_u32(s_tbar + 4));
     for (int t = 0;; ++t) {
       const int slot = t & 1;
-      mbar_wait(tbar_full + 8 * slot, (uint32_t)(t >> 1) & 1u, s_abort, p.err);
+      mbar_wait(tbar_full + 8 * slot, (uint32_t)(t >> 1) & 1u, s_abort, p.err, p.spin_limit);
       __syncwarp();
       if (*s_abort) break;
       const StScoreTask& tk = s_task[slot];
@@ -1097,7 +1101,7 @@ decode_attn_stream_kernel(const DecodeParams p, const __grid_constant__ CUtensor
     for (int s = 0; s < NS; ++s) {
       const int armed = s_flags[16 + s];
       if (armed == 0) continue;
-      for (uint32_t i = 0; i < kStSpinLimit; ++i)
+      for (uint32_t i = 0; i < kStSpinLimit; ++i)  // (the full default limit: these loads were issued and will land)
         if (mbar_try_wait(bar_full + 8 * s, (uint32_t)(armed - 1))) break;
     }
   }

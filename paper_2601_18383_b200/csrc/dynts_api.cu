@@ -132,6 +132,8 @@ struct dynts_cache {
   std::vector<int> seq_budget, len_h, tot_h, pinned_h, target_h, active_h;  // host mirrors of the per-sequence state
   int layer_cursor = 0;      // next layer expected by dynts_decode_attn_layer
   int cluster = 0, variant = 0;
+  unsigned int wait_limit = dynts::kStSpinLimit;  // polls of a bounded device-side wait
+  int drop_item = -1;        // one-shot: the next streaming decode launch omits this tile load of CTA 0 (timeout-path test)
   int evict_split = 0;       // CTAs per slab of the eviction: 0 automatic, 1/2/4/8 forced, -1 the one-CTA kernel with shared-memory keys
   int score_source = 0;      // 0: attention mass accumulates (Eq. 6); 1: the caller supplies scores (Eq. 7)
   int parity = 0;            // half of the logit scratch the next decode step writes
@@ -366,6 +368,8 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
 
   // Lengths with the launch (streaming kernel): not while the stream is being captured, since a
   // replayed graph would carry the lengths of the capture.
+  p.spin_limit = c->wait_limit;
+  p.drop_item = -1;
   p.n_host = 0;
   if (Nb <= dynts::kHostLens) {
     cudaStreamCaptureStatus cap_status = cudaStreamCaptureStatusNone;
@@ -435,6 +439,8 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
       if (fs != DYNTS_OK) return fs;
     }
     p.defer = defer ? 1 : 0;
+    p.drop_item = c->drop_item;
+    c->drop_item = -1;
     auto* stream_kernel = !kv8 ? dynts::decode_attn_stream_kernel<false, true>
                                : (defer ? dynts::decode_attn_stream_kernel<true, true> : dynts::decode_attn_stream_kernel<true, false>);
     cudaLaunchConfig_t sc;
@@ -1107,6 +1113,20 @@ dynts_status_t dynts_cache_set_launch(dynts_cache_t* c, int cluster, int variant
   return DYNTS_OK;
 }
 
+dynts_status_t dynts_cache_set_wait_limit(dynts_cache_t* c, unsigned int polls) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (polls < 64u) return fail(DYNTS_ERR_INVALID_ARG, "the limit must be at least 64 polls");
+  c->wait_limit = polls;
+  return DYNTS_OK;
+}
+
+dynts_status_t dynts_debug_drop_tile_load(dynts_cache_t* c, int item) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (item < 0) return fail(DYNTS_ERR_INVALID_ARG, "item must not be negative");
+  c->drop_item = item;
+  return DYNTS_OK;
+}
+
 dynts_status_t dynts_cache_set_evict_launch(dynts_cache_t* c, int split) {
   if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
   if (!(split == -1 || split == 0 || split == 1 || split == 2 || split == 4 || split == 8))
@@ -1412,6 +1432,24 @@ dynts_status_t dynts_evict_noalloc(void* K, void* V, int* pos, float* score, int
   const unsigned groups = (unsigned)((pieces + 3) / 4);
   dynts::evict_compact_kernel<<<dim3(2 * groups, (unsigned)n_slabs, 1), dynts::kCompactThreads, 0, st>>>(p);
   CUDA_TRY(cudaGetLastError());
+  return DYNTS_OK;
+}
+
+dynts_status_t dynts_evict_noalloc_status(void* stream) {
+  int dev = -1;
+  CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return fail(DYNTS_ERR_INVALID_ARG, "device index %d not supported", dev);
+  int* base = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    base = g_noalloc_ptr[dev];
+  }
+  if (!base) return DYNTS_OK;  // no call on this device yet
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int word = 0;  // (a pageable destination: the copy is staged by the runtime, nothing is allocated here)
+  CUDA_TRY(cudaMemcpyAsync(&word, base + 3, sizeof(int), cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  if (word != 0) return fail(DYNTS_ERR_DEVICE, "the last dynts_evict_noalloc call found inconsistent lengths on the device (status word 0x%x) and moved nothing for those slabs", word);
   return DYNTS_OK;
 }
 

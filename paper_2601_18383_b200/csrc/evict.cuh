@@ -72,6 +72,15 @@ __global__ void __launch_bounds__(kSelectThreads) evict_select_kernel(const Evic
   const int M = p.pinned[b];
   const int lo = M, hi = n - p.window;  // selection window [lo, hi)
   const int k = tgt - M - p.window;     // survivors wanted from it (host guarantees 0 <= k < hi - lo)
+  if (n > p.cap || M < 0 || k < 0 || hi < lo || k > hi - lo) {  // uniform over the CTA; the host's checks prevent it
+    if (tid == 0) {
+      atomicOr(p.err, kErrLenOverflow);  // recorded, and nothing moves
+      hdr[0] = n;
+      hdr[1] = n;
+      hdr[2] = n;
+    }
+    return;
+  }
 
   extern __shared__ __align__(16) uint32_t esm[];
   uint32_t* raw = esm;                                   // [cap] score bit patterns

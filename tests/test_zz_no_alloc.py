@@ -57,7 +57,7 @@ def _check(cfg, rows, seed):
     D.dynts_evict_noalloc(K, V, pos, score, slabs, cfg.head_dim, D.DYNTS_BF16 if cfg.dtype == "bf16" else D.DYNTS_FP32,
                           cap, rows, cfg.prompt, cfg.window, cfg.budget,
                           torch.cuda.current_stream().cuda_stream)
-    torch.cuda.synchronize()
+    D.dynts_evict_noalloc_status(torch.cuda.current_stream().cuda_stream)   # waits; raises if a device-side check fired
     n = min(rows, cfg.budget)
     for i, (Kr, Vr, pr, sr) in enumerate(ref):
         assert Kr.shape[0] == n
