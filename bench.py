@@ -475,8 +475,9 @@ def time_predictor(batch, device, peak, d=4096, iters=40):
 
 
 def time_prefill(cfg, device, iters=10):
-    """Times dynts_prefill_attn on the workload's prompt (all layers, batch, heads); flops = 4 d per
-    (query, key) pair of the causal triangle; peak = the measured dense bf16 GEMM rate."""
+    """Times the prompt attention (dynts_prompt_attn: Eq. 4-5 over the workload's prompt, all heads of
+    up to 8 layers; the fill of the slabs is not part of it); flops = 4 d per (query, key) pair of the
+    causal triangle; peak = the measured dense bf16 GEMM rate."""
     import torch
     import paper_2601_18383_b200 as D
     sub = cfg.scaled(layers=min(cfg.layers, 8), seq_budgets=None, budget=max(cfg.budget, cfg.prompt))
@@ -489,13 +490,14 @@ def time_prefill(cfg, device, iters=10):
     out = torch.empty_like(q)
     st = torch.cuda.current_stream(device)
     for _ in range(3):
-        cache.prefill_attn(q, k, v, out)
+        cache.prompt_attn(q, k, v, out)
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record(st)
     for _ in range(iters):
-        cache.prefill_attn(q, k, v, out)
+        cache.prompt_attn(q, k, v, out)
     b.record(st)
     torch.cuda.synchronize(device)
+    cache.poll_error()
     us = a.elapsed_time(b) * 1e3 / iters
     cache.close()
     flops = 4 * 128 * (T * (T + 1) // 2) * sub.layers * sub.batch * sub.q_heads
@@ -505,9 +507,9 @@ def time_prefill(cfg, device, iters=10):
     except Exception:
         peak_tf, kind = 1590.0, "fallback"
     tf = flops / (us * 1e-6) / 1e12
-    return {"prompt_tokens": T, "layers_timed": sub.layers, "us_per_call": round(us, 1), "flops": flops, "bound": "tensor",
-            "achieved": round(tf, 1), "peak": peak_tf, "peak_kind": kind, "unit": "TFLOP/s", "frac": round(tf / peak_tf, 4),
-            "note": "includes the copy of the prompt K/V rows into the slabs"}
+    return {"kernel": "prefill_attn (tcgen05.mma, accumulators in tensor memory, TMA operands)", "prompt_tokens": T,
+            "layers_timed": sub.layers, "us_per_call": round(us, 1), "flops": flops, "bound": "tensor",
+            "achieved": round(tf, 1), "peak": peak_tf, "peak_kind": kind, "unit": "TFLOP/s", "frac": round(tf / peak_tf, 4)}
 
 
 def oracle_baseline(cfg, cache, q_ring, k_ring, v_ring, budget_s=20.0, slabs=None):

@@ -105,10 +105,15 @@ dynts_status_t dynts_prefill(dynts_cache_t* c, const void* k, const void* v, int
  *   q, out: device [L, Nb, Hq, n_tokens, d];  k, v: device [L, Nb, Hkv, n_tokens, d]; bf16, d = 128.
  * The rows are stored exactly as dynts_prefill stores them (the first n_pinned pinned with score
  * +inf); prompt attention adds nothing to the scores (the paper pins the question instead of
- * scoring it).  A dense contraction: runs on the tensor pipe.  Other dtypes and head sizes:
- * DYNTS_ERR_INVALID_ARG. */
+ * scoring it).  A dense contraction: it runs on the tensor cores (tcgen05, accumulators in tensor
+ * memory, operands by TMA).  Other dtypes and head sizes: DYNTS_ERR_INVALID_ARG.  A bounded wait
+ * inside the kernel that runs out is reported by dynts_poll_error (DYNTS_ERR_DEVICE). */
 dynts_status_t dynts_prefill_attn(dynts_cache_t* c, const void* q, const void* k, const void* v, void* out, int n_tokens,
                                   int n_pinned);
+
+/* The attention part of dynts_prefill_attn alone (Eq. 4-5 for t = 1..n_tokens): reads q, k, v,
+ * writes out, leaves the cache untouched.  Same shapes and restrictions. */
+dynts_status_t dynts_prompt_attn(dynts_cache_t* c, const void* q, const void* k, const void* v, void* out, int n_tokens);
 
 /* The same for one sequence of a ragged batch; k, v: device [L, Hkv, n_tokens, d].  Marks the
  * sequence active. */

@@ -67,6 +67,7 @@ _sigs = {
     "dynts_cache_set_stream": (C.c_int, [_P, _P]),
     "dynts_prefill": (C.c_int, [_P, _P, _P, C.c_int, C.c_int]),
     "dynts_prefill_attn": (C.c_int, [_P, _P, _P, _P, _P, C.c_int, C.c_int]),
+    "dynts_prompt_attn": (C.c_int, [_P, _P, _P, _P, _P, C.c_int]),
     "dynts_prefill_seq": (C.c_int, [_P, C.c_int, _P, _P, C.c_int, C.c_int]),
     "dynts_decode_attn": (C.c_int, [_P, _P, _P, _P, _P, _P]),
     "dynts_decode_attn_layer": (C.c_int, [_P, C.c_int, _P, _P, _P, _P, _P]),
@@ -182,6 +183,10 @@ def dynts_prefill(c, k, v, n_tokens, n_pinned):
 
 def dynts_prefill_attn(c, q, k, v, out, n_tokens, n_pinned):
     return _check(lib.dynts_prefill_attn(c, _ptr(q), _ptr(k), _ptr(v), _ptr(out), n_tokens, n_pinned))
+
+
+def dynts_prompt_attn(c, q, k, v, out, n_tokens):
+    return _check(lib.dynts_prompt_attn(c, _ptr(q), _ptr(k), _ptr(v), _ptr(out), n_tokens))
 
 
 def dynts_prefill_seq(c, seq, k, v, n_tokens, n_pinned):
@@ -363,6 +368,9 @@ class Cache:
     def prefill_attn(self, q, k, v, out, n_pinned=None):
         T = k.shape[-2]
         return dynts_prefill_attn(self.handle, q, k, v, out, T, T if n_pinned is None else n_pinned)
+
+    def prompt_attn(self, q, k, v, out):
+        return dynts_prompt_attn(self.handle, q, k, v, out, k.shape[-2])
 
     def prefill_seq(self, seq, k, v, n_pinned=None):
         T = k.shape[-2]

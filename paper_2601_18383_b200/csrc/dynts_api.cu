@@ -815,6 +815,58 @@ dynts_status_t dynts_prefill(dynts_cache_t* c, const void* k, const void* v, int
   return do_prefill(c, -1, k, v, n_tokens, n_pinned);
 }
 
+dynts_status_t dynts_prompt_attn(dynts_cache_t* c, const void* q, const void* k, const void* v, void* out, int n_tokens) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (!q || !out || !k || !v || !aligned16(q) || !aligned16(out) || !aligned16(k) || !aligned16(v))
+    return fail(DYNTS_ERR_INVALID_ARG, "q, k, v and out must be non-NULL and 16-byte aligned");
+  if ((c->cfg.dtype != DYNTS_BF16 && c->cfg.dtype != DYNTS_BF16_KV8) || c->cfg.head_dim != 128)
+    return fail(DYNTS_ERR_INVALID_ARG, "prefill attention needs bf16 q/k/v and head_dim 128");
+  if (n_tokens < 1) return fail(DYNTS_ERR_INVALID_ARG, "n_tokens must be positive");
+  dynts_status_t st = materialise(c);
+  if (st != DYNTS_OK) return st;
+  const long long lb = (long long)c->cfg.layers * c->cfg.batch;
+  if (lb > 65535 || (long long)n_tokens * 256 >= (1ll << 40))
+    return fail(DYNTS_ERR_INVALID_ARG, "layers x batch %lld or n_tokens %d beyond the launch limits", lb, n_tokens);
+  if (!c->attr_prefill) {
+    CUDA_TRY(cudaFuncSetAttribute(dynts::prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dynts::kPfSmemBytes));
+    c->attr_prefill = true;
+  }
+  // Tensor maps over the caller's tensors, [heads][n_tokens][128]: a box never reaches into the next
+  // head, rows beyond the prompt come back as zeros.  128-byte swizzle, boxes of 64 elements.
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+  if (!fn || qres != cudaDriverEntryPointSuccess) return fail(DYNTS_ERR_CUDA, "the driver has no cuTensorMapEncodeTiled");
+  tensor_map_encode_fn encode = reinterpret_cast<tensor_map_encode_fn>(fn);
+  CUtensorMap mq, mk, mv;
+  const cuuint64_t strides[2] = {256, (cuuint64_t)n_tokens * 256};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  auto make = [&](CUtensorMap* m, const void* base, int heads, int box_rows) -> CUresult {
+    const cuuint64_t dims[3] = {128, (cuuint64_t)n_tokens, (cuuint64_t)lb * heads};
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+    return encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  };
+  CUresult r = make(&mq, q, c->cfg.q_heads, dynts::kPfRows);
+  if (r == CUDA_SUCCESS) r = make(&mk, k, c->cfg.kv_heads, dynts::kPfKeys);
+  if (r == CUDA_SUCCESS) r = make(&mv, v, c->cfg.kv_heads, dynts::kPfKeys);
+  if (r != CUDA_SUCCESS) return fail(DYNTS_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
+  dynts::PrefillAttnParams p;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.err = c->err_dev;
+  p.stop = reinterpret_cast<int*>(c->ticket()) + 4;  // a spare word of the ticket block (zero since the cache was created)
+  p.T = n_tokens;
+  p.Hq = c->cfg.q_heads;
+  p.Hkv = c->cfg.kv_heads;
+  p.scale_log2 = (float)(1.4426950408889634 / std::sqrt(128.0));
+  const dim3 grid((unsigned)((n_tokens + dynts::kPfRows - 1) / dynts::kPfRows), (unsigned)c->cfg.q_heads, (unsigned)lb);
+  dynts::prefill_attn_kernel<<<grid, dynts::kPfThreads, dynts::kPfSmemBytes, c->stream>>>(p, mq, mk, mv);
+  CUDA_TRY(cudaGetLastError());
+  c->launches += 1;
+  return DYNTS_OK;
+}
+
 dynts_status_t dynts_prefill_attn(dynts_cache_t* c, const void* q, const void* k, const void* v, void* out, int n_tokens,
                                   int n_pinned) {
   if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
@@ -825,25 +877,7 @@ dynts_status_t dynts_prefill_attn(dynts_cache_t* c, const void* q, const void* k
   if (n_tokens < 1) return fail(DYNTS_ERR_INVALID_ARG, "n_tokens must be positive");
   dynts_status_t st = do_prefill(c, -1, k, v, n_tokens, n_pinned);  // rows, positions, pins
   if (st != DYNTS_OK) return st;
-  if (!c->attr_prefill) {
-    CUDA_TRY(cudaFuncSetAttribute(dynts::prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dynts::kPfSmemBytes));
-    c->attr_prefill = true;
-  }
-  dynts::PrefillAttnParams p;
-  p.q = static_cast<const __nv_bfloat16*>(q);
-  p.k = static_cast<const __nv_bfloat16*>(k);
-  p.v = static_cast<const __nv_bfloat16*>(v);
-  p.out = static_cast<__nv_bfloat16*>(out);
-  p.T = n_tokens;
-  p.Hq = c->cfg.q_heads;
-  p.Hkv = c->cfg.kv_heads;
-  p.scale_log2 = (float)(1.4426950408889634 / std::sqrt(128.0));
-  const dim3 grid((unsigned)((n_tokens + dynts::kPfRows - 1) / dynts::kPfRows), (unsigned)c->cfg.q_heads,
-                  (unsigned)(c->cfg.layers * c->cfg.batch));
-  dynts::prefill_attn_kernel<<<grid, dynts::kPfThreads, dynts::kPfSmemBytes, c->stream>>>(p);
-  CUDA_TRY(cudaGetLastError());
-  c->launches += 1;
-  return DYNTS_OK;
+  return dynts_prompt_attn(c, q, k, v, out, n_tokens);
 }
 
 dynts_status_t dynts_prefill_seq(dynts_cache_t* c, int seq, const void* k, const void* v, int n_tokens, int n_pinned) {

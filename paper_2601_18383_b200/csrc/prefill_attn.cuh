@@ -1,220 +1,302 @@
 // Prefill attention for sm_100a: every prompt position attends to the positions up to and
 // including itself (Eq. 4-5 with t = 1..M), bf16, head_dim 128, grouped query heads.  This is the
 // phase that fills the question window (Section 4.2); unlike the decode step it is a dense
-// contraction (M x M x d per head), so all of it runs on the tensor pipe.
+// contraction (M x M x d per head), and it runs on the 5th-generation tensor path: tcgen05.mma with
+// the accumulators in tensor memory, operands brought into shared memory by TMA tile loads.
 //
-// One CTA = 64 query rows of one query head (4 warps x 16 rows); it walks the key/value rows in
-// tiles of 64 up to the diagonal.  K and V tiles are staged in shared memory by 16-byte cp.async
-// copies, double-buffered, with the 16-byte pieces of a row XOR-swizzled by the row index so that
-// ldmatrix reads are bank-conflict-free.  S = Q K^T and O += P V are mma.sync m16n8k16 (bf16 in,
-// fp32 accumulate); the S accumulators are re-used in registers as the A operand of the second
-// product; the softmax is kept online per row (running max and sum, rescale of O).
+// One CTA = 128 query rows of one query head.  It walks the key/value rows in tiles of 64 up to the
+// diagonal; per tile
+//     S  = Q K^T          M 128 x N 64 x K 128   (8 instructions of K = 16; Q and K tiles K-major)
+//     P  = exp2(S * scale - rowmax)               (online softmax: running max and sum per row)
+//     O += P V            M 128 x N 128 x K 64   (4 instructions; P K-major, V MN-major)
+// Five warps.  Warps 0-3 are the softmax warps: thread r owns query row r, i.e. lane r of tensor
+// memory -- it reads its row of S with tcgen05.ld, keeps the row's running max and sum, rescales
+// its row of O in tensor memory when the max moves, and writes its row of P (bf16) into a
+// shared-memory tile in the 128-byte-swizzled layout the MMA's descriptor expects.  One thread of
+// warp 4 issues everything asynchronous: the TMA loads (Q once; K and V tiles into two stages each,
+// requested as soon as the product that read the stage before has completed) and the MMAs, whose
+// completion it hands to the softmax warps through mbarriers (tcgen05.commit).  S is double
+// buffered in tensor memory (columns 0-63 / 64-127; O in 128-255), so S of tile j + 1 is computed
+// while the softmax of tile j runs.  112 KB of shared memory and 256 columns of tensor memory per
+// CTA: two CTAs share an SM and fill each other's bubbles.
+//
+// Tiles above the diagonal are never loaded.  Rows and keys beyond the prompt come back from TMA
+// as zeros (the tensor maps are [heads][T][128], so a box never reaches into the next head) and
+// are masked like the keys above the diagonal.  No load uses cluster multicast.  Every wait is
+// bounded: on expiry the CTA raises the timeout bit of the status word, every later wait returns
+// at once, the CTA waits (bounded) for what it has in flight, frees its tensor memory and ends.
 #pragma once
 
+#include <cuda.h>
 #include <math_constants.h>
 
 #include "common.cuh"
-#include "decode_attn.cuh"  // mma_bf16_m16n8k16, pack_bf16x2
+#include "decode_stream.cuh"  // mbarrier wrappers, smem_u32
+#include "tc5.cuh"
 
 namespace dynts {
 
-constexpr int kPfRows = 64;      // query rows per CTA and key rows per tile
-constexpr int kPfThreads = 128;
-constexpr int kPfTileBytes = kPfRows * 256;  // 64 rows x 128 bf16
-constexpr int kPfSmemBytes = 4 * kPfTileBytes;  // K x 2, V x 2; the Q tile borrows the second K buffer until its fragments are in registers
+constexpr int kPfRows = 128;                      // query rows per CTA
+constexpr int kPfKeys = 64;                       // key rows per tile
+constexpr int kPfThreads = 160;                   // 4 softmax warps + 1 warp for TMA and MMA issue
+constexpr int kPfQBytes = kPfRows * 256;          // two boxes of 128 rows x 64 bf16
+constexpr int kPfKvBytes = kPfKeys * 256;         // two boxes of 64 rows x 64 bf16
+constexpr int kPfPBytes = kPfRows * 128;          // 128 rows x 64 bf16
+// Two CTAs must fit the 227 KB of an SM (each also costs 1 KB of system space), so there is no room
+// for alignment slack: the dynamic shared memory is declared 1024-byte aligned (what the 128-byte
+// swizzle needs) and the kernel checks that it is.
+constexpr int kPfSmemBytes = kPfQBytes + 4 * kPfKvBytes + kPfPBytes + 128;
+constexpr uint32_t kPfTmemCols = 256;             // S0 | S1 | O
+constexpr uint32_t kPfSpinLimit = 1u << 21;
 
 struct PrefillAttnParams {
-  const __nv_bfloat16* q;  // [L, Nb, Hq, T, 128]
-  const __nv_bfloat16* k;  // [L, Nb, Hkv, T, 128]
-  const __nv_bfloat16* v;
   __nv_bfloat16* out;      // [L, Nb, Hq, T, 128]
+  int* err;                // pinned host status word
+  int* stop;               // device word: non-zero once a CTA of this cache's prefill launches has given up a wait
   int T, Hq, Hkv;
   float scale_log2;
 };
 
-__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, bool valid) {
-  const int bytes = valid ? 16 : 0;  // src-size 0: the destination is filled with zeros
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void pf_ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-               : "r"(addr));
-}
-__device__ __forceinline__ void pf_ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-               : "r"(addr));
+__device__ __forceinline__ void pf_tma_load(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
 }
 
-// Copies rows [row0, row0 + 64) of a [T][128] bf16 matrix into a swizzled tile: piece c (16 bytes)
-// of tile row r lands at r * 256 + ((c ^ (r & 7)) * 16).  Rows at or beyond T become zeros.
-__device__ __forceinline__ void pf_load_tile(uint32_t tile, const __nv_bfloat16* src, int row0, int T, int tid) {
-#pragma unroll
-  for (int i = 0; i < (kPfRows * 16) / kPfThreads; ++i) {
-    const int e = tid + i * kPfThreads;
-    const int r = e >> 4, c = e & 15;
-    const bool ok = row0 + r < T;
-    const __nv_bfloat16* s = src + (size_t)(ok ? row0 + r : 0) * 128 + c * 8;
-    cp_async_16(tile + r * 256 + ((c ^ (r & 7)) << 4), s, ok);
-  }
-}
+__global__ void __launch_bounds__(kPfThreads, 2)
+prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                    const __grid_constant__ CUtensorMap tmV) {
+  extern __shared__ __align__(1024) uint8_t pf_smem[];
+  uint8_t* sm = pf_smem;
+  const uint32_t sQ = smem_u32(sm);                       // [2 halves of head_dim][128 rows][128 B]
+  const uint32_t sK = sQ + kPfQBytes;                     // [2 stages][2 halves][64 rows][128 B]
+  const uint32_t sV = sK + 2 * kPfKvBytes;                // the same
+  uint8_t* sP_ptr = sm + kPfQBytes + 4 * kPfKvBytes;      // [128 rows][128 B]
+  const uint32_t sP = smem_u32(sP_ptr);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sP_ptr + kPfPBytes);
+  // barriers: 0 Q, 1-2 K stages, 3-4 V stages, 5-6 S buffers, 7 O, 8 P, 9 drain
+  const uint32_t bar0 = smem_u32(bars);
+  auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 10);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
-// grid = (query tiles, Hq, L * Nb); tiles are taken from the last (longest) to the first.
-__global__ void __launch_bounds__(kPfThreads, 3) prefill_attn_kernel(const PrefillAttnParams p) {
-  extern __shared__ __align__(128) uint8_t pf_smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int gid = lane >> 2, tig = lane & 3;
   const int T = p.T;
-  const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;
-  const int hq = blockIdx.y, lb = blockIdx.z;
-  const int h = hq / (p.Hq / p.Hkv);
-  const __nv_bfloat16* Q = p.q + ((size_t)lb * p.Hq + hq) * T * 128;
-  const __nv_bfloat16* K = p.k + ((size_t)lb * p.Hkv + h) * T * 128;
-  const __nv_bfloat16* V = p.v + ((size_t)lb * p.Hkv + h) * T * 128;
-  __nv_bfloat16* O = p.out + ((size_t)lb * p.Hq + hq) * T * 128;
-  const uint32_t sK = (uint32_t)__cvta_generic_to_shared(pf_smem), sV = sK + 2 * kPfTileBytes;  // two buffers each
-  const uint32_t sQ = sK + kPfTileBytes;  // = K buffer 1, free until the first prefetch
-  const int q0 = qt * kPfRows;
+  const int q0 = blockIdx.x * kPfRows;
+  const int h = blockIdx.y, lb = blockIdx.z;
+  const int zq = lb * p.Hq + h;
+  const int zkv = lb * p.Hkv + h / (p.Hq / p.Hkv);
+  const int q_last = min(T - 1, q0 + kPfRows - 1);
+  const int n_kt = q_last / kPfKeys + 1;  // key tiles up to the diagonal
 
-  pf_load_tile(sQ, Q, q0, T, tid);
-  pf_load_tile(sK, K, 0, T, tid);
-  pf_load_tile(sV, V, 0, T, tid);
-  cp_async_commit();
-  cp_async_wait<0>();
+  if (tid == 0) {
+    for (int i = 0; i < 10; ++i) mbar_init(bar(i), i == 8 ? (kPfThreads - 32) : 1);
+    // (a launch whose waits run out must not take one time limit per CTA: the CTAs that start after the
+    // first one gave up see the word and skip their work)
+    *s_abort = *reinterpret_cast<volatile int*>(p.stop) != 0 ? 1 : 0;
+    if ((smem_u32(sm) & 1023u) != 0u) {  // the tiles would not be where the swizzle expects them
+      atomicOr(p.err, kErrStreamBounds);
+      *s_abort = 1;
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 4) {
+    tc5::tmem_alloc(smem_u32(s_tmem), kPfTmemCols);
+    tc5::tmem_relinquish();
+  }
+  tc5::fence_before_sync();
   __syncthreads();
+  tc5::fence_after_sync();
+  const uint32_t tmem = *s_tmem;
+  const uint32_t tS0 = tmem, tO = tmem + 128;  // S buffer b at column 64 b
 
-  // Q fragments of this warp's 16 rows: A operand of all 8 k-steps
-  uint32_t qa[8][4];
-  {
-    const int r = warp * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+  if (warp == 4) {
+    if (lane == 0) {
+      // ================= the issuing thread: TMA loads and MMAs =================
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmQ)) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmK)) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmV)) : "memory");
+      auto load_k = [&](int j) {
+        const uint32_t dst = sK + (uint32_t)(j & 1) * kPfKvBytes;
+        mbar_arrive_expect_tx(bar(1 + (j & 1)), kPfKvBytes);
+        pf_tma_load(dst, &tmK, 0, j * kPfKeys, zkv, bar(1 + (j & 1)));
+        pf_tma_load(dst + kPfKvBytes / 2, &tmK, 64, j * kPfKeys, zkv, bar(1 + (j & 1)));
+      };
+      auto load_v = [&](int j) {
+        const uint32_t dst = sV + (uint32_t)(j & 1) * kPfKvBytes;
+        mbar_arrive_expect_tx(bar(3 + (j & 1)), kPfKvBytes);
+        pf_tma_load(dst, &tmV, 0, j * kPfKeys, zkv, bar(3 + (j & 1)));
+        pf_tma_load(dst + kPfKvBytes / 2, &tmV, 64, j * kPfKeys, zkv, bar(3 + (j & 1)));
+      };
+      constexpr uint32_t idesc_s = tc5::idesc_bf16_f32(kPfRows, kPfKeys, 0, 0);   // Q K^T: both K-major
+      constexpr uint32_t idesc_o = tc5::idesc_bf16_f32(kPfRows, 128, 0, 1);       // P V: V is MN-major
+      auto mma_s = [&](int j) {  // S_j = Q K_j^T into S buffer j & 1
+        const uint32_t kb = sK + (uint32_t)(j & 1) * kPfKvBytes;
 #pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
-      const int c = 2 * kk + (lane >> 4);
-      pf_ldmatrix_x4(sQ + r * 256 + ((c ^ (r & 7)) << 4), qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3]);
-    }
-  }
-  __syncthreads();  // every warp has its Q fragments: the buffer may be overwritten by the first prefetch
-  float o[16][4];
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint32_t a = sQ + (uint32_t)(kk >> 2) * (kPfQBytes / 2) + (uint32_t)(kk & 3) * 32;
+          const uint32_t b = kb + (uint32_t)(kk >> 2) * (kPfKvBytes / 2) + (uint32_t)(kk & 3) * 32;
+          tc5::mma_bf16_ss(tS0 + 64u * (uint32_t)(j & 1), tc5::smem_desc_sw128(a, 16, 1024), tc5::smem_desc_sw128(b, 16, 1024), idesc_s,
+                           kk > 0);
+        }
+        tc5::mma_commit(bar(5 + (j & 1)));
+      };
+      auto mma_o = [&](int j) {  // O += P_j V_j
+        const uint32_t vb = sV + (uint32_t)(j & 1) * kPfKvBytes;
 #pragma unroll
-  for (int db = 0; db < 16; ++db)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) o[db][e] = 0.f;
-  float m_run[2] = {-CUDART_INF_F, -CUDART_INF_F}, l_run[2] = {0.f, 0.f};
-  const int qi0 = q0 + warp * 16 + gid;  // this thread's rows: qi0 and qi0 + 8
+        for (int kk = 0; kk < 4; ++kk)  // 16 keys per step: 32 bytes along a row of P, two 8-row groups of V
+          tc5::mma_bf16_ss(tO, tc5::smem_desc_sw128(sP + (uint32_t)kk * 32, 16, 1024),
+                           tc5::smem_desc_sw128(vb + (uint32_t)kk * 2048, kPfKvBytes / 2, 1024), idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+        tc5::mma_commit(bar(7));
+      };
 
-  for (int kt = 0; kt <= qt; ++kt) {
-    const int buf = kt & 1;
-    if (kt < qt) {  // prefetch the next tile into the other buffer
-      pf_load_tile(sK + (buf ^ 1) * kPfTileBytes, K, (kt + 1) * kPfRows, T, tid);
-      pf_load_tile(sV + (buf ^ 1) * kPfTileBytes, V, (kt + 1) * kPfRows, T, tid);
-      cp_async_commit();
-      cp_async_wait<1>();
-    } else {
-      cp_async_wait<0>();
-    }
-    __syncthreads();
-    const uint32_t tK = sK + buf * kPfTileBytes, tV = sV + buf * kPfTileBytes;
-
-    // S = Q K^T: 8 blocks of 8 keys
-    float sacc[8][4];
-#pragma unroll
-    for (int nb = 0; nb < 8; ++nb)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) sacc[nb][e] = 0.f;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {  // pairs of key blocks
-      const int r = 16 * j + (lane >> 4) * 8 + (lane & 7);
-#pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {
-        const int c = 2 * kk + ((lane >> 3) & 1);
-        uint32_t b0, b1, b2, b3;
-        pf_ldmatrix_x4(tK + r * 256 + ((c ^ (r & 7)) << 4), b0, b1, b2, b3);
-        mma_bf16_m16n8k16(sacc[2 * j], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b0, b1);
-        mma_bf16_m16n8k16(sacc[2 * j + 1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b2, b3);
+      mbar_arrive_expect_tx(bar(0), kPfQBytes);
+      pf_tma_load(sQ, &tmQ, 0, q0, zq, bar(0));
+      pf_tma_load(sQ + kPfQBytes / 2, &tmQ, 64, q0, zq, bar(0));
+      load_k(0);
+      load_v(0);
+      if (n_kt > 1) {
+        load_k(1);
+        load_v(1);
+      }
+      mbar_wait(bar(0), 0u, s_abort, p.err, kPfSpinLimit);
+      mbar_wait(bar(1), 0u, s_abort, p.err, kPfSpinLimit);
+      tc5::fence_after_sync();
+      if (!*s_abort) mma_s(0);
+      if (n_kt > 1) {
+        mbar_wait(bar(2), 0u, s_abort, p.err, kPfSpinLimit);
+        tc5::fence_after_sync();
+        if (!*s_abort) mma_s(1);
+      }
+      for (int j = 0; j < n_kt && !*s_abort; ++j) {
+        const int st = j & 1;
+        if (j >= 1 && j + 1 < n_kt) {  // the V stage of tile j - 1 is free once O += P V of that tile has completed
+          mbar_wait(bar(7), (uint32_t)((j - 1) & 1), s_abort, p.err, kPfSpinLimit);
+          if (!*s_abort) load_v(j + 1);
+        }
+        if (j + 2 < n_kt) {            // the K stage of tile j is free once S_j has completed
+          mbar_wait(bar(5 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);
+          if (!*s_abort) load_k(j + 2);
+        }
+        mbar_wait(bar(8), (uint32_t)(j & 1), s_abort, p.err, kPfSpinLimit);           // P_j written, O rescaled, S_j read
+        mbar_wait(bar(3 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // V_j has landed
+        tc5::fence_after_sync();
+        if (*s_abort) break;
+        mma_o(j);
+        if (j + 2 < n_kt) {
+          mbar_wait(bar(1 + st), (uint32_t)(((j + 2) >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // K_{j+2} has landed
+          tc5::fence_after_sync();
+          if (!*s_abort) mma_s(j + 2);
+        }
+      }
+      if (*s_abort) {
+        atomicOr(p.stop, 1);
+        // Something gave up.  Give what this thread started a bounded time to finish before the shared
+        // and tensor memory are released: the tile loads (every armed barrier completes its phase when
+        // its bytes have landed) and the MMAs (one more commit).
+        for (int i = 0; i < 5; ++i)
+          for (uint32_t s = 0; s < 2; ++s)
+            for (uint32_t w = 0; w < (1u << 16); ++w)
+              if (mbar_try_wait(bar(i), s)) break;
+        tc5::mma_commit(bar(9));
+        for (uint32_t w = 0; w < kPfSpinLimit; ++w)
+          if (mbar_try_wait(bar(9), 0u)) break;
       }
     }
-    // scale, causal mask (only the diagonal tile needs it), online softmax of rows qi0 and qi0 + 8
-    float mx[2] = {-CUDART_INF_F, -CUDART_INF_F};
+  } else {
+    // ================= softmax warps: thread = query row = tensor-memory lane =================
+    const int qpos = q0 + tid;
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    float m = -CUDART_INF_F, l = 0.f;
+    for (int j = 0; j < n_kt; ++j) {
+      mbar_wait(bar(5 + (j & 1)), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // S_j is complete
+      tc5::fence_after_sync();
+      uint32_t s_lo[32], s_hi[32];
+      tc5::tmem_ld32(tS0 + lane_base + 64u * (uint32_t)(j & 1), s_lo);
+      tc5::tmem_ld32(tS0 + lane_base + 64u * (uint32_t)(j & 1) + 32u, s_hi);
+      tc5::tmem_wait_ld();
+      const int key0 = j * kPfKeys;
+      float mx = -CUDART_INF_F;
 #pragma unroll
-    for (int nb = 0; nb < 8; ++nb) {
+      for (int c = 0; c < 32; ++c) {
+        const float a = (key0 + c <= qpos) ? __uint_as_float(s_lo[c]) * p.scale_log2 : -CUDART_INF_F;
+        const float b = (key0 + 32 + c <= qpos) ? __uint_as_float(s_hi[c]) * p.scale_log2 : -CUDART_INF_F;
+        s_lo[c] = __float_as_uint(a);
+        s_hi[c] = __float_as_uint(b);
+        mx = fmaxf(mx, fmaxf(a, b));
+      }
+      // The reference maximum m of a row only has to keep exp2(x - m) in range, not to equal the true
+      // maximum: it is moved (and O and l rescaled) only when the tile's maximum exceeds it by more
+      // than 2^8, so P stays below 256 (bf16 and fp32 have the range) and most tiles rescale nothing.
+      const bool move = mx > m + 8.0f;       // always at the first tile (m = -inf; key 0 is visible to every row)
+      const float m_new = move ? mx : m;
+      const float alpha = move ? fast_exp2(m - m_new) : 1.0f;  // 0 at the first tile, where l and O are empty
+      float sum = 0.f;
+      uint32_t pk[32];  // the row's 64 weights as bf16 pairs
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int kj = kt * kPfRows + 8 * nb + 2 * tig + (e & 1);
-        const int qi = qi0 + (e >> 1) * 8;
-        float x = sacc[nb][e] * p.scale_log2;
-        if (kt == qt && (kj > qi || kj >= T)) x = -CUDART_INF_F;
-        sacc[nb][e] = x;
-        mx[e >> 1] = fmaxf(mx[e >> 1], x);
+      for (int c = 0; c < 16; ++c) {
+        const float a0 = fast_exp2(__uint_as_float(s_lo[2 * c]) - m_new), a1 = fast_exp2(__uint_as_float(s_lo[2 * c + 1]) - m_new);
+        const float b0 = fast_exp2(__uint_as_float(s_hi[2 * c]) - m_new), b1 = fast_exp2(__uint_as_float(s_hi[2 * c + 1]) - m_new);
+        sum += (a0 + a1) + (b0 + b1);
+        pk[c] = pack_bf16x2(a0, a1);
+        pk[16 + c] = pack_bf16x2(b0, b1);
+      }
+      l = l * alpha + sum;
+      m = m_new;
+      if (j > 0) {
+        // O += P V of the tile before must be complete before O is rescaled and before P is overwritten
+        mbar_wait(bar(7), (uint32_t)((j - 1) & 1), s_abort, p.err, kPfSpinLimit);
+        tc5::fence_after_sync();
+        if (__any_sync(0xffffffffu, move)) {  // warp-uniform: the tensor-memory accesses are collective
+#pragma unroll
+          for (int c0 = 0; c0 < 128; c0 += 32) {
+            uint32_t o[32];
+            tc5::tmem_ld32(tO + lane_base + (uint32_t)c0, o);
+            tc5::tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+            tc5::tmem_st32(tO + lane_base + (uint32_t)c0, o);
+          }
+          tc5::tmem_wait_st();
+        }
+      }
+      // the row of P: 16-byte chunk c of row r goes to chunk c ^ (r & 7) of the row's 128 bytes
+#pragma unroll
+      for (int c = 0; c < 8; ++c)
+        *reinterpret_cast<uint4*>(sP_ptr + tid * 128 + ((c ^ (tid & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMA reads P through the async proxy
+      tc5::fence_before_sync();
+      mbar_arrive(bar(8));
+    }
+    // epilogue: the row of O, normalised, rounded to bf16
+    mbar_wait(bar(7), (uint32_t)((n_kt - 1) & 1), s_abort, p.err, kPfSpinLimit);
+    tc5::fence_after_sync();
+    const float inv_l = 1.0f / l;
+    __nv_bfloat16* orow = p.out + ((size_t)zq * T + (size_t)min(qpos, T - 1)) * 128;
+    const bool aborted = *s_abort != 0;  // (then tensor memory may not hold what this row expects: nothing is written)
+#pragma unroll
+    for (int c0 = 0; c0 < 128; c0 += 32) {
+      uint32_t o[32];
+      tc5::tmem_ld32(tO + lane_base + (uint32_t)c0, o);
+      tc5::tmem_wait_ld();
+      if (qpos < T && !aborted) {
+#pragma unroll
+        for (int c = 0; c < 32; c += 8) {
+          uint4 w;
+          w.x = pack_bf16x2(__uint_as_float(o[c]) * inv_l, __uint_as_float(o[c + 1]) * inv_l);
+          w.y = pack_bf16x2(__uint_as_float(o[c + 2]) * inv_l, __uint_as_float(o[c + 3]) * inv_l);
+          w.z = pack_bf16x2(__uint_as_float(o[c + 4]) * inv_l, __uint_as_float(o[c + 5]) * inv_l);
+          w.w = pack_bf16x2(__uint_as_float(o[c + 6]) * inv_l, __uint_as_float(o[c + 7]) * inv_l);
+          *reinterpret_cast<uint4*>(orow + c0 + c) = w;
+        }
       }
     }
-    float corr[2], ms[2];
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
-      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
-      const float mn = fmaxf(m_run[r], mx[r]);
-      ms[r] = (mn == -CUDART_INF_F) ? 0.f : mn;  // a row past the end of the prompt sees nothing
-      corr[r] = fast_exp2(m_run[r] - ms[r]);
-      m_run[r] = mn;
-    }
-    float ls[2] = {0.f, 0.f};
-    uint32_t pa[4][4];  // P as A fragments of the 4 k-steps (16 keys each)
-#pragma unroll
-    for (int nb = 0; nb < 8; ++nb) {
-      const float p0 = fast_exp2(sacc[nb][0] - ms[0]), p1 = fast_exp2(sacc[nb][1] - ms[0]);
-      const float p2 = fast_exp2(sacc[nb][2] - ms[1]), p3 = fast_exp2(sacc[nb][3] - ms[1]);
-      ls[0] += p0 + p1;
-      ls[1] += p2 + p3;
-      pa[nb >> 1][(nb & 1) * 2] = pack_bf16x2(p0, p1);      // a0 / a2: row gid
-      pa[nb >> 1][(nb & 1) * 2 + 1] = pack_bf16x2(p2, p3);  // a1 / a3: row gid + 8
-    }
-#pragma unroll
-    for (int r = 0; r < 2; ++r) l_run[r] = l_run[r] * corr[r] + ls[r];
-#pragma unroll
-    for (int db = 0; db < 16; ++db) {
-      o[db][0] *= corr[0];
-      o[db][1] *= corr[0];
-      o[db][2] *= corr[1];
-      o[db][3] *= corr[1];
-    }
-    // O += P V
-#pragma unroll
-    for (int t = 0; t < 4; ++t) {
-      const int r = 16 * t + ((lane >> 3) & 1) * 8 + (lane & 7);
-#pragma unroll
-      for (int cp = 0; cp < 8; ++cp) {
-        const int c = 2 * cp + (lane >> 4);
-        uint32_t b0, b1, b2, b3;
-        pf_ldmatrix_x4_trans(tV + r * 256 + ((c ^ (r & 7)) << 4), b0, b1, b2, b3);
-        mma_bf16_m16n8k16(o[2 * cp], pa[t][0], pa[t][1], pa[t][2], pa[t][3], b0, b1);
-        mma_bf16_m16n8k16(o[2 * cp + 1], pa[t][0], pa[t][1], pa[t][2], pa[t][3], b2, b3);
-      }
-    }
-    __syncthreads();  // the buffer is overwritten by the prefetch of the next iteration
   }
-
-#pragma unroll
-  for (int r = 0; r < 2; ++r) {
-    l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
-    l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
-  }
-#pragma unroll
-  for (int r = 0; r < 2; ++r) {
-    const int qi = qi0 + 8 * r;
-    if (qi < T) {
-      const float inv = 1.0f / l_run[r];
-      __nv_bfloat16* row = O + (size_t)qi * 128;
-#pragma unroll
-      for (int db = 0; db < 16; ++db)
-        *reinterpret_cast<uint32_t*>(row + 8 * db + 2 * tig) = pack_bf16x2(o[db][2 * r] * inv, o[db][2 * r + 1] * inv);
-    }
-  }
+  tc5::fence_before_sync();
+  __syncthreads();
+  if (warp == 4) tc5::tmem_dealloc(tmem, kPfTmemCols);
 }
 
 }  // namespace dynts
