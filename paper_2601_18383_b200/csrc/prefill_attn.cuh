@@ -9,13 +9,15 @@
 //     S  = Q K^T          M 128 x N 64 x K 128   (8 instructions of K = 16; Q and K tiles K-major)
 //     P  = exp2(S * scale - rowmax)               (online softmax: running max and sum per row)
 //     O += P V            M 128 x N 128 x K 64   (4 instructions; P K-major, V MN-major)
-// Five warps.  Warps 0-3 are the softmax warps: thread r owns query row r, i.e. lane r of tensor
+// Six warps.  Warps 0-3 are the softmax warps: thread r owns query row r, i.e. lane r of tensor
 // memory -- it reads its row of S with tcgen05.ld, keeps the row's running max and sum, rescales
 // its row of O in tensor memory when the max moves, and writes its row of P (bf16) into a
 // shared-memory tile in the 128-byte-swizzled layout the MMA's descriptor expects.  One thread of
-// warp 4 issues everything asynchronous: the TMA loads (Q once; K and V tiles into two stages each,
-// requested as soon as the product that read the stage before has completed) and the MMAs, whose
-// completion it hands to the softmax warps through mbarriers (tcgen05.commit).  S is double
+// warp 4 issues the TMA loads (Q once; K and V tiles into two stages each, requested as soon as the
+// product that read the stage before has completed), one thread of warp 5 the MMAs, whose
+// completion reaches the other warps through mbarriers (tcgen05.commit).  Each of those two threads
+// is a chain of waits and issues of a few hundred cycles apiece, which is why they are two: the
+// loads never delay a product.  S is double
 // buffered in tensor memory (columns 0-63 / 64-127; O in 128-255), so S of tile j + 1 is computed
 // while the softmax of tile j runs.  112 KB of shared memory and 256 columns of tensor memory per
 // CTA: two CTAs share an SM and fill each other's bubbles.
@@ -38,7 +40,7 @@ namespace dynts {
 
 constexpr int kPfRows = 128;                      // query rows per CTA
 constexpr int kPfKeys = 64;                       // key rows per tile
-constexpr int kPfThreads = 160;                   // 4 softmax warps + 1 warp for TMA and MMA issue
+constexpr int kPfThreads = 192;                   // 4 softmax warps, one warp whose first lane issues the TMA loads, one whose first lane issues the MMAs
 constexpr int kPfQBytes = kPfRows * 256;          // two boxes of 128 rows x 64 bf16
 constexpr int kPfKvBytes = kPfKeys * 256;         // two boxes of 64 rows x 64 bf16
 constexpr int kPfPBytes = kPfRows * 128;          // 128 rows x 64 bf16
@@ -91,7 +93,7 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
   const int n_kt = q_last / kPfKeys + 1;  // key tiles up to the diagonal
 
   if (tid == 0) {
-    for (int i = 0; i < 10; ++i) mbar_init(bar(i), i == 8 ? (kPfThreads - 32) : 1);
+    for (int i = 0; i < 10; ++i) mbar_init(bar(i), i == 8 ? kPfRows : 1);
     // (a launch whose waits run out must not take one time limit per CTA: the CTAs that start after the
     // first one gave up see the word and skip their work)
     *s_abort = *reinterpret_cast<volatile int*>(p.stop) != 0 ? 1 : 0;
@@ -114,7 +116,7 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
 
   if (warp == 4) {
     if (lane == 0) {
-      // ================= the issuing thread: TMA loads and MMAs =================
+      // ================= the loading thread: TMA tile loads =================
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmQ)) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmK)) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmV)) : "memory");
@@ -130,37 +132,67 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
         pf_tma_load(dst, &tmV, 0, j * kPfKeys, zkv, bar(3 + (j & 1)));
         pf_tma_load(dst + kPfKvBytes / 2, &tmV, 64, j * kPfKeys, zkv, bar(3 + (j & 1)));
       };
+      if (!*s_abort) {
+        mbar_arrive_expect_tx(bar(0), kPfQBytes);
+        pf_tma_load(sQ, &tmQ, 0, q0, zq, bar(0));
+        pf_tma_load(sQ + kPfQBytes / 2, &tmQ, 64, q0, zq, bar(0));
+        load_k(0);
+        load_v(0);
+        if (n_kt > 1) {
+          load_k(1);
+          load_v(1);
+        }
+      }
+      // A stage is requested again as soon as the product that read it has completed: K of tile j + 2
+      // after S_j, V of tile j + 1 after O += P V of tile j - 1.  (Neither barrier can run two phases
+      // ahead of this thread: the product that would complete the next phase needs the very tile
+      // this thread loads after the wait.)
+      for (int j = 0; j < n_kt && !*s_abort; ++j) {
+        if (j + 2 < n_kt) {
+          mbar_wait(bar(5 + (j & 1)), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);
+          if (!*s_abort) load_k(j + 2);
+        }
+        if (j >= 1 && j + 1 < n_kt) {
+          mbar_wait(bar(7), (uint32_t)((j - 1) & 1), s_abort, p.err, kPfSpinLimit);
+          if (!*s_abort) load_v(j + 1);
+        }
+      }
+      if (*s_abort) {
+        // Something gave up.  Give the tile loads this thread started a bounded time to land before the
+        // shared memory is released (every armed barrier completes its phase when its bytes are there).
+        atomicOr(p.stop, 1);
+        for (int i = 0; i < 5; ++i)
+          for (uint32_t ph = 0; ph < 2; ++ph)
+            for (uint32_t w = 0; w < (1u << 16); ++w)
+              if (mbar_try_wait(bar(i), ph)) break;
+      }
+    }
+  } else if (warp == 5) {
+    if (lane == 0) {
+      // ================= the issuing thread: MMAs =================
+      // Operand descriptors differ only in their start-address field (bits 0-13, in units of 16 bytes):
+      // one descriptor per tile is built here, the per-instruction offsets are added to its low word.
       constexpr uint32_t idesc_s = tc5::idesc_bf16_f32(kPfRows, kPfKeys, 0, 0);   // Q K^T: both K-major
       constexpr uint32_t idesc_o = tc5::idesc_bf16_f32(kPfRows, 128, 0, 1);       // P V: V is MN-major
+      const uint64_t dQ = tc5::smem_desc_sw128(sQ, 16, 1024);
+      const uint64_t dK = tc5::smem_desc_sw128(sK, 16, 1024);
+      const uint64_t dP = tc5::smem_desc_sw128(sP, 16, 1024);
+      const uint64_t dV = tc5::smem_desc_sw128(sV, kPfKvBytes / 2, 1024);
       auto mma_s = [&](int j) {  // S_j = Q K_j^T into S buffer j & 1
-        const uint32_t kb = sK + (uint32_t)(j & 1) * kPfKvBytes;
+        const uint64_t dKj = dK + (uint64_t)((uint32_t)(j & 1) * (kPfKvBytes >> 4));
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint32_t a = sQ + (uint32_t)(kk >> 2) * (kPfQBytes / 2) + (uint32_t)(kk & 3) * 32;
-          const uint32_t b = kb + (uint32_t)(kk >> 2) * (kPfKvBytes / 2) + (uint32_t)(kk & 3) * 32;
-          tc5::mma_bf16_ss(tS0 + 64u * (uint32_t)(j & 1), tc5::smem_desc_sw128(a, 16, 1024), tc5::smem_desc_sw128(b, 16, 1024), idesc_s,
-                           kk > 0);
-        }
+        for (int kk = 0; kk < 8; ++kk)  // head_dim 16 kk .. 16 kk + 15: half kk >> 2 of the tile, 32 bytes per step inside a row
+          tc5::mma_bf16_ss(tS0 + 64u * (uint32_t)(j & 1), dQ + (uint64_t)((kk >> 2) * (kPfQBytes >> 5) + (kk & 3) * 2),
+                           dKj + (uint64_t)((kk >> 2) * (kPfKvBytes >> 5) + (kk & 3) * 2), idesc_s, kk > 0);
         tc5::mma_commit(bar(5 + (j & 1)));
       };
       auto mma_o = [&](int j) {  // O += P_j V_j
-        const uint32_t vb = sV + (uint32_t)(j & 1) * kPfKvBytes;
+        const uint64_t dVj = dV + (uint64_t)((uint32_t)(j & 1) * (kPfKvBytes >> 4));
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk)  // 16 keys per step: 32 bytes along a row of P, two 8-row groups of V
-          tc5::mma_bf16_ss(tO, tc5::smem_desc_sw128(sP + (uint32_t)kk * 32, 16, 1024),
-                           tc5::smem_desc_sw128(vb + (uint32_t)kk * 2048, kPfKvBytes / 2, 1024), idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+        for (int kk = 0; kk < 4; ++kk)  // 16 keys per step: 32 bytes along a row of P, two 8-row groups (2048 bytes) of V
+          tc5::mma_bf16_ss(tO, dP + (uint64_t)(kk * 2), dVj + (uint64_t)(kk * 128), idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
         tc5::mma_commit(bar(7));
       };
-
-      mbar_arrive_expect_tx(bar(0), kPfQBytes);
-      pf_tma_load(sQ, &tmQ, 0, q0, zq, bar(0));
-      pf_tma_load(sQ + kPfQBytes / 2, &tmQ, 64, q0, zq, bar(0));
-      load_k(0);
-      load_v(0);
-      if (n_kt > 1) {
-        load_k(1);
-        load_v(1);
-      }
       mbar_wait(bar(0), 0u, s_abort, p.err, kPfSpinLimit);
       mbar_wait(bar(1), 0u, s_abort, p.err, kPfSpinLimit);
       tc5::fence_after_sync();
@@ -172,16 +204,8 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
       }
       for (int j = 0; j < n_kt && !*s_abort; ++j) {
         const int st = j & 1;
-        if (j >= 1 && j + 1 < n_kt) {  // the V stage of tile j - 1 is free once O += P V of that tile has completed
-          mbar_wait(bar(7), (uint32_t)((j - 1) & 1), s_abort, p.err, kPfSpinLimit);
-          if (!*s_abort) load_v(j + 1);
-        }
-        if (j + 2 < n_kt) {            // the K stage of tile j is free once S_j has completed
-          mbar_wait(bar(5 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);
-          if (!*s_abort) load_k(j + 2);
-        }
-        mbar_wait(bar(8), (uint32_t)(j & 1), s_abort, p.err, kPfSpinLimit);           // P_j written, O rescaled, S_j read
-        mbar_wait(bar(3 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // V_j has landed
+        mbar_wait(bar(3 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // V_j has landed (asked for long ago)
+        mbar_wait(bar(8), (uint32_t)(j & 1), s_abort, p.err, kPfSpinLimit);              // P_j written, O rescaled, S_j read
         tc5::fence_after_sync();
         if (*s_abort) break;
         mma_o(j);
@@ -192,14 +216,8 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
         }
       }
       if (*s_abort) {
+        // give the MMAs already issued a bounded time to finish before the tensor memory is released
         atomicOr(p.stop, 1);
-        // Something gave up.  Give what this thread started a bounded time to finish before the shared
-        // and tensor memory are released: the tile loads (every armed barrier completes its phase when
-        // its bytes have landed) and the MMAs (one more commit).
-        for (int i = 0; i < 5; ++i)
-          for (uint32_t s = 0; s < 2; ++s)
-            for (uint32_t w = 0; w < (1u << 16); ++w)
-              if (mbar_try_wait(bar(i), s)) break;
         tc5::mma_commit(bar(9));
         for (uint32_t w = 0; w < kPfSpinLimit; ++w)
           if (mbar_try_wait(bar(9), 0u)) break;
