@@ -8,19 +8,22 @@
 // diagonal; per tile
 //     S  = Q K^T          M 128 x N 64 x K 128   (8 instructions of K = 16; Q and K tiles K-major)
 //     P  = exp2(S * scale - rowmax)               (online softmax: running max and sum per row)
-//     O += P V            M 128 x N 128 x K 64   (4 instructions; P K-major, V MN-major)
+//     O += P V            M 128 x N 128 x K 64   (4 instructions; P from tensor memory, V MN-major)
 // Six warps.  Warps 0-3 are the softmax warps: thread r owns query row r, i.e. lane r of tensor
 // memory -- it reads its row of S with tcgen05.ld, keeps the row's running max and sum, rescales
-// its row of O in tensor memory when the max moves, and writes its row of P (bf16) into a
-// shared-memory tile in the 128-byte-swizzled layout the MMA's descriptor expects.  One thread of
+// its row of O in tensor memory when the max moves, and writes its row of P (bf16, two per column)
+// back into tensor memory over the S tile it came from, where the second product reads it as its
+// A operand: P never touches shared memory and the softmax of a tile does not wait for the product
+// of the tile before (unless the row's reference maximum has to move).  One thread of
 // warp 4 issues the TMA loads (Q once; K and V tiles into two stages each, requested as soon as the
 // product that read the stage before has completed), one thread of warp 5 the MMAs, whose
 // completion reaches the other warps through mbarriers (tcgen05.commit).  Each of those two threads
 // is a chain of waits and issues of a few hundred cycles apiece, which is why they are two: the
 // loads never delay a product.  S is double
 // buffered in tensor memory (columns 0-63 / 64-127; O in 128-255), so S of tile j + 1 is computed
-// while the softmax of tile j runs.  112 KB of shared memory and 256 columns of tensor memory per
-// CTA: two CTAs share an SM and fill each other's bubbles.
+// while the softmax of tile j runs; S of tile j + 2 overwrites the P of tile j and is issued once
+// O += P V of tile j has completed.  96 KB of shared memory
+// and 256 columns of tensor memory per CTA: two CTAs share an SM and fill each other's bubbles.
 //
 // Tiles above the diagonal are never loaded.  Rows and keys beyond the prompt come back from TMA
 // as zeros (the tensor maps are [heads][T][128], so a box never reaches into the next head) and
@@ -43,11 +46,10 @@ constexpr int kPfKeys = 64;                       // key rows per tile
 constexpr int kPfThreads = 192;                   // 4 softmax warps, one warp whose first lane issues the TMA loads, one whose first lane issues the MMAs
 constexpr int kPfQBytes = kPfRows * 256;          // two boxes of 128 rows x 64 bf16
 constexpr int kPfKvBytes = kPfKeys * 256;         // two boxes of 64 rows x 64 bf16
-constexpr int kPfPBytes = kPfRows * 128;          // 128 rows x 64 bf16
 // Two CTAs must fit the 227 KB of an SM (each also costs 1 KB of system space), so there is no room
 // for alignment slack: the dynamic shared memory is declared 1024-byte aligned (what the 128-byte
 // swizzle needs) and the kernel checks that it is.
-constexpr int kPfSmemBytes = kPfQBytes + 4 * kPfKvBytes + kPfPBytes + 128;
+constexpr int kPfSmemBytes = kPfQBytes + 4 * kPfKvBytes + 128;
 constexpr uint32_t kPfTmemCols = 256;             // S0 | S1 | O
 constexpr uint32_t kPfSpinLimit = 1u << 21;
 
@@ -74,13 +76,14 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
   const uint32_t sQ = smem_u32(sm);                       // [2 halves of head_dim][128 rows][128 B]
   const uint32_t sK = sQ + kPfQBytes;                     // [2 stages][2 halves][64 rows][128 B]
   const uint32_t sV = sK + 2 * kPfKvBytes;                // the same
-  uint8_t* sP_ptr = sm + kPfQBytes + 4 * kPfKvBytes;      // [128 rows][128 B]
-  const uint32_t sP = smem_u32(sP_ptr);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sP_ptr + kPfPBytes);
-  // barriers: 0 Q, 1-2 K stages, 3-4 V stages, 5-6 S buffers, 7 O, 8 P, 9 drain
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sm + kPfQBytes + 4 * kPfKvBytes);
+  // barriers: 0 Q, 1-2 K stages landed, 3-4 V stages landed, 5-6 S buffers complete, 7 O += P V complete, 8-9 P written
+  // (per S buffer), 10-11 V stages read, 12 the last O += P V complete, 13 drain.  Every barrier a thread waits on out of step with its producer is
+  // one per buffer or stage: a parity wait tells a phase from the one before it, not from the one two before, and
+  // with one barrier per buffer the phase after next cannot begin before the waiter has moved on.
   const uint32_t bar0 = smem_u32(bars);
   auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 10);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 14);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -93,7 +96,7 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
   const int n_kt = q_last / kPfKeys + 1;  // key tiles up to the diagonal
 
   if (tid == 0) {
-    for (int i = 0; i < 10; ++i) mbar_init(bar(i), i == 8 ? kPfRows : 1);
+    for (int i = 0; i < 14; ++i) mbar_init(bar(i), (i == 8 || i == 9) ? kPfRows : 1);
     // (a launch whose waits run out must not take one time limit per CTA: the CTAs that start after the
     // first one gave up see the word and skip their work)
     *s_abort = *reinterpret_cast<volatile int*>(p.stop) != 0 ? 1 : 0;
@@ -144,16 +147,16 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
         }
       }
       // A stage is requested again as soon as the product that read it has completed: K of tile j + 2
-      // after S_j, V of tile j + 1 after O += P V of tile j - 1.  (Neither barrier can run two phases
-      // ahead of this thread: the product that would complete the next phase needs the very tile
-      // this thread loads after the wait.)
+      // after S_j, V of tile j + 1 after O += P V of tile j - 1.  (Neither of these per-stage barriers
+      // can run two phases ahead of this thread: the product that would complete the next phase needs
+      // the very tile this thread loads after the wait.)
       for (int j = 0; j < n_kt && !*s_abort; ++j) {
         if (j + 2 < n_kt) {
           mbar_wait(bar(5 + (j & 1)), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);
           if (!*s_abort) load_k(j + 2);
         }
         if (j >= 1 && j + 1 < n_kt) {
-          mbar_wait(bar(7), (uint32_t)((j - 1) & 1), s_abort, p.err, kPfSpinLimit);
+          mbar_wait(bar(10 + ((j - 1) & 1)), (uint32_t)(((j - 1) >> 1) & 1), s_abort, p.err, kPfSpinLimit);
           if (!*s_abort) load_v(j + 1);
         }
       }
@@ -176,7 +179,6 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
       constexpr uint32_t idesc_o = tc5::idesc_bf16_f32(kPfRows, 128, 0, 1);       // P V: V is MN-major
       const uint64_t dQ = tc5::smem_desc_sw128(sQ, 16, 1024);
       const uint64_t dK = tc5::smem_desc_sw128(sK, 16, 1024);
-      const uint64_t dP = tc5::smem_desc_sw128(sP, 16, 1024);
       const uint64_t dV = tc5::smem_desc_sw128(sV, kPfKvBytes / 2, 1024);
       auto mma_s = [&](int j) {  // S_j = Q K_j^T into S buffer j & 1
         const uint64_t dKj = dK + (uint64_t)((uint32_t)(j & 1) * (kPfKvBytes >> 4));
@@ -189,9 +191,12 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
       auto mma_o = [&](int j) {  // O += P_j V_j
         const uint64_t dVj = dV + (uint64_t)((uint32_t)(j & 1) * (kPfKvBytes >> 4));
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk)  // 16 keys per step: 32 bytes along a row of P, two 8-row groups (2048 bytes) of V
-          tc5::mma_bf16_ss(tO, dP + (uint64_t)(kk * 2), dVj + (uint64_t)(kk * 128), idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+        for (int kk = 0; kk < 4; ++kk)  // 16 keys per step: 8 columns of P (over S buffer j & 1), two 8-row groups (2048 bytes) of V
+          tc5::mma_bf16_ts(tO, tS0 + 64u * (uint32_t)(j & 1) + 8u * (uint32_t)kk, dVj + (uint64_t)(kk * 128), idesc_o,
+                           (j > 0 || kk > 0) ? 1u : 0u);
         tc5::mma_commit(bar(7));
+        tc5::mma_commit(bar(10 + (j & 1)));  // the V stage of tile j may be loaded again
+        if (j == n_kt - 1) tc5::mma_commit(bar(12));  // O is final
       };
       mbar_wait(bar(0), 0u, s_abort, p.err, kPfSpinLimit);
       mbar_wait(bar(1), 0u, s_abort, p.err, kPfSpinLimit);
@@ -205,12 +210,15 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
       for (int j = 0; j < n_kt && !*s_abort; ++j) {
         const int st = j & 1;
         mbar_wait(bar(3 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // V_j has landed (asked for long ago)
-        mbar_wait(bar(8), (uint32_t)(j & 1), s_abort, p.err, kPfSpinLimit);              // P_j written, O rescaled, S_j read
+        mbar_wait(bar(8 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // P_j written, O rescaled, S_j read
         tc5::fence_after_sync();
         if (*s_abort) break;
         mma_o(j);
         if (j + 2 < n_kt) {
           mbar_wait(bar(1 + st), (uint32_t)(((j + 2) >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // K_{j+2} has landed
+          // S_{j+2} overwrites the columns P_j is read from: the product that reads them must have completed
+          // (consecutive MMAs overlap in the pipe; a write after a read of tensor memory is not ordered by issue)
+          mbar_wait(bar(7), (uint32_t)(j & 1), s_abort, p.err, kPfSpinLimit);
           tc5::fence_after_sync();
           if (!*s_abort) mma_s(j + 2);
         }
@@ -218,9 +226,9 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
       if (*s_abort) {
         // give the MMAs already issued a bounded time to finish before the tensor memory is released
         atomicOr(p.stop, 1);
-        tc5::mma_commit(bar(9));
+        tc5::mma_commit(bar(13));
         for (uint32_t w = 0; w < kPfSpinLimit; ++w)
-          if (mbar_try_wait(bar(9), 0u)) break;
+          if (mbar_try_wait(bar(13), 0u)) break;
       }
     }
   } else {
@@ -263,33 +271,30 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
       }
       l = l * alpha + sum;
       m = m_new;
-      if (j > 0) {
-        // O += P V of the tile before must be complete before O is rescaled and before P is overwritten
+      if (j > 0 && __any_sync(0xffffffffu, move)) {  // warp-uniform: the tensor-memory accesses are collective
+        // O += P V of the tile before must be complete before O is rescaled.  (That of the tile before it
+        // is: S_j was issued after it had completed.  So the parity wait cannot mistake the phases.)
         mbar_wait(bar(7), (uint32_t)((j - 1) & 1), s_abort, p.err, kPfSpinLimit);
         tc5::fence_after_sync();
-        if (__any_sync(0xffffffffu, move)) {  // warp-uniform: the tensor-memory accesses are collective
 #pragma unroll
-          for (int c0 = 0; c0 < 128; c0 += 32) {
-            uint32_t o[32];
-            tc5::tmem_ld32(tO + lane_base + (uint32_t)c0, o);
-            tc5::tmem_wait_ld();
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          uint32_t o[32];
+          tc5::tmem_ld32(tO + lane_base + (uint32_t)c0, o);
+          tc5::tmem_wait_ld();
 #pragma unroll
-            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-            tc5::tmem_st32(tO + lane_base + (uint32_t)c0, o);
-          }
-          tc5::tmem_wait_st();
+          for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+          tc5::tmem_st32(tO + lane_base + (uint32_t)c0, o);
         }
       }
-      // the row of P: 16-byte chunk c of row r goes to chunk c ^ (r & 7) of the row's 128 bytes
-#pragma unroll
-      for (int c = 0; c < 8; ++c)
-        *reinterpret_cast<uint4*>(sP_ptr + tid * 128 + ((c ^ (tid & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMA reads P through the async proxy
+      // the row of P over the first 32 columns of the S tile it was computed from (this thread has read
+      // its row of S; nothing else reads that buffer before the product that follows)
+      tc5::tmem_st32(tS0 + lane_base + 64u * (uint32_t)(j & 1), pk);
+      tc5::tmem_wait_st();
       tc5::fence_before_sync();
-      mbar_arrive(bar(8));
+      mbar_arrive(bar(8 + (j & 1)));
     }
     // epilogue: the row of O, normalised, rounded to bf16
-    mbar_wait(bar(7), (uint32_t)((n_kt - 1) & 1), s_abort, p.err, kPfSpinLimit);
+    mbar_wait(bar(12), 0u, s_abort, p.err, kPfSpinLimit);  // (a barrier of its own: it has this one phase)
     tc5::fence_after_sync();
     const float inv_l = 1.0f / l;
     __nv_bfloat16* orow = p.out + ((size_t)zq * T + (size_t)min(qpos, T - 1)) * 128;
