@@ -9,17 +9,18 @@
 //     S  = Q K^T          M 128 x N 64 x K 128   (8 instructions of K = 16; Q and K tiles K-major)
 //     P  = exp2(S * scale - rowmax)               (online softmax: running max and sum per row)
 //     O += P V            M 128 x N 128 x K 64   (4 instructions; P from tensor memory, V MN-major)
-// Six warps.  Warps 0-3 are the softmax warps: thread r owns query row r, i.e. lane r of tensor
+// Seven warps.  Warps 0-3 are the softmax warps: thread r owns query row r, i.e. lane r of tensor
 // memory -- it reads its row of S with tcgen05.ld, keeps the row's running max and sum, rescales
 // its row of O in tensor memory when the max moves, and writes its row of P (bf16, two per column)
 // back into tensor memory over the S tile it came from, where the second product reads it as its
 // A operand: P never touches shared memory and the softmax of a tile does not wait for the product
 // of the tile before (unless the row's reference maximum has to move).  One thread of
 // warp 4 issues the TMA loads (Q once; K and V tiles into two stages each, requested as soon as the
-// product that read the stage before has completed), one thread of warp 5 the MMAs, whose
-// completion reaches the other warps through mbarriers (tcgen05.commit).  Each of those two threads
-// is a chain of waits and issues of a few hundred cycles apiece, which is why they are two: the
-// loads never delay a product.  S is double
+// product that read the stage before has completed), one thread of warp 5 the second product and
+// one of warp 6 the first, whose completion reaches the other warps through mbarriers
+// (tcgen05.commit).  Each of those threads is a chain of waits and issues of a few hundred cycles
+// apiece (a wait on a completed barrier about 300, an MMA about 90), which is why they are three:
+// the chain of one never delays the others.  S is double
 // buffered in tensor memory (columns 0-63 / 64-127; O in 128-255), so S of tile j + 1 is computed
 // while the softmax of tile j runs; S of tile j + 2 overwrites the P of tile j and is issued once
 // O += P V of tile j has completed.  96 KB of shared memory
@@ -43,7 +44,7 @@ namespace dynts {
 
 constexpr int kPfRows = 128;                      // query rows per CTA
 constexpr int kPfKeys = 64;                       // key rows per tile
-constexpr int kPfThreads = 192;                   // 4 softmax warps, one warp whose first lane issues the TMA loads, one whose first lane issues the MMAs
+constexpr int kPfThreads = 224;                   // 4 softmax warps and three warps whose first lanes issue the TMA loads, O += P V, S = Q K^T
 constexpr int kPfQBytes = kPfRows * 256;          // two boxes of 128 rows x 64 bf16
 constexpr int kPfKvBytes = kPfKeys * 256;         // two boxes of 64 rows x 64 bf16
 // Two CTAs must fit the 227 KB of an SM (each also costs 1 KB of system space), so there is no room
@@ -78,12 +79,12 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
   const uint32_t sV = sK + 2 * kPfKvBytes;                // the same
   uint64_t* bars = reinterpret_cast<uint64_t*>(sm + kPfQBytes + 4 * kPfKvBytes);
   // barriers: 0 Q, 1-2 K stages landed, 3-4 V stages landed, 5-6 S buffers complete, 7 O += P V complete, 8-9 P written
-  // (per S buffer), 10-11 V stages read, 12 the last O += P V complete, 13 drain.  Every barrier a thread waits on out of step with its producer is
+  // (per S buffer), 10-11 V stages read, 12 the last O += P V complete, 13-14 drain.  Every barrier a thread waits on out of step with its producer is
   // one per buffer or stage: a parity wait tells a phase from the one before it, not from the one two before, and
   // with one barrier per buffer the phase after next cannot begin before the waiter has moved on.
   const uint32_t bar0 = smem_u32(bars);
   auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 14);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 15);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -96,7 +97,7 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
   const int n_kt = q_last / kPfKeys + 1;  // key tiles up to the diagonal
 
   if (tid == 0) {
-    for (int i = 0; i < 14; ++i) mbar_init(bar(i), (i == 8 || i == 9) ? kPfRows : 1);
+    for (int i = 0; i < 15; ++i) mbar_init(bar(i), (i == 8 || i == 9) ? kPfRows : 1);
     // (a launch whose waits run out must not take one time limit per CTA: the CTAs that start after the
     // first one gave up see the word and skip their work)
     *s_abort = *reinterpret_cast<volatile int*>(p.stop) != 0 ? 1 : 0;
@@ -172,31 +173,47 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
     }
   } else if (warp == 5) {
     if (lane == 0) {
-      // ================= the issuing thread: MMAs =================
+      // ================= the thread that issues O += P V =================
       // Operand descriptors differ only in their start-address field (bits 0-13, in units of 16 bytes):
-      // one descriptor per tile is built here, the per-instruction offsets are added to its low word.
-      constexpr uint32_t idesc_s = tc5::idesc_bf16_f32(kPfRows, kPfKeys, 0, 0);   // Q K^T: both K-major
+      // one descriptor per tensor is built here, the per-instruction offsets are added to its low word.
       constexpr uint32_t idesc_o = tc5::idesc_bf16_f32(kPfRows, 128, 0, 1);       // P V: V is MN-major
+      const uint64_t dV = tc5::smem_desc_sw128(sV, kPfKvBytes / 2, 1024);
+      for (int j = 0; j < n_kt && !*s_abort; ++j) {
+        const int st = j & 1;
+        mbar_wait(bar(3 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // V_j has landed (asked for long ago)
+        mbar_wait(bar(8 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // P_j written, O rescaled, S_j read
+        tc5::fence_after_sync();
+        if (*s_abort) break;
+        const uint64_t dVj = dV + (uint64_t)((uint32_t)st * (kPfKvBytes >> 4));
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)  // 16 keys per step: 8 columns of P (over S buffer j & 1), two 8-row groups (2048 bytes) of V
+          tc5::mma_bf16_ts(tO, tS0 + 64u * (uint32_t)st + 8u * (uint32_t)kk, dVj + (uint64_t)(kk * 128), idesc_o,
+                           (j > 0 || kk > 0) ? 1u : 0u);
+        tc5::mma_commit(bar(7));
+        tc5::mma_commit(bar(10 + st));  // P_j and the V stage of tile j have been read
+        if (j == n_kt - 1) tc5::mma_commit(bar(12));  // O is final
+      }
+      if (*s_abort) {
+        // give the MMAs already issued a bounded time to finish before the tensor memory is released
+        atomicOr(p.stop, 1);
+        tc5::mma_commit(bar(13));
+        for (uint32_t w = 0; w < kPfSpinLimit; ++w)
+          if (mbar_try_wait(bar(13), 0u)) break;
+      }
+    }
+  } else if (warp == 6) {
+    if (lane == 0) {
+      // ================= the thread that issues S = Q K^T =================
+      constexpr uint32_t idesc_s = tc5::idesc_bf16_f32(kPfRows, kPfKeys, 0, 0);   // both operands K-major
       const uint64_t dQ = tc5::smem_desc_sw128(sQ, 16, 1024);
       const uint64_t dK = tc5::smem_desc_sw128(sK, 16, 1024);
-      const uint64_t dV = tc5::smem_desc_sw128(sV, kPfKvBytes / 2, 1024);
-      auto mma_s = [&](int j) {  // S_j = Q K_j^T into S buffer j & 1
+      auto mma_s = [&](int j) {  // S_j into S buffer j & 1
         const uint64_t dKj = dK + (uint64_t)((uint32_t)(j & 1) * (kPfKvBytes >> 4));
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)  // head_dim 16 kk .. 16 kk + 15: half kk >> 2 of the tile, 32 bytes per step inside a row
           tc5::mma_bf16_ss(tS0 + 64u * (uint32_t)(j & 1), dQ + (uint64_t)((kk >> 2) * (kPfQBytes >> 5) + (kk & 3) * 2),
                            dKj + (uint64_t)((kk >> 2) * (kPfKvBytes >> 5) + (kk & 3) * 2), idesc_s, kk > 0);
         tc5::mma_commit(bar(5 + (j & 1)));
-      };
-      auto mma_o = [&](int j) {  // O += P_j V_j
-        const uint64_t dVj = dV + (uint64_t)((uint32_t)(j & 1) * (kPfKvBytes >> 4));
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk)  // 16 keys per step: 8 columns of P (over S buffer j & 1), two 8-row groups (2048 bytes) of V
-          tc5::mma_bf16_ts(tO, tS0 + 64u * (uint32_t)(j & 1) + 8u * (uint32_t)kk, dVj + (uint64_t)(kk * 128), idesc_o,
-                           (j > 0 || kk > 0) ? 1u : 0u);
-        tc5::mma_commit(bar(7));
-        tc5::mma_commit(bar(10 + (j & 1)));  // the V stage of tile j may be loaded again
-        if (j == n_kt - 1) tc5::mma_commit(bar(12));  // O is final
       };
       mbar_wait(bar(0), 0u, s_abort, p.err, kPfSpinLimit);
       mbar_wait(bar(1), 0u, s_abort, p.err, kPfSpinLimit);
@@ -207,28 +224,21 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
         tc5::fence_after_sync();
         if (!*s_abort) mma_s(1);
       }
-      for (int j = 0; j < n_kt && !*s_abort; ++j) {
+      for (int j = 0; j + 2 < n_kt && !*s_abort; ++j) {
         const int st = j & 1;
-        mbar_wait(bar(3 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // V_j has landed (asked for long ago)
-        mbar_wait(bar(8 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // P_j written, O rescaled, S_j read
+        // S_{j+2} overwrites the columns P_j is read from, so O += P V of tile j must have completed (the
+        // two products come from different threads and nothing but this barrier orders them); and its K
+        // tile must have landed.
+        mbar_wait(bar(10 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);
+        mbar_wait(bar(1 + st), (uint32_t)(((j + 2) >> 1) & 1), s_abort, p.err, kPfSpinLimit);
         tc5::fence_after_sync();
-        if (*s_abort) break;
-        mma_o(j);
-        if (j + 2 < n_kt) {
-          mbar_wait(bar(1 + st), (uint32_t)(((j + 2) >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // K_{j+2} has landed
-          // S_{j+2} overwrites the columns P_j is read from: the product that reads them must have completed
-          // (consecutive MMAs overlap in the pipe; a write after a read of tensor memory is not ordered by issue)
-          mbar_wait(bar(7), (uint32_t)(j & 1), s_abort, p.err, kPfSpinLimit);
-          tc5::fence_after_sync();
-          if (!*s_abort) mma_s(j + 2);
-        }
+        if (!*s_abort) mma_s(j + 2);
       }
       if (*s_abort) {
-        // give the MMAs already issued a bounded time to finish before the tensor memory is released
         atomicOr(p.stop, 1);
-        tc5::mma_commit(bar(13));
+        tc5::mma_commit(bar(14));
         for (uint32_t w = 0; w < kPfSpinLimit; ++w)
-          if (mbar_try_wait(bar(13), 0u)) break;
+          if (mbar_try_wait(bar(14), 0u)) break;
       }
     }
   } else {
