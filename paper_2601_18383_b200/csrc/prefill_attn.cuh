@@ -229,8 +229,8 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
         // S_{j+2} overwrites the columns P_j is read from, so O += P V of tile j must have completed (the
         // two products come from different threads and nothing but this barrier orders them); and its K
         // tile must have landed.
+        mbar_wait(bar(1 + st), (uint32_t)(((j + 2) >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // (lands first: asked for when S_j completed)
         mbar_wait(bar(10 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);
-        mbar_wait(bar(1 + st), (uint32_t)(((j + 2) >> 1) & 1), s_abort, p.err, kPfSpinLimit);
         tc5::fence_after_sync();
         if (!*s_abort) mma_s(j + 2);
       }
@@ -254,31 +254,43 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
       tc5::tmem_ld32(tS0 + lane_base + 64u * (uint32_t)(j & 1) + 32u, s_hi);
       tc5::tmem_wait_ld();
       const int key0 = j * kPfKeys;
-      float mx = -CUDART_INF_F;
+      // Only the tiles that reach the diagonal need the mask (uniform over the CTA); the rest of the
+      // row arithmetic works on the raw products: the scale is positive, so the maximum can be taken
+      // before it is applied, and it is folded into the exponent's multiply-add.
+      if (key0 + kPfKeys - 1 > q0) {
 #pragma unroll
-      for (int c = 0; c < 32; ++c) {
-        const float a = (key0 + c <= qpos) ? __uint_as_float(s_lo[c]) * p.scale_log2 : -CUDART_INF_F;
-        const float b = (key0 + 32 + c <= qpos) ? __uint_as_float(s_hi[c]) * p.scale_log2 : -CUDART_INF_F;
-        s_lo[c] = __float_as_uint(a);
-        s_hi[c] = __float_as_uint(b);
-        mx = fmaxf(mx, fmaxf(a, b));
+        for (int c = 0; c < 32; ++c) {
+          if (key0 + c > qpos) s_lo[c] = 0xff800000u;       // -inf
+          if (key0 + 32 + c > qpos) s_hi[c] = 0xff800000u;
+        }
       }
+      float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+#pragma unroll
+      for (int c = 0; c < 32; c += 4) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) mx4[u] = fmaxf(mx4[u], fmaxf(__uint_as_float(s_lo[c + u]), __uint_as_float(s_hi[c + u])));
+      }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
       // The reference maximum m of a row only has to keep exp2(x - m) in range, not to equal the true
       // maximum: it is moved (and O and l rescaled) only when the tile's maximum exceeds it by more
       // than 2^8, so P stays below 256 (bf16 and fp32 have the range) and most tiles rescale nothing.
       const bool move = mx > m + 8.0f;       // always at the first tile (m = -inf; key 0 is visible to every row)
       const float m_new = move ? mx : m;
       const float alpha = move ? fast_exp2(m - m_new) : 1.0f;  // 0 at the first tile, where l and O are empty
-      float sum = 0.f;
+      const float neg_m = -m_new;
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t pk[32];  // the row's 64 weights as bf16 pairs
 #pragma unroll
       for (int c = 0; c < 16; ++c) {
-        const float a0 = fast_exp2(__uint_as_float(s_lo[2 * c]) - m_new), a1 = fast_exp2(__uint_as_float(s_lo[2 * c + 1]) - m_new);
-        const float b0 = fast_exp2(__uint_as_float(s_hi[2 * c]) - m_new), b1 = fast_exp2(__uint_as_float(s_hi[2 * c + 1]) - m_new);
-        sum += (a0 + a1) + (b0 + b1);
+        const float a0 = fast_exp2(fmaf(__uint_as_float(s_lo[2 * c]), p.scale_log2, neg_m));
+        const float a1 = fast_exp2(fmaf(__uint_as_float(s_lo[2 * c + 1]), p.scale_log2, neg_m));
+        const float b0 = fast_exp2(fmaf(__uint_as_float(s_hi[2 * c]), p.scale_log2, neg_m));
+        const float b1 = fast_exp2(fmaf(__uint_as_float(s_hi[2 * c + 1]), p.scale_log2, neg_m));
+        sum4[c & 3] += (a0 + a1) + (b0 + b1);
         pk[c] = pack_bf16x2(a0, a1);
         pk[16 + c] = pack_bf16x2(b0, b1);
       }
+      const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
       l = l * alpha + sum;
       m = m_new;
       if (j > 0 && __any_sync(0xffffffffu, move)) {  // warp-uniform: the tensor-memory accesses are collective
