@@ -115,6 +115,13 @@ dynts_status_t dynts_prefill_attn(dynts_cache_t* c, const void* q, const void* k
  * writes out, leaves the cache untouched.  Same shapes and restrictions. */
 dynts_status_t dynts_prompt_attn(dynts_cache_t* c, const void* q, const void* k, const void* v, void* out, int n_tokens);
 
+/* dynts_prefill_attn one layer at a time, for a model whose layer l + 1 prompt activations depend on
+ * layer l's attention output: q, out: device [Nb, Hq, n_tokens, d]; k, v: device [Nb, Hkv, n_tokens, d].
+ * Stores the layer's rows and computes its prompt attention.  Call for layers 0 .. L-1 in order with
+ * the same n_tokens and n_pinned; the sequences' lengths are set with the last layer. */
+dynts_status_t dynts_prefill_attn_layer(dynts_cache_t* c, int layer, const void* q, const void* k, const void* v, void* out,
+                                        int n_tokens, int n_pinned);
+
 /* The same for one sequence of a ragged batch; k, v: device [L, Hkv, n_tokens, d].  Marks the
  * sequence active. */
 dynts_status_t dynts_prefill_seq(dynts_cache_t* c, int seq, const void* k, const void* v, int n_tokens, int n_pinned);
@@ -262,6 +269,12 @@ dynts_status_t dynts_predictor_mlp(const void* h, const void* W1, const float* b
 
 /* Ragged batches: mark a sequence finished (length 0, inactive) until its next prefill_seq. */
 dynts_status_t dynts_seq_reset(dynts_cache_t* c, int seq);
+
+/* Re-reads the per-sequence lengths from the device into the host copy (synchronises the stream).
+ * Needed after replays of a captured graph that changed the lengths (decode steps advance them on
+ * the device only), before the next direct call that depends on them (an eviction, a decode step
+ * outside a graph). */
+dynts_status_t dynts_cache_refresh_lengths(dynts_cache_t* c);
 
 /* Host mirror of a sequence's cache length (no synchronisation); -1 on a bad argument. */
 int dynts_cache_len(const dynts_cache_t* c, int seq);

@@ -68,6 +68,8 @@ _sigs = {
     "dynts_prefill": (C.c_int, [_P, _P, _P, C.c_int, C.c_int]),
     "dynts_prefill_attn": (C.c_int, [_P, _P, _P, _P, _P, C.c_int, C.c_int]),
     "dynts_prompt_attn": (C.c_int, [_P, _P, _P, _P, _P, C.c_int]),
+    "dynts_prefill_attn_layer": (C.c_int, [_P, C.c_int, _P, _P, _P, _P, C.c_int, C.c_int]),
+    "dynts_cache_refresh_lengths": (C.c_int, [_P]),
     "dynts_prefill_seq": (C.c_int, [_P, C.c_int, _P, _P, C.c_int, C.c_int]),
     "dynts_decode_attn": (C.c_int, [_P, _P, _P, _P, _P, _P]),
     "dynts_decode_attn_layer": (C.c_int, [_P, C.c_int, _P, _P, _P, _P, _P]),
@@ -183,6 +185,14 @@ def dynts_prefill(c, k, v, n_tokens, n_pinned):
 
 def dynts_prefill_attn(c, q, k, v, out, n_tokens, n_pinned):
     return _check(lib.dynts_prefill_attn(c, _ptr(q), _ptr(k), _ptr(v), _ptr(out), n_tokens, n_pinned))
+
+
+def dynts_prefill_attn_layer(c, layer, q, k, v, out, n_tokens, n_pinned):
+    return _check(lib.dynts_prefill_attn_layer(c, layer, _ptr(q), _ptr(k), _ptr(v), _ptr(out), n_tokens, n_pinned))
+
+
+def dynts_cache_refresh_lengths(c):
+    return _check(lib.dynts_cache_refresh_lengths(c))
 
 
 def dynts_prompt_attn(c, q, k, v, out, n_tokens):
@@ -368,6 +378,13 @@ class Cache:
     def prefill_attn(self, q, k, v, out, n_pinned=None):
         T = k.shape[-2]
         return dynts_prefill_attn(self.handle, q, k, v, out, T, T if n_pinned is None else n_pinned)
+
+    def prefill_attn_layer(self, layer, q, k, v, out, n_pinned=None):
+        T = k.shape[-2]
+        return dynts_prefill_attn_layer(self.handle, layer, q, k, v, out, T, T if n_pinned is None else n_pinned)
+
+    def refresh_lengths(self):
+        return dynts_cache_refresh_lengths(self.handle)
 
     def prompt_attn(self, q, k, v, out):
         return dynts_prompt_attn(self.handle, q, k, v, out, k.shape[-2])

@@ -537,7 +537,9 @@ dynts_status_t check_decode_args(const dynts_cache* c, const void* q, const void
   return DYNTS_OK;
 }
 
-dynts_status_t do_prefill(dynts_cache* c, int seq, const void* k, const void* v, int T, int n_pinned) {
+// layer < 0: all layers (k, v hold L layers); else that one layer (k, v hold one), the lengths being
+// published with the last layer.
+dynts_status_t do_prefill(dynts_cache* c, int seq, const void* k, const void* v, int T, int n_pinned, int layer = -1) {
   if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
   dynts_status_t st = materialise(c);
   if (st != DYNTS_OK) return st;
@@ -575,13 +577,17 @@ dynts_status_t do_prefill(dynts_cache* c, int seq, const void* k, const void* v,
   p.T = T;
   p.n_pinned = n_pinned;
   p.seq = seq;
-  const unsigned ny = (unsigned)(seq < 0 ? c->slabs() : (size_t)c->cfg.layers * c->cfg.kv_heads);
+  const int n_layers = layer < 0 ? c->cfg.layers : 1;
+  const bool publish = layer < 0 || layer == c->cfg.layers - 1;
+  p.layer0 = layer < 0 ? 0 : layer;
+  p.set_len = publish ? 1 : 0;
+  const unsigned ny = (unsigned)((size_t)n_layers * (seq < 0 ? c->cfg.batch : 1) * c->cfg.kv_heads);
   const size_t pieces = (size_t)T * c->cfg.head_dim * c->elt / 16;  // 16-byte pieces of the source
   const unsigned nx = (unsigned)std::max<size_t>(1, std::min<size_t>(64, (pieces + 255) / 256));
   dynts::prefill_kernel<<<dim3(nx, ny, 1), 256, 0, c->stream>>>(p);
   CUDA_TRY(cudaGetLastError());
   c->launches += 1;
-  for (int b = 0; b < c->cfg.batch; ++b) {
+  for (int b = 0; b < c->cfg.batch && publish; ++b) {
     if (seq >= 0 && b != seq) continue;
     c->len_h[b] = T;
     c->tot_h[b] = T;
@@ -815,7 +821,11 @@ dynts_status_t dynts_prefill(dynts_cache_t* c, const void* k, const void* v, int
   return do_prefill(c, -1, k, v, n_tokens, n_pinned);
 }
 
-dynts_status_t dynts_prompt_attn(dynts_cache_t* c, const void* q, const void* k, const void* v, void* out, int n_tokens) {
+}  // extern "C"
+
+namespace {
+
+dynts_status_t prompt_attn(dynts_cache* c, const void* q, const void* k, const void* v, void* out, int n_tokens, int n_layers) {
   if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
   if (!q || !out || !k || !v || !aligned16(q) || !aligned16(out) || !aligned16(k) || !aligned16(v))
     return fail(DYNTS_ERR_INVALID_ARG, "q, k, v and out must be non-NULL and 16-byte aligned");
@@ -824,7 +834,7 @@ dynts_status_t dynts_prompt_attn(dynts_cache_t* c, const void* q, const void* k,
   if (n_tokens < 1) return fail(DYNTS_ERR_INVALID_ARG, "n_tokens must be positive");
   dynts_status_t st = materialise(c);
   if (st != DYNTS_OK) return st;
-  const long long lb = (long long)c->cfg.layers * c->cfg.batch;
+  const long long lb = (long long)n_layers * c->cfg.batch;
   if (lb > 65535 || (long long)n_tokens * 256 >= (1ll << 40))
     return fail(DYNTS_ERR_INVALID_ARG, "layers x batch %lld or n_tokens %d beyond the launch limits", lb, n_tokens);
   if (!c->attr_prefill) {
@@ -864,6 +874,40 @@ dynts_status_t dynts_prompt_attn(dynts_cache_t* c, const void* q, const void* k,
   dynts::prefill_attn_kernel<<<grid, dynts::kPfThreads, dynts::kPfSmemBytes, c->stream>>>(p, mq, mk, mv);
   CUDA_TRY(cudaGetLastError());
   c->launches += 1;
+  return DYNTS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+dynts_status_t dynts_prompt_attn(dynts_cache_t* c, const void* q, const void* k, const void* v, void* out, int n_tokens) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  return prompt_attn(c, q, k, v, out, n_tokens, c->cfg.layers);
+}
+
+dynts_status_t dynts_prefill_attn_layer(dynts_cache_t* c, int layer, const void* q, const void* k, const void* v, void* out,
+                                        int n_tokens, int n_pinned) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (layer < 0 || layer >= c->cfg.layers) return fail(DYNTS_ERR_INVALID_ARG, "layer %d out of range", layer);
+  if (!q || !out || !aligned16(q) || !aligned16(out))
+    return fail(DYNTS_ERR_INVALID_ARG, "q and out must be non-NULL and 16-byte aligned");
+  if ((c->cfg.dtype != DYNTS_BF16 && c->cfg.dtype != DYNTS_BF16_KV8) || c->cfg.head_dim != 128)
+    return fail(DYNTS_ERR_INVALID_ARG, "prefill attention needs bf16 q/k/v and head_dim 128");
+  if (n_tokens < 1) return fail(DYNTS_ERR_INVALID_ARG, "n_tokens must be positive");
+  dynts_status_t st = do_prefill(c, -1, k, v, n_tokens, n_pinned, layer);  // this layer's rows; lengths with the last layer
+  if (st != DYNTS_OK) return st;
+  return prompt_attn(c, q, k, v, out, n_tokens, 1);
+}
+
+dynts_status_t dynts_cache_refresh_lengths(dynts_cache_t* c) {
+  if (!c) return fail(DYNTS_ERR_INVALID_ARG, "NULL cache");
+  if (!c->ready) return DYNTS_OK;
+  if (c->layer_cursor != 0) return fail(DYNTS_ERR_STATE, "a layer-by-layer step is in progress");
+  CUDA_TRY(cudaStreamSynchronize(c->stream));
+  const int Nb = c->cfg.batch;
+  CUDA_TRY(cudaMemcpy(c->len_h.data(), c->len(), Nb * sizeof(int), cudaMemcpyDeviceToHost));
+  CUDA_TRY(cudaMemcpy(c->tot_h.data(), c->tot(), Nb * sizeof(int), cudaMemcpyDeviceToHost));
   return DYNTS_OK;
 }
 

@@ -926,6 +926,8 @@ struct PrefillParams {
   int* pinned;
   int* active;
   int L, Nb, Hkv, d, cap, elt_bytes, T, n_pinned, seq;
+  int layer0;              // the source tensors hold the layers layer0 .. (as many as the grid covers)
+  int set_len;             // 1: this launch also publishes length, position counter, pins and the active flag
   int kv8;                 // 1: k, v are bf16 and the slabs take their E4M3 codes (elt_bytes = 1)
   float k_scale, v_scale;
 };
@@ -936,10 +938,10 @@ __global__ void __launch_bounds__(256) prefill_kernel(const PrefillParams p) {
   if (p.seq < 0) {
     h = sl % p.Hkv;
     b = (sl / p.Hkv) % p.Nb;
-    l = sl / (p.Hkv * p.Nb);
+    l = p.layer0 + sl / (p.Hkv * p.Nb);
   } else {
     h = sl % p.Hkv;
-    l = sl / p.Hkv;
+    l = p.layer0 + sl / p.Hkv;
     b = p.seq;
   }
   const size_t slab = ((size_t)l * p.Nb + b) * p.Hkv + h;
@@ -979,7 +981,7 @@ __global__ void __launch_bounds__(256) prefill_kernel(const PrefillParams p) {
     p.score[slab * p.cap + t] = t < p.n_pinned ? __int_as_float(0x7f800000) : 0.f;
     p.comp[slab * p.cap + t] = 0.f;
   }
-  if (blockIdx.x == 0 && threadIdx.x == 0 && l == 0 && h == 0) {
+  if (p.set_len && blockIdx.x == 0 && threadIdx.x == 0 && l == p.layer0 && h == 0) {
     p.len[b] = p.T;
     p.tot[b] = p.T;
     p.pinned[b] = p.n_pinned;

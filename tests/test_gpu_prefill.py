@@ -101,3 +101,62 @@ def test_prefill_attention_into_a_cache_of_8_bit_rows():
         assert np.array_equal(Vc.numpy(), O.fp8_e4m3_encode(v[l, 0, h] / np.float32(vs)))
         assert np.array_equal(pos.numpy(), np.arange(T)) and np.isinf(score.numpy()).all()
     a.close(); b.close()
+
+
+def test_prefill_attention_layer_by_layer_equals_the_all_layers_call():
+    """dynts_prefill_attn_layer for layers 0..L-1 leaves the same outputs and the same cache as one
+    dynts_prefill_attn over all layers; the lengths appear with the last layer."""
+    T = 150
+    cfg = W.get_config("c2_llama8b").scaled(layers=3, batch=2, kv_heads=2, q_heads=8, prompt=T, budget=256, window=8,
+                                             evict_interval=16)
+    q, k, v = _qkv(cfg, T, 93)
+    a, b = H.make_gpu(cfg), H.make_gpu(cfg)
+    qd, kd, vd = H.dev(q, cfg), H.dev(k, cfg), H.dev(v, cfg)
+    oa = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, T, 128), dtype=torch.bfloat16, device="cuda:0")
+    ob = torch.full_like(oa, float("nan"))
+    a.prefill_attn(qd, kd, vd, oa, n_pinned=100)
+    for l in range(cfg.layers):
+        assert b.len(0) == 0
+        b.prefill_attn_layer(l, qd[l], kd[l], vd[l], ob[l], n_pinned=100)
+    assert b.len(0) == T == b.len(1)
+    torch.cuda.synchronize()
+    a.poll_error(); b.poll_error()
+    assert torch.equal(oa.view(torch.int16), ob.view(torch.int16))
+    for sl in [(0, 0, 0), (1, 1, 1), (2, 0, 1)]:
+        Ka, Va, pa, sa = a.export_slab(*sl)
+        Kb, Vb, pb, sb = b.export_slab(*sl)
+        assert torch.equal(H.bits(Ka), H.bits(Kb)) and torch.equal(H.bits(Va), H.bits(Vb))
+        assert torch.equal(pa, pb) and torch.equal(H.bits(sa), H.bits(sb))
+        assert np.isinf(sa.numpy()[:100]).all() and (sa.numpy()[100:] == 0).all()
+    a.close(); b.close()
+
+
+def test_lengths_are_refreshed_after_graph_replays():
+    """A captured decode step advances the lengths on the device only; dynts_cache_refresh_lengths
+    brings the host copy up to date, after which a direct eviction sees the rows."""
+    from workloads import gen
+    cfg = W.get_config("c2_llama8b").scaled(layers=2, batch=2, prompt=32, budget=128, window=16, evict_interval=32)
+    gpu = H.make_gpu(cfg)
+    k, v = gen.torch_keys_values(cfg, 94, 100, "cuda:0")
+    gpu.prefill(k, v, n_pinned=cfg.prompt)
+    q, kn, vn = [x[0] for x in gen.torch_step_ring(cfg, 94, 1, "cuda:0")]
+    out = torch.empty((cfg.layers, cfg.batch, cfg.q_heads, 128), dtype=torch.bfloat16, device="cuda:0")
+    gpu.decode_attn(q, kn, vn, out)                    # eager warm-up: 101 rows
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        gpu.set_stream(side)
+        with torch.cuda.graph(graph, stream=side):
+            gpu.decode_attn(q, kn, vn, out)            # captured, not run: the host copy says 102 afterwards
+    gpu.set_stream(torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    for _ in range(40):
+        graph.replay()
+    gpu.refresh_lengths()
+    assert gpu.len(0) == 141 == gpu.len(1)
+    gpu.poll_error()
+    H.check_evict_bit_exact(gpu, cfg, 0)
+    assert gpu.len(0) == cfg.budget
+    gpu.close()
