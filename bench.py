@@ -630,6 +630,8 @@ def main():
     ap.add_argument("--sustain-seconds", type=float, default=2.0,
                     help="length of the sustained region that follows the K timed steps (0: skip it)")
     ap.add_argument("--no-extras", action="store_true", help="skip the predictor-head and prefill-attention timings")
+    ap.add_argument("--extras-only", action="store_true",
+                    help="time only the predictor head and the prefill attention of the workload (a short run, e.g. to profile them)")
     ap.add_argument("--score-source", default="attention", choices=["attention", "external"],
                     help="attention: Eq. 6 mass accumulated online (default); external: one predictor score per token (Eq. 7)")
     ap.add_argument("--selection", default="slab", choices=["slab", "global"],
@@ -667,7 +669,12 @@ def main():
             _orig(self, *a, **kw)
             self.set_launch(args.cluster, args.variant)
         D.Cache.__init__ = _init
-    res = run_ours(args, cfg, rank, world, device)
+    if args.extras_only:
+        peak, _ = measured_peaks()
+        res = {"config": workload_config(cfg, args, world), "predictor_mlp": time_predictor(cfg.batch, device, peak),
+               "prefill_attn": time_prefill(cfg, device) if cfg.dtype == "bf16" and cfg.head_dim == 128 else None}
+    else:
+        res = run_ours(args, cfg, rank, world, device)
     if rank == 0:
         print(json.dumps(res), flush=True)
     if world > 1:

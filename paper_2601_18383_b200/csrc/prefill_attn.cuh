@@ -44,7 +44,7 @@ namespace dynts {
 
 constexpr int kPfRows = 128;                      // query rows per CTA
 constexpr int kPfKeys = 64;                       // key rows per tile
-constexpr int kPfThreads = 224;                   // 4 softmax warps and three warps whose first lanes issue the TMA loads, O += P V, S = Q K^T
+constexpr int kPfThreads = 224;                   // 4 softmax warps, one warp whose first lane issues the TMA loads, one warp each for O += P V and S = Q K^T
 constexpr int kPfQBytes = kPfRows * 256;          // two boxes of 128 rows x 64 bf16
 constexpr int kPfKvBytes = kPfKeys * 256;         // two boxes of 64 rows x 64 bf16
 // Two CTAs must fit the 227 KB of an SM (each also costs 1 KB of system space), so there is no room
@@ -172,19 +172,24 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
       }
     }
   } else if (warp == 5) {
-    if (lane == 0) {
-      // ================= the thread that issues O += P V =================
-      // Operand descriptors differ only in their start-address field (bits 0-13, in units of 16 bytes):
-      // one descriptor per tensor is built here, the per-instruction offsets are added to its low word.
-      constexpr uint32_t idesc_o = tc5::idesc_bf16_f32(kPfRows, 128, 0, 1);       // P V: V is MN-major
-      const uint64_t dV = tc5::smem_desc_sw128(sV, kPfKvBytes / 2, 1024);
-      for (int j = 0; j < n_kt && !*s_abort; ++j) {
-        const int st = j & 1;
-        mbar_wait(bar(3 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // V_j has landed (asked for long ago)
-        mbar_wait(bar(8 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // P_j written, O rescaled, S_j read
-        tc5::fence_after_sync();
-        if (*s_abort) break;
-        const uint64_t dVj = dV + (uint64_t)((uint32_t)st * (kPfKvBytes >> 4));
+    // ================= the warp that issues O += P V =================
+    // The whole warp runs the loop and polls the barriers (a warp of pollers notices a completed phase
+    // sooner than one lane: 492 -> 468 us on config 3's prompt); one elected lane issues.  (Issued from code that only
+    // one lane runs, an MMA cost about twice as long: its descriptors then live in ordinary registers
+    // and have to be moved to uniform ones one by one.)
+    // Operand descriptors differ only in their start-address field (bits 0-13, in units of 16 bytes):
+    // one descriptor per tensor is built here, the per-instruction offsets are added to its low word.
+    constexpr uint32_t idesc_o = tc5::idesc_bf16_f32(kPfRows, 128, 0, 1);       // P V: V is MN-major
+    const uint64_t dV = tc5::smem_desc_sw128(sV, kPfKvBytes / 2, 1024);
+    for (int j = 0; j < n_kt && !*s_abort; ++j) {
+      const int st = j & 1;
+      mbar_wait(bar(3 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // V_j has landed (asked for long ago)
+      mbar_wait(bar(8 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // P_j written, O rescaled, S_j read
+      __syncwarp();
+      tc5::fence_after_sync();
+      if (*s_abort) break;
+      const uint64_t dVj = dV + (uint64_t)((uint32_t)st * (kPfKvBytes >> 4));
+      if (tc5::elect_one()) {
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk)  // 16 keys per step: 8 columns of P (over S buffer j & 1), two 8-row groups (2048 bytes) of V
           tc5::mma_bf16_ts(tO, tS0 + 64u * (uint32_t)st + 8u * (uint32_t)kk, dVj + (uint64_t)(kk * 128), idesc_o,
@@ -193,53 +198,58 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
         tc5::mma_commit(bar(10 + st));  // P_j and the V stage of tile j have been read
         if (j == n_kt - 1) tc5::mma_commit(bar(12));  // O is final
       }
-      if (*s_abort) {
-        // give the MMAs already issued a bounded time to finish before the tensor memory is released
-        atomicOr(p.stop, 1);
-        tc5::mma_commit(bar(13));
-        for (uint32_t w = 0; w < kPfSpinLimit; ++w)
-          if (mbar_try_wait(bar(13), 0u)) break;
-      }
+      __syncwarp();
+    }
+    if (*s_abort && tc5::elect_one()) {
+      // give the MMAs already issued a bounded time to finish before the tensor memory is released
+      atomicOr(p.stop, 1);
+      tc5::mma_commit(bar(13));
+      for (uint32_t w = 0; w < kPfSpinLimit; ++w)
+        if (mbar_try_wait(bar(13), 0u)) break;
     }
   } else if (warp == 6) {
-    if (lane == 0) {
-      // ================= the thread that issues S = Q K^T =================
-      constexpr uint32_t idesc_s = tc5::idesc_bf16_f32(kPfRows, kPfKeys, 0, 0);   // both operands K-major
-      const uint64_t dQ = tc5::smem_desc_sw128(sQ, 16, 1024);
-      const uint64_t dK = tc5::smem_desc_sw128(sK, 16, 1024);
-      auto mma_s = [&](int j) {  // S_j into S buffer j & 1
-        const uint64_t dKj = dK + (uint64_t)((uint32_t)(j & 1) * (kPfKvBytes >> 4));
+    // ================= the warp that issues S = Q K^T =================
+    constexpr uint32_t idesc_s = tc5::idesc_bf16_f32(kPfRows, kPfKeys, 0, 0);   // both operands K-major
+    const uint64_t dQ = tc5::smem_desc_sw128(sQ, 16, 1024);
+    const uint64_t dK = tc5::smem_desc_sw128(sK, 16, 1024);
+    auto mma_s = [&](int j) {  // S_j into S buffer j & 1
+      const uint64_t dKj = dK + (uint64_t)((uint32_t)(j & 1) * (kPfKvBytes >> 4));
+      if (tc5::elect_one()) {
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)  // head_dim 16 kk .. 16 kk + 15: half kk >> 2 of the tile, 32 bytes per step inside a row
           tc5::mma_bf16_ss(tS0 + 64u * (uint32_t)(j & 1), dQ + (uint64_t)((kk >> 2) * (kPfQBytes >> 5) + (kk & 3) * 2),
                            dKj + (uint64_t)((kk >> 2) * (kPfKvBytes >> 5) + (kk & 3) * 2), idesc_s, kk > 0);
         tc5::mma_commit(bar(5 + (j & 1)));
-      };
-      mbar_wait(bar(0), 0u, s_abort, p.err, kPfSpinLimit);
-      mbar_wait(bar(1), 0u, s_abort, p.err, kPfSpinLimit);
+      }
+      __syncwarp();
+    };
+    mbar_wait(bar(0), 0u, s_abort, p.err, kPfSpinLimit);
+    mbar_wait(bar(1), 0u, s_abort, p.err, kPfSpinLimit);
+    __syncwarp();
+    tc5::fence_after_sync();
+    if (!*s_abort) mma_s(0);
+    if (n_kt > 1) {
+      mbar_wait(bar(2), 0u, s_abort, p.err, kPfSpinLimit);
+      __syncwarp();
       tc5::fence_after_sync();
-      if (!*s_abort) mma_s(0);
-      if (n_kt > 1) {
-        mbar_wait(bar(2), 0u, s_abort, p.err, kPfSpinLimit);
-        tc5::fence_after_sync();
-        if (!*s_abort) mma_s(1);
-      }
-      for (int j = 0; j + 2 < n_kt && !*s_abort; ++j) {
-        const int st = j & 1;
-        // S_{j+2} overwrites the columns P_j is read from, so O += P V of tile j must have completed (the
-        // two products come from different threads and nothing but this barrier orders them); and its K
-        // tile must have landed.
-        mbar_wait(bar(1 + st), (uint32_t)(((j + 2) >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // (lands first: asked for when S_j completed)
-        mbar_wait(bar(10 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);
-        tc5::fence_after_sync();
-        if (!*s_abort) mma_s(j + 2);
-      }
-      if (*s_abort) {
-        atomicOr(p.stop, 1);
-        tc5::mma_commit(bar(14));
-        for (uint32_t w = 0; w < kPfSpinLimit; ++w)
-          if (mbar_try_wait(bar(14), 0u)) break;
-      }
+      if (!*s_abort) mma_s(1);
+    }
+    for (int j = 0; j + 2 < n_kt && !*s_abort; ++j) {
+      const int st = j & 1;
+      // S_{j+2} overwrites the columns P_j is read from, so O += P V of tile j must have completed (the
+      // two products come from different warps and nothing but this barrier orders them); and its K
+      // tile must have landed.
+      mbar_wait(bar(1 + st), (uint32_t)(((j + 2) >> 1) & 1), s_abort, p.err, kPfSpinLimit);  // (lands first: asked for when S_j completed)
+      mbar_wait(bar(10 + st), (uint32_t)((j >> 1) & 1), s_abort, p.err, kPfSpinLimit);
+      __syncwarp();
+      tc5::fence_after_sync();
+      if (!*s_abort) mma_s(j + 2);
+    }
+    if (*s_abort && tc5::elect_one()) {
+      atomicOr(p.stop, 1);
+      tc5::mma_commit(bar(14));
+      for (uint32_t w = 0; w < kPfSpinLimit; ++w)
+        if (mbar_try_wait(bar(14), 0u)) break;
     }
   } else {
     // ================= softmax warps: thread = query row = tensor-memory lane =================
