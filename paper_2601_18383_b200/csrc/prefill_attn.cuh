@@ -96,19 +96,49 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
   const int q_last = min(T - 1, q0 + kPfRows - 1);
   const int n_kt = q_last / kPfKeys + 1;  // key tiles up to the diagonal
 
+  // Set-up, spread over the warps so that the first tile loads are on their way as early as possible:
+  // the loading thread initialises the barriers its loads complete on and issues Q, K_0, V_0 (K_1, V_1)
+  // at once; thread 0 initialises the other barriers; warp 5 allocates the tensor memory.
+  const bool lead4 = warp == 4 && lane == 0;
+  auto load_k = [&](int j) {
+    const uint32_t dst = sK + (uint32_t)(j & 1) * kPfKvBytes;
+    mbar_arrive_expect_tx(bar(1 + (j & 1)), kPfKvBytes);
+    pf_tma_load(dst, &tmK, 0, j * kPfKeys, zkv, bar(1 + (j & 1)));
+    pf_tma_load(dst + kPfKvBytes / 2, &tmK, 64, j * kPfKeys, zkv, bar(1 + (j & 1)));
+  };
+  auto load_v = [&](int j) {
+    const uint32_t dst = sV + (uint32_t)(j & 1) * kPfKvBytes;
+    mbar_arrive_expect_tx(bar(3 + (j & 1)), kPfKvBytes);
+    pf_tma_load(dst, &tmV, 0, j * kPfKeys, zkv, bar(3 + (j & 1)));
+    pf_tma_load(dst + kPfKvBytes / 2, &tmV, 64, j * kPfKeys, zkv, bar(3 + (j & 1)));
+  };
+  if (lead4) {
+    for (int i = 0; i < 5; ++i) mbar_init(bar(i), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    if ((smem_u32(sm) & 1023u) == 0u) {  // (else the tiles would not be where the swizzle expects them: see below)
+      mbar_arrive_expect_tx(bar(0), kPfQBytes);
+      pf_tma_load(sQ, &tmQ, 0, q0, zq, bar(0));
+      pf_tma_load(sQ + kPfQBytes / 2, &tmQ, 64, q0, zq, bar(0));
+      load_k(0);
+      load_v(0);
+      if (n_kt > 1) {
+        load_k(1);
+        load_v(1);
+      }
+    }
+  }
   if (tid == 0) {
-    for (int i = 0; i < 15; ++i) mbar_init(bar(i), (i == 8 || i == 9) ? kPfRows : 1);
-    // (a launch whose waits run out must not take one time limit per CTA: the CTAs that start after the
-    // first one gave up see the word and skip their work)
-    *s_abort = *reinterpret_cast<volatile int*>(p.stop) != 0 ? 1 : 0;
-    if ((smem_u32(sm) & 1023u) != 0u) {  // the tiles would not be where the swizzle expects them
+    for (int i = 5; i < 15; ++i) mbar_init(bar(i), (i == 8 || i == 9) ? kPfRows : 1);
+    *s_abort = 0;
+    if ((smem_u32(sm) & 1023u) != 0u) {
       atomicOr(p.err, kErrStreamBounds);
       *s_abort = 1;
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 4) {
+  if (warp == 5) {
     tc5::tmem_alloc(smem_u32(s_tmem), kPfTmemCols);
     tc5::tmem_relinquish();
   }
@@ -121,32 +151,9 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
   if (warp == 4) {
     if (lane == 0) {
       // ================= the loading thread: TMA tile loads =================
-      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmQ)) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmK)) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmV)) : "memory");
-      auto load_k = [&](int j) {
-        const uint32_t dst = sK + (uint32_t)(j & 1) * kPfKvBytes;
-        mbar_arrive_expect_tx(bar(1 + (j & 1)), kPfKvBytes);
-        pf_tma_load(dst, &tmK, 0, j * kPfKeys, zkv, bar(1 + (j & 1)));
-        pf_tma_load(dst + kPfKvBytes / 2, &tmK, 64, j * kPfKeys, zkv, bar(1 + (j & 1)));
-      };
-      auto load_v = [&](int j) {
-        const uint32_t dst = sV + (uint32_t)(j & 1) * kPfKvBytes;
-        mbar_arrive_expect_tx(bar(3 + (j & 1)), kPfKvBytes);
-        pf_tma_load(dst, &tmV, 0, j * kPfKeys, zkv, bar(3 + (j & 1)));
-        pf_tma_load(dst + kPfKvBytes / 2, &tmV, 64, j * kPfKeys, zkv, bar(3 + (j & 1)));
-      };
-      if (!*s_abort) {
-        mbar_arrive_expect_tx(bar(0), kPfQBytes);
-        pf_tma_load(sQ, &tmQ, 0, q0, zq, bar(0));
-        pf_tma_load(sQ + kPfQBytes / 2, &tmQ, 64, q0, zq, bar(0));
-        load_k(0);
-        load_v(0);
-        if (n_kt > 1) {
-          load_k(1);
-          load_v(1);
-        }
-      }
+      // (A launch whose waits run out must not take one time limit per CTA: the CTAs that start after the
+      // first one gave up see the stop word here and skip the rest; their waits are bounded anyway.)
+      if (*reinterpret_cast<volatile int*>(p.stop) != 0) *s_abort = 1;
       // A stage is requested again as soon as the product that read it has completed: K of tile j + 2
       // after S_j, V of tile j + 1 after O += P V of tile j - 1.  (Neither of these per-stage barriers
       // can run two phases ahead of this thread: the product that would complete the next phase needs
@@ -332,26 +339,30 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
     __nv_bfloat16* orow = p.out + ((size_t)zq * T + (size_t)min(qpos, T - 1)) * 128;
     const bool aborted = *s_abort != 0;  // (then tensor memory may not hold what this row expects: nothing is written)
 #pragma unroll
-    for (int c0 = 0; c0 < 128; c0 += 32) {
-      uint32_t o[32];
-      tc5::tmem_ld32(tO + lane_base + (uint32_t)c0, o);
+    for (int c0 = 0; c0 < 128; c0 += 64) {
+      uint32_t o[2][32];
+      tc5::tmem_ld32(tO + lane_base + (uint32_t)c0, o[0]);
+      tc5::tmem_ld32(tO + lane_base + (uint32_t)c0 + 32u, o[1]);
       tc5::tmem_wait_ld();
       if (qpos < T && !aborted) {
 #pragma unroll
-        for (int c = 0; c < 32; c += 8) {
-          uint4 w;
-          w.x = pack_bf16x2(__uint_as_float(o[c]) * inv_l, __uint_as_float(o[c + 1]) * inv_l);
-          w.y = pack_bf16x2(__uint_as_float(o[c + 2]) * inv_l, __uint_as_float(o[c + 3]) * inv_l);
-          w.z = pack_bf16x2(__uint_as_float(o[c + 4]) * inv_l, __uint_as_float(o[c + 5]) * inv_l);
-          w.w = pack_bf16x2(__uint_as_float(o[c + 6]) * inv_l, __uint_as_float(o[c + 7]) * inv_l);
-          *reinterpret_cast<uint4*>(orow + c0 + c) = w;
+        for (int hh = 0; hh < 2; ++hh) {
+#pragma unroll
+          for (int c = 0; c < 32; c += 8) {
+            uint4 w;
+            w.x = pack_bf16x2(__uint_as_float(o[hh][c]) * inv_l, __uint_as_float(o[hh][c + 1]) * inv_l);
+            w.y = pack_bf16x2(__uint_as_float(o[hh][c + 2]) * inv_l, __uint_as_float(o[hh][c + 3]) * inv_l);
+            w.z = pack_bf16x2(__uint_as_float(o[hh][c + 4]) * inv_l, __uint_as_float(o[hh][c + 5]) * inv_l);
+            w.w = pack_bf16x2(__uint_as_float(o[hh][c + 6]) * inv_l, __uint_as_float(o[hh][c + 7]) * inv_l);
+            *reinterpret_cast<uint4*>(orow + c0 + 32 * hh + c) = w;
+          }
         }
       }
     }
   }
   tc5::fence_before_sync();
   __syncthreads();
-  if (warp == 4) tc5::tmem_dealloc(tmem, kPfTmemCols);
+  if (warp == 5) tc5::tmem_dealloc(tmem, kPfTmemCols);
 }
 
 }  // namespace dynts
