@@ -419,6 +419,8 @@ def run_ours(args, cfg, rank, world, device):
     prefill = None
     if rank == 0 and world == 1 and cfg.dtype == "bf16" and cfg.head_dim == 128 and not args.no_extras:
         prefill = time_prefill(cfg, device)
+        prefill["long_prompt"] = {k: v for k, v in time_prefill(cfg, device, prompt=4096).items()
+                                  if k in ("prompt_tokens", "layers_timed", "us_per_call", "flops", "achieved", "frac")}
 
     # ---- CPU baseline: the oracle, as it stands, on this machine's host cores (rank 0, N = 1) ------
     cpu = None
@@ -474,13 +476,18 @@ def time_predictor(batch, device, peak, d=4096, iters=40):
             "achieved": round(gbs, 1), "peak": peak, "unit": "GB/s", "frac": round(gbs / peak, 4)}
 
 
-def time_prefill(cfg, device, iters=10):
+def time_prefill(cfg, device, iters=10, prompt=None):
     """Times the prompt attention (dynts_prompt_attn: Eq. 4-5 over the workload's prompt, all heads of
     up to 8 layers; the fill of the slabs is not part of it); flops = 4 d per (query, key) pair of the
-    causal triangle; peak = the measured dense bf16 GEMM rate."""
+    causal triangle; peak = the measured dense bf16 GEMM rate.  With `prompt`, the same heads on a
+    prompt of that length, the batch shrunk to keep the token count (the long-prompt regime, where the
+    per-tile rate shows rather than the fill and drain of the short items)."""
     import torch
     import paper_2601_18383_b200 as D
     sub = cfg.scaled(layers=min(cfg.layers, 8), seq_budgets=None, budget=max(cfg.budget, cfg.prompt))
+    if prompt is not None:
+        batch = max(1, min(cfg.batch, cfg.batch * cfg.prompt // prompt))
+        sub = sub.scaled(prompt=prompt, batch=batch, budget=max(cfg.budget, prompt))
     T = sub.prompt
     cache = D.Cache(sub.layers, sub.batch, sub.q_heads, sub.kv_heads, sub.head_dim, sub.budget, sub.window, sub.evict_interval,
                     dtype="bf16", device=device)
@@ -673,6 +680,8 @@ def main():
         peak, _ = measured_peaks()
         res = {"config": workload_config(cfg, args, world), "predictor_mlp": time_predictor(cfg.batch, device, peak),
                "prefill_attn": time_prefill(cfg, device) if cfg.dtype == "bf16" and cfg.head_dim == 128 else None}
+        if res["prefill_attn"]:
+            res["prefill_attn"]["long_prompt"] = time_prefill(cfg, device, prompt=4096)
     else:
         res = run_ours(args, cfg, rank, world, device)
     if rank == 0:

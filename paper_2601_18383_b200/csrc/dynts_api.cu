@@ -835,8 +835,9 @@ dynts_status_t prompt_attn(dynts_cache* c, const void* q, const void* k, const v
   dynts_status_t st = materialise(c);
   if (st != DYNTS_OK) return st;
   const long long lb = (long long)n_layers * c->cfg.batch;
-  if (lb > 65535 || (long long)n_tokens * 256 >= (1ll << 40))
-    return fail(DYNTS_ERR_INVALID_ARG, "layers x batch %lld or n_tokens %d beyond the launch limits", lb, n_tokens);
+  const long long n_qt = (n_tokens + dynts::kPfRows - 1) / dynts::kPfRows;
+  if (lb * c->cfg.q_heads * n_qt >= (1ll << 30) || (long long)n_tokens * 256 >= (1ll << 40))
+    return fail(DYNTS_ERR_INVALID_ARG, "layers x batch %lld with n_tokens %d beyond the launch limits", lb, n_tokens);
   if (!c->attr_prefill) {
     CUDA_TRY(cudaFuncSetAttribute(dynts::prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dynts::kPfSmemBytes));
     c->attr_prefill = true;
@@ -869,8 +870,12 @@ dynts_status_t prompt_attn(dynts_cache* c, const void* q, const void* k, const v
   p.T = n_tokens;
   p.Hq = c->cfg.q_heads;
   p.Hkv = c->cfg.kv_heads;
+  p.n_qt = (int)n_qt;
+  p.n_heads = (int)(lb * c->cfg.q_heads);
   p.scale_log2 = (float)(1.4426950408889634 / std::sqrt(128.0));
-  const dim3 grid((unsigned)((n_tokens + dynts::kPfRows - 1) / dynts::kPfRows), (unsigned)c->cfg.q_heads, (unsigned)lb);
+  // two CTAs per SM (what their shared memory allows), each looping over its share of the (query tile, head) items
+  const long long n_work = n_qt * p.n_heads;
+  const unsigned grid = (unsigned)std::min<long long>(n_work, 2ll * c->sm_count);
   dynts::prefill_attn_kernel<<<grid, dynts::kPfThreads, dynts::kPfSmemBytes, c->stream>>>(p, mq, mk, mv);
   CUDA_TRY(cudaGetLastError());
   c->launches += 1;
