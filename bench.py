@@ -33,7 +33,7 @@ UNIT = "tokens/s"
 BYTES_PER_SLOT = 520          # K row 256 + V row 256 + fp32 score read-modify-write 8 (bf16 d=128, fp32 d=64)
 # DRAM bytes moved per algorithmic byte by the decode kernel, from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of one launch / its algorithmic bytes).
-NCU_TRAFFIC_RATIO = 1.070
+NCU_TRAFFIC_RATIO = 1.067
 
 
 def measured_peaks():
