@@ -380,14 +380,14 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
         for (int c = 1; c < 32; ++c)
           if (c > lane) s_hi[c] = 0xff800000u;
       }
-      auto max_half = [](const uint32_t (&sv)[32]) {
+      auto max_half = [](const uint32_t (&sv)[32]) {  // four chains of three-input maxima
         float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-        for (int c = 0; c < 32; c += 4) {
+        for (int c = 0; c < 32; c += 8) {
 #pragma unroll
-          for (int u = 0; u < 4; ++u) mx4[u] = fmaxf(mx4[u], __uint_as_float(sv[c + u]));
+          for (int u = 0; u < 4; ++u) mx4[u] = tc5::f_max3(mx4[u], __uint_as_float(sv[c + u]), __uint_as_float(sv[c + 4 + u]));
         }
-        return fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        return tc5::f_max3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]);
       };
       float mxr = -CUDART_INF_F;
       if (lo_live) mxr = max_half(s_lo);
@@ -402,16 +402,20 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
       const float neg_m = -m_new;
       const float scale_log2 = p.scale_log2;
       uint32_t pk[32];  // the row's 64 weights as bf16 pairs
-      auto exp_half = [neg_m, scale_log2](const uint32_t (&sv)[32], uint32_t* out) {
-        float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      const uint64_t scale2 = tc5::f2_pack(scale_log2, scale_log2), negm2 = tc5::f2_pack(neg_m, neg_m);
+      auto exp_half = [scale2, negm2](const uint32_t (&sv)[32], uint32_t* out) {
+        uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};  // four chains of (even, odd) column sums
 #pragma unroll
         for (int c = 0; c < 16; ++c) {
-          const float a0 = fast_exp2(fmaf(__uint_as_float(sv[2 * c]), scale_log2, neg_m));
-          const float a1 = fast_exp2(fmaf(__uint_as_float(sv[2 * c + 1]), scale_log2, neg_m));
-          sum4[c & 3] += a0 + a1;
+          float x0, x1;
+          tc5::f2_unpack(tc5::f2_fma(tc5::f2_pack(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1])), scale2, negm2), x0, x1);
+          const float a0 = fast_exp2(x0), a1 = fast_exp2(x1);
+          sum2[c & 3] = tc5::f2_add(sum2[c & 3], tc5::f2_pack(a0, a1));
           out[c] = pack_bf16x2(a0, a1);
         }
-        return (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+        float e, o;
+        tc5::f2_unpack(tc5::f2_add(tc5::f2_add(sum2[0], sum2[1]), tc5::f2_add(sum2[2], sum2[3])), e, o);
+        return e + o;
       };
       float sum = 0.f;
       if (lo_live) {
@@ -456,6 +460,7 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
     mbar_wait(bar(12), (uint32_t)(it & 1), s_abort, p.err, kPfSpinLimit);
     tc5::fence_after_sync();
     const float inv_l = 1.0f / l;
+    const uint64_t inv2 = tc5::f2_pack(inv_l, inv_l);
     const bool aborted = *s_abort != 0;  // (then tensor memory may not hold what this row expects: nothing is written)
     // Half a row (64 columns, 128 bytes) at a time goes through the warp's staging tile so that the
     // global stores are whole 128-byte lines: a thread writes its half row as eight 16-byte chunks,
@@ -475,13 +480,15 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
       for (int hh = 0; hh < 2; ++hh) {
 #pragma unroll
         for (int c = 0; c < 32; c += 8) {
-          uint4 w;
-          w.x = pack_bf16x2(__uint_as_float(o[hh][c]) * inv_l, __uint_as_float(o[hh][c + 1]) * inv_l);
-          w.y = pack_bf16x2(__uint_as_float(o[hh][c + 2]) * inv_l, __uint_as_float(o[hh][c + 3]) * inv_l);
-          w.z = pack_bf16x2(__uint_as_float(o[hh][c + 4]) * inv_l, __uint_as_float(o[hh][c + 5]) * inv_l);
-          w.w = pack_bf16x2(__uint_as_float(o[hh][c + 6]) * inv_l, __uint_as_float(o[hh][c + 7]) * inv_l);
+          uint32_t w[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            float y0, y1;
+            tc5::f2_unpack(tc5::f2_mul(tc5::f2_pack(__uint_as_float(o[hh][c + 2 * u]), __uint_as_float(o[hh][c + 2 * u + 1])), inv2), y0, y1);
+            w[u] = pack_bf16x2(y0, y1);
+          }
           const int chunk = 4 * hh + (c >> 3);
-          *reinterpret_cast<uint4*>(stage + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = w;
+          *reinterpret_cast<uint4*>(stage + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
       __syncwarp();
