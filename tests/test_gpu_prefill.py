@@ -43,6 +43,28 @@ def test_prefill_attention_matches_oracle(T, G):
     gpu.close()
 
 
+@pytest.mark.parametrize("T", [130, 320])
+def test_prefill_attention_with_several_items_per_cta(T):
+    """More (query tile, head) items than the grid has CTAs (two per SM): every CTA walks several
+    items back to back -- the loads and the first product of the next item are issued while the
+    current one is still in the softmax, half the grid walks its list backwards -- and every row
+    still matches the oracle."""
+    cfg = W.get_config("c3_qwen7b").scaled(layers=3, batch=4, prompt=T, budget=max(T, 64), window=8, evict_interval=16)
+    n_items = -(-T // 128) * cfg.layers * cfg.batch * cfg.q_heads
+    assert n_items > 2 * 2 * torch.cuda.get_device_properties(0).multi_processor_count
+    q, k, v = _qkv(cfg, T, 90 + T)
+    gpu = H.make_gpu(cfg)
+    out = torch.full((cfg.layers, cfg.batch, cfg.q_heads, T, 128), float("nan"), dtype=torch.bfloat16, device="cuda:0")
+    gpu.prompt_attn(H.dev(q, cfg), H.dev(k, cfg), H.dev(v, cfg), out)
+    gpu.synchronize()
+    gpu.poll_error()
+    ref = O.prefill_attention(q, k, v)
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert H.rel_err_vectors(got, ref) <= H.TOL_OUT["bf16"]
+    gpu.close()
+
+
 def test_decode_after_prefill_attention_continues_the_sequence():
     """The last prefill row and the first decode step are the same operation on consecutive
     tokens: run prefill over T tokens, then decode token T + 1, and compare both with a prefill
