@@ -107,6 +107,29 @@ def physical_gpu_index(local_index: int) -> int:
     return local_index
 
 
+def rank_seed(cfg, rank):
+    """Seed of a rank's synthetic cache: every rank holds its own batch of the workload (independent
+    sequences, sharded over the ranks with no exchange between them)."""
+    return 1000 * int(cfg.name[1]) + rank
+
+
+def max_over_ranks(x, world, device=None):
+    """The slowest rank's time: what the whole job took (an all-reduce over the process group; the
+    only collective of the benchmark, and none of the data path's)."""
+    if world == 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(batch, steps, world, seconds):
+    """Tokens per second of the whole job: every rank decodes `batch` sequences for `steps` steps."""
+    return batch * steps * world / seconds
+
+
 def workload_config(cfg, args, world):
     """The `config` object of the JSON line: a description of the workload that both arms print
     alike (nothing in it depends on which implementation ran)."""
@@ -158,7 +181,7 @@ def run_ours(args, cfg, rank, world, device):
     kv8 = args.kv_dtype == "fp8"
     if kv8 and (cfg.dtype != "bf16" or cfg.head_dim % 16):
         raise SystemExit("--kv-dtype fp8 needs a bf16 workload")
-    seed = 1000 * int(cfg.name[1]) + rank
+    seed = rank_seed(cfg, rank)
     # one set of planted directions for the steady-state fill and for the decode queries
     u = gen.torch_unit_dirs(cfg, seed, device) if cfg.dist == "planted" else None
     cache = setup_cache(cfg, seed, device, kv8, u=u)
@@ -240,12 +263,8 @@ def run_ours(args, cfg, rank, world, device):
     launches = cache.launch_count() - launches0
     evictions_in_region = state["evictions"] - ev_before
     cache.poll_error()
-    if world > 1:
-        t = torch.tensor([ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    tokens = cfg.batch * K * world
-    value = tokens / (ms * 1e-3)
+    ms = max_over_ranks(ms, world, device)
+    value = job_throughput(cfg.batch, K, world, ms * 1e-3)
 
     # ---- per-kernel durations: whole eviction cycles, whatever K is -------------------------------
     # Every cycle is E back-to-back decode launches (one event pair around the run, so the average
@@ -346,10 +365,7 @@ def run_ours(args, cfg, rank, world, device):
         sus_clk = sus_sampler.stop()
         ends = [marks[0].elapsed_time(m) for m in marks[1:]]            # ms since the start, on the device
         total_ms = ends[-1]
-        if world > 1:
-            t = torch.tensor([total_ms], device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            total_ms = float(t.item())
+        total_ms = max_over_ranks(total_ms, world, device)
         # each cycle is attributed to the clock sample nearest to its middle, then binned by 50 MHz
         bins = {}
         if sus_sampler.samples:
@@ -400,11 +416,8 @@ def run_ours(args, cfg, rank, world, device):
                 e2e_evictions += 1
         torch.cuda.synchronize(device)
         dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
-        e2e = {"value": round(cfg.batch * Ke * world / dt, 1), "unit": UNIT,
+        dt = max_over_ranks(dt, world, device)
+        e2e = {"value": round(job_throughput(cfg.batch, Ke, world, dt), 1), "unit": UNIT,
                "h2d_bytes_per_step": int(hq[0].numel() * hq[0].element_size() + 2 * hk[0].numel() * hk[0].element_size()),
                "d2h_bytes_per_step": int(hout.numel() * hout.element_size()), "steps": Ke, "evictions": e2e_evictions,
                "api": "dynts_decode_attn_host every step + dynts_evict every %d steps" % E}
