@@ -13,7 +13,7 @@ step at the end, the length / time sawtooth per 64-step chunk (beside Section 5'
 the length), peak KV rows and bytes; across arms: speed-up, KV memory ratio and Appendix A's
 attention-flop ratio.
 
-    python bench_model.py [--tokens 4096] [--budget 3072] [--out gpurun_out/model_loop.json]
+    python bench_model.py [--tokens 4096] [--budget 3072] [--out model_loop.json]
 
 `--late-state` instead times 128 steps in the state a 16384-token decode reaches, the caches
 filled with seeded synthetic K/V rows (no trajectory, no evictions falling due).

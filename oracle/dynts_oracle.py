@@ -11,7 +11,7 @@ What each function follows in the paper:
   included) and Eq. 5 (weighted sum of values).
 * ``decode_step`` (delta/score part) -- Eq. 6: a token's importance is the attention it receives
   summed over query rows.  Here the rows are the decode queries seen so far, summed over the
-  query heads that share the KV head (Appendix B.1 aggregates heads; sum is this build's reading).
+  query heads that share the KV head (Appendix B.1 aggregates heads; sum is the reading taken here).
 * ``prefill_attention`` -- the same Eq. 4-5 for every prompt position (the prefill phase that fills
   the question window of Section 4.2).
 * ``select_keep`` / ``evict`` -- Section 4.2: the question window (the first M rows) and the local
@@ -374,7 +374,7 @@ def predictor_mlp(h: np.ndarray, W1, b1, W2, b2, W3, b3, activation: str = "none
     """Importance Predictor head (Section 4.1, Appendix A): a three-layer MLP d -> 2d -> d/2 -> 1 on
     the final hidden state h [Nb, d]; returns one score per sequence, float64.  W_i is [out, in].
     The paper calls the layers linear and names no activation; ``activation`` ("none" or "relu",
-    applied after the first two layers) is this build's parameter."""
+    applied after the first two layers) is a parameter of this library."""
     act = (lambda x: x) if activation == "none" else (lambda x: np.maximum(x, 0.0))
     x = np.asarray(h, dtype=np.float64)
     y1 = act(x @ np.asarray(W1, dtype=np.float64).T + np.asarray(b1, dtype=np.float64))
@@ -386,7 +386,7 @@ def predictor_mlp(h: np.ndarray, W1, b1, W2, b2, W3, b3, activation: str = "none
 def paper_target(M: int, B: int, W_l: int, ratio: float) -> int:
     """Rows kept by one selection of Section 4.2: the question window (M rows), the local window
     (W_l rows) and the top ratio * W_s rows of the selection window, W_s = B - M - W_l.  The paper
-    does not say how ratio * W_s is rounded; this build rounds down."""
+    does not say how ratio * W_s is rounded; it is rounded down here."""
     W_s = B - M - W_l
     if W_s < 0:
         raise ValueError("question window + local window exceed the budget")

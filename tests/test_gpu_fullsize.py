@@ -109,7 +109,7 @@ def test_config4_full_size_ragged():
 def test_config5_attention_shapes_layer_by_layer():
     """The attention part of the full-model configuration (32 layers, 32/8 heads, batch 8, budget
     3072), driven the way a model drives it: one call per layer.  Window 128 and interval 64 are
-    this build's reading (the configuration names neither)."""
+    the reading taken here (the configuration names neither)."""
     cfg = W.get_config("c2_llama8b").scaled(name="c5_attn", batch=8, budget=3072, window=128, evict_interval=64,
                                              prompt=256, density=0.03)
     gpu = _steady_state(cfg, 5100, cfg.capacity - 2)

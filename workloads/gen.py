@@ -74,8 +74,8 @@ CONFIGS = {
     "c2_llama8b": WorkloadConfig("c2_llama8b", 32, 1, 32, 8, 128, 256, 16384, 2048, 128, 64, "bf16", "planted", 0.05),
     # Qwen-7B-shaped attention stack, batch 16
     "c3_qwen7b": WorkloadConfig("c3_qwen7b", 28, 16, 28, 4, 128, 512, 32768, 4096, 256, 128, "bf16", "planted", 0.02),
-    # ragged throughput batch with Llama-8B attention shapes; prompt 256 and window 128 are this
-    # build's choice (the workload statement leaves them open)
+    # ragged throughput batch with Llama-8B attention shapes; prompt 256 and window 128 are chosen
+    # here (the workload statement leaves them open)
     "c4_ragged": WorkloadConfig("c4_ragged", 32, 64, 32, 8, 128, 256, 32768, 3072, 128, 64, "bf16", "student_t", 0.0,
                                 seq_budgets=_RB, seq_decode_steps=_RS),
 }
