@@ -348,6 +348,57 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
   } else {
     // ================= softmax warps: thread = query row = tensor-memory lane =================
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    // epilogue of an item: the row of O, normalised, rounded to bf16.  (A barrier of its own, one phase per
+    // item: the next item's first O = P V, which would complete the phase after, waits for the P this
+    // thread writes once it has read its row of O here.)
+    auto epilogue = [&](float l, int q0, int zq, int it) {
+    mbar_wait(bar(12), (uint32_t)(it & 1), s_abort, p.err, kPfSpinLimit);
+    tc5::fence_after_sync();
+    const float inv_l = 1.0f / l;
+    const uint64_t inv2 = tc5::f2_pack(inv_l, inv_l);
+    const bool aborted = *s_abort != 0;  // (then tensor memory may not hold what this row expects: nothing is written)
+    // Half a row (64 columns, 128 bytes) at a time goes through the warp's staging tile so that the
+    // global stores are whole 128-byte lines: a thread writes its half row as eight 16-byte chunks,
+    // chunk c at position c ^ (row & 7) (conflict-free), then every eight lanes read one row back and
+    // store it.  (Stored straight from the registers, a warp's store touched 32 different lines, and
+    // the 16 of them took 1.4 us per item.)
+    uint8_t* stage = s_out + warp * (32 * 128);
+    __nv_bfloat16* obase = p.out + ((size_t)zq * T + (size_t)(q0 + warp * 32)) * 128;
+    const int rows_here = T - (q0 + warp * 32);  // rows of this warp inside the prompt (may be <= 0 or > 32)
+#pragma unroll
+    for (int c0 = 0; c0 < 128; c0 += 64) {
+      uint32_t o[2][32];
+      tc5::tmem_ld32(tO + lane_base + (uint32_t)c0, o[0]);
+      tc5::tmem_ld32(tO + lane_base + (uint32_t)c0 + 32u, o[1]);
+      tc5::tmem_wait_ld();
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+#pragma unroll
+        for (int c = 0; c < 32; c += 8) {
+          uint32_t w[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            float y0, y1;
+            tc5::f2_unpack(tc5::f2_mul(tc5::f2_pack(__uint_as_float(o[hh][c + 2 * u]), __uint_as_float(o[hh][c + 2 * u + 1])), inv2), y0, y1);
+            w[u] = pack_bf16x2(y0, y1);
+          }
+          const int chunk = 4 * hh + (c >> 3);
+          *reinterpret_cast<uint4*>(stage + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      __syncwarp();
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int row = 4 * i + (lane >> 3), chunk = lane & 7;
+        const uint4 w = *reinterpret_cast<const uint4*>(stage + row * 128 + ((chunk ^ (row & 7)) << 4));
+        if (row < rows_here && !aborted) *reinterpret_cast<uint4*>(obase + (size_t)row * 128 + c0 + chunk * 8) = w;
+      }
+      __syncwarp();
+    }
+    };
+    bool ep_on = false;  // an item whose epilogue is still to run, and what it needs
+    float ep_l = 0.f;
+    int ep_q0 = 0, ep_zq = 0, ep_it = 0;
     PfCursor cur = first;
     int g = 0;  // flat tile index: S buffer g & 1
     while (cur.it < n_items) {
@@ -447,6 +498,13 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
           tc5::tmem_st32(tO + lane_base + (uint32_t)c0, o);
         }
       }
+      // At the first tile of an item the epilogue of the item before is still to run: its last
+      // O += P V has had the time of this tile's row arithmetic to complete, and the first O = P V of
+      // this item, which overwrites O, cannot be issued before the P stored below.
+      if (ep_on) {
+        epilogue(ep_l, ep_q0, ep_zq, ep_it);
+        ep_on = false;
+      }
       // the row of P over the first 32 columns of the S tile it was computed from (this thread has read
       // its row of S; nothing else reads that buffer before the product that follows)
       tc5::tmem_st32(tS0 + lane_base + 64u * (uint32_t)(g & 1), pk);
@@ -454,54 +512,16 @@ prefill_attn_kernel(const PrefillAttnParams p, const __grid_constant__ CUtensorM
       tc5::fence_before_sync();
       mbar_arrive(bar(8 + (g & 1)));
     }
-    // epilogue: the row of O, normalised, rounded to bf16.  (A barrier of its own, one phase per item: the
-    // next item's first O = P V, which would complete the phase after, waits for the P this thread writes
-    // once it has read its row of O here.)
-    mbar_wait(bar(12), (uint32_t)(it & 1), s_abort, p.err, kPfSpinLimit);
-    tc5::fence_after_sync();
-    const float inv_l = 1.0f / l;
-    const uint64_t inv2 = tc5::f2_pack(inv_l, inv_l);
-    const bool aborted = *s_abort != 0;  // (then tensor memory may not hold what this row expects: nothing is written)
-    // Half a row (64 columns, 128 bytes) at a time goes through the warp's staging tile so that the
-    // global stores are whole 128-byte lines: a thread writes its half row as eight 16-byte chunks,
-    // chunk c at position c ^ (row & 7) (conflict-free), then every eight lanes read one row back and
-    // store it.  (Stored straight from the registers, a warp's store touched 32 different lines, and
-    // the 16 of them took 1.4 us per item.)
-    uint8_t* stage = s_out + warp * (32 * 128);
-    __nv_bfloat16* obase = p.out + ((size_t)zq * T + (size_t)(q0 + warp * 32)) * 128;
-    const int rows_here = T - (q0 + warp * 32);  // rows of this warp inside the prompt (may be <= 0 or > 32)
-#pragma unroll
-    for (int c0 = 0; c0 < 128; c0 += 64) {
-      uint32_t o[2][32];
-      tc5::tmem_ld32(tO + lane_base + (uint32_t)c0, o[0]);
-      tc5::tmem_ld32(tO + lane_base + (uint32_t)c0 + 32u, o[1]);
-      tc5::tmem_wait_ld();
-#pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-#pragma unroll
-        for (int c = 0; c < 32; c += 8) {
-          uint32_t w[4];
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            float y0, y1;
-            tc5::f2_unpack(tc5::f2_mul(tc5::f2_pack(__uint_as_float(o[hh][c + 2 * u]), __uint_as_float(o[hh][c + 2 * u + 1])), inv2), y0, y1);
-            w[u] = pack_bf16x2(y0, y1);
-          }
-          const int chunk = 4 * hh + (c >> 3);
-          *reinterpret_cast<uint4*>(stage + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-        }
-      }
-      __syncwarp();
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int row = 4 * i + (lane >> 3), chunk = lane & 7;
-        const uint4 w = *reinterpret_cast<const uint4*>(stage + row * 128 + ((chunk ^ (row & 7)) << 4));
-        if (row < rows_here && !aborted) *reinterpret_cast<uint4*>(obase + (size_t)row * 128 + c0 + chunk * 8) = w;
-      }
-      __syncwarp();
-    }
+    // The item's epilogue is run inside the first tile of the next item (see above): the weights of
+    // that tile are computed while the last O += P V of this item completes.
+    ep_on = true;
+    ep_l = l;
+    ep_q0 = q0;
+    ep_zq = zq;
+    ep_it = it;
     pf_seek(cur, it + 1, n_items, p);
     }  // items
+    if (ep_on) epilogue(ep_l, ep_q0, ep_zq, ep_it);
   }
   tc5::fence_before_sync();
   __syncthreads();
