@@ -65,6 +65,34 @@ def test_prefill_attention_with_several_items_per_cta(T):
     gpu.close()
 
 
+@pytest.mark.parametrize("T", [200, 512])
+def test_prefill_attention_when_the_row_maximum_keeps_moving(T):
+    """Keys whose norm grows along the prompt: the largest logit of a row sits in its latest tiles and
+    exceeds the maximum of the tiles before by far more than the slack the kernel allows its
+    reference maximum (2^8), so the accumulated output and sum are rescaled again and again."""
+    cfg = W.get_config("c2_llama8b").scaled(layers=1, batch=2, kv_heads=2, q_heads=8, prompt=T, budget=max(T, 64),
+                                             window=8, evict_interval=16)
+    q, k, v = _qkv(cfg, T, 300 + T)
+    grow = (1.0 + np.arange(T) / 16.0)[None, None, None, :, None]
+    k = W.to_cache_dtype(k * grow, "bf16")
+    ref = O.prefill_attention(q, k, v)
+    # the recipe does what it says: along the last row, a later tile of 64 keys tops everything before it
+    # by more than 8 in base-2 units at least once
+    qh, kh = q[0, 0, 0].astype(np.float64), k[0, 0, 0].astype(np.float64)
+    lg = (qh[T - 1] @ kh.T) / np.sqrt(128.0) * np.log2(np.e)
+    tile_max = [lg[j:j + 64].max() for j in range(0, T, 64)]
+    assert any(tile_max[j] > max(tile_max[:j]) + 8 for j in range(1, len(tile_max)))
+    gpu = H.make_gpu(cfg)
+    out = torch.full((cfg.layers, cfg.batch, cfg.q_heads, T, 128), float("nan"), dtype=torch.bfloat16, device="cuda:0")
+    gpu.prompt_attn(H.dev(q, cfg), H.dev(k, cfg), H.dev(v, cfg), out)
+    gpu.synchronize()
+    gpu.poll_error()
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert H.rel_err_vectors(got, ref) <= H.TOL_OUT["bf16"]
+    gpu.close()
+
+
 def test_decode_after_prefill_attention_continues_the_sequence():
     """The last prefill row and the first decode step are the same operation on consecutive
     tokens: run prefill over T tokens, then decode token T + 1, and compare both with a prefill
