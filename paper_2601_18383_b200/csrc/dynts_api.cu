@@ -427,6 +427,14 @@ dynts_status_t launch_decode(dynts_cache* c, int layer0, int n_layers, const voi
       if (uniform && (kv8 ? (nearly_all || (mostly && per <= 2)) : mostly)) {
         p.slabs_per_cta = (int)per;
         ctas = (int)used;
+      } else if (!kv8 && c->cluster == 0 && slabs <= c->sm_count) {
+        // Fewer slabs than SMs (one layer of a small batch): every slab is shared by several CTAs
+        // however the list is cut.  One CTA per SM then halves the partial results per slab, and
+        // the CTAs of the next launch in the stream find room to become resident and run their
+        // set-up during this launch's tail.  (64 slabs of 3080 rows: 31.0 us per launch against
+        // 34.3 us with two CTAs per SM, the best of 64..296 CTAs; 116 against 133 us at 16500
+        // rows; from 192 slabs on two per SM are faster again.)
+        ctas = std::min(ctas, c->sm_count);
       }
     }
     // The score pass of every CTA's last slab moves into the next launch when the pieces are whole
